@@ -1,0 +1,134 @@
+"""Pins for the merge-weight, merge and unmerge oracle (Sec. 4.2) and the block loop."""
+import math
+
+import numpy as np
+import pytest
+
+import gen
+from oracle import toma_oracle as O
+
+
+def test_scale_and_softmax_axis_closed_form():
+    # d = 4, tau = 0.5  =>  tau*sqrt(d) = 1: logits are plain dot products
+    x = np.array([[1.0, 0, 0, 0],          # destination 0
+                  [0, 1.0, 0, 0],          # destination 1
+                  [math.log(3.0), 0, 0, 0]])  # a source: logits (ln 3, 0) -> shares (3/4, 1/4)
+    idx = np.array([0, 1])
+    for tau, share in ((0.5, 3 / 4), (0.25, 9 / 10)):  # halving tau doubles the logits
+        L = x[idx] @ x.T / (tau * 2.0)
+        A = np.exp(L) / np.exp(L).sum(axis=0, keepdims=True)
+        w = O.merge_weights(x, idx, tau)
+        assert A[0, 2] == pytest.approx(share)
+        # undo the row normalisation with the closed-form row sums
+        assert w[0, 2] == pytest.approx(share / A[0].sum())
+        assert w[1, 2] == pytest.approx((1 - share) / A[1].sum())
+
+
+def test_weight_invariants_on_a_real_tile():
+    c = gen.config("cfg2", batch=1)
+    x = gen.features(c)[0]
+    tile = O.split_regions(x, c.grid_h, c.grid_w, c.tile_h, c.tile_w)[7]
+    idx, _ = O.select_tile(tile, c.d_loc)
+    w = O.merge_weights(tile, idx, c.tau)
+    assert w.shape == (c.d_loc, c.n_loc)
+    assert np.all(w >= 0)
+    assert np.allclose(w.sum(axis=1), 1.0, atol=1e-12)          # merge rows sum to 1
+    Z = 1.0 / w[np.arange(c.d_loc), idx]                          # not used further; rows are positive
+    assert np.all(np.isfinite(Z))
+    # before row normalisation every source's shares sum to 1: recover A = w * Z_row
+    xs = tile.astype(np.float64)
+    L = xs[idx] @ xs.T / (c.tau * math.sqrt(c.dim))
+    A = np.exp(L - L.max(0)) / np.exp(L - L.max(0)).sum(0)
+    assert np.allclose(A.sum(axis=0), 1.0)
+    assert np.allclose(w, A / A.sum(1, keepdims=True))
+
+
+def test_orthogonal_groups_give_group_means():
+    d, groups, rep = 16, 4, 3
+    protos = np.eye(d)[:groups] * 3.0
+    x = np.repeat(protos, rep, axis=0)
+    x = x + 0.01 * np.arange(x.size).reshape(x.shape) / x.size  # break exact duplication a little
+    idx, _ = O.select_tile(x, groups)
+    w = O.merge_weights(x, idx, 0.05)  # cold softmax: hard assignment
+    member = np.repeat(np.arange(groups), rep)
+    want = np.zeros((groups, groups * rep))
+    for g in range(groups):
+        want[g, member == g] = 1.0 / rep
+    order = np.argsort(idx)  # destinations come in pick order; compare group-wise
+    assert np.allclose(w[order], want, atol=1e-6)
+    merged = O.merge(w, x)
+    for j, g in enumerate(member[idx]):
+        assert np.allclose(merged[j], x[member == g].mean(axis=0), atol=1e-5)
+    y = np.arange(groups * d, dtype=np.float64).reshape(groups, d)
+    un = O.unmerge(w, y)
+    for k in range(groups * rep):
+        j = list(member[idx]).index(member[k])
+        assert np.allclose(un[k], y[j] / rep, atol=1e-5)
+
+
+def test_hot_temperature_gives_tile_mean():
+    rng = np.random.default_rng(0)
+    x = rng.normal(size=(16, 8))
+    idx = np.array([3, 7, 11])
+    w = O.merge_weights(x, idx, 1e9)
+    assert np.allclose(w, 1.0 / 16)
+    assert np.allclose(O.merge(w, x), np.tile(x.mean(0), (3, 1)))
+
+
+def test_identity_and_permutation_weights_round_trip_exactly():
+    rng = np.random.default_rng(1)
+    x = gen.round_to_dtype(rng.normal(size=(8, 5)).astype(np.float32), "bf16").astype(np.float64)
+    eye = np.eye(8)
+    assert np.array_equal(O.unmerge(eye, O.merge(eye, x)), x)
+    perm = eye[rng.permutation(8)]
+    assert np.array_equal(O.merge(perm, x), x[np.argmax(perm, axis=1)])
+    assert np.array_equal(O.unmerge(perm, O.merge(perm, x)), x)   # A A^T = I  =>  A^T is the inverse
+
+
+def test_merge_and_unmerge_are_the_two_matrix_products():
+    rng = np.random.default_rng(2)
+    w = rng.random((3, 7))
+    x = rng.normal(size=(7, 4))
+    y = rng.normal(size=(3, 4))
+    m = O.merge(w, x)
+    u = O.unmerge(w, y)
+    for i in range(3):
+        for c in range(4):
+            assert m[i, c] == pytest.approx(sum(w[i, k] * x[k, c] for k in range(7)))
+    for k in range(7):
+        for c in range(4):
+            assert u[k, c] == pytest.approx(sum(w[i, k] * y[i, c] for i in range(3)))
+
+
+def test_block_step_reuse_schedule_and_layout():
+    c = gen.config("cfg3", batch=1, grid_h=16, grid_w=16, tile_h=8, tile_w=8, dim=64, n_heads=2,
+                   head_dim=32, steps=4, reuse_interval=2)
+    st = O.BlockState()
+    kw = dict(grid_h=16, grid_w=16, tile_h=8, tile_w=8, merge_ratio=0.5, tau=c.tau, n_heads=2,
+              reuse_interval=2)
+    seen = []
+    for t, x in enumerate(gen.feature_sequence(c)):
+        out, merged, att = O.block_step(x, t, st, **kw)
+        seen.append(st.idx.copy())
+        assert out.shape == x.shape and merged.shape == (1, 4 * 32, 64)
+    assert np.array_equal(seen[0], seen[1]) and np.array_equal(seen[2], seen[3])
+    assert not np.array_equal(seen[0], seen[2])
+    # tile-major, pick-order layout of merged rows
+    x0 = gen.features(c, 0)[0].astype(np.float64)
+    st = O.BlockState()
+    _, merged, _ = O.block_step(x0[None], 0, st, **kw)
+    ids = O.tile_token_ids(16, 16, 8, 8)
+    p = 2
+    assert np.allclose(merged[0, p * 32:(p + 1) * 32], O.merge(st.w[0, p], x0[ids[p]]))
+
+
+def test_block_step_passes_text_tokens_through():
+    c = gen.config("cfg4", grid_h=16, grid_w=16, tile_h=8, tile_w=8, dim=32, n_heads=2, head_dim=16, n_extra=5)
+    x = gen.features(c)
+    st = O.BlockState()
+    out, merged, att = O.block_step(x, 0, st, grid_h=16, grid_w=16, tile_h=8, tile_w=8, merge_ratio=0.5,
+                                    tau=0.1, n_heads=2, reuse_interval=1, n_extra=5)
+    D = 4 * 32
+    assert merged.shape == (1, D + 5, 32)
+    assert np.array_equal(merged[0, D:], x[0, 256:].astype(np.float64))
+    assert np.array_equal(out[0, 256:], att[0, D:])
