@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the ToMA block path on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference] [--workload cfg3]
+
+A "step" is one toma_block call (Algorithm 3 with the reuse schedule of Sec. 4.3.2)
+on one batch of synthetic SDXL-shaped tokens.  Step t of the timed region uses
+schedule position t mod 10 of the workload's 10-step sequence, so with reuse
+interval 5 two steps in ten recompute selection and weights.  Prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "toma_block_tokens_per_s"
+UNIT = "tokens/s"
+L2_FLUSH_BYTES = 256 << 20
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "tf_burst": p["bf16_tflops"], "tf_sustained": p["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tf_burst": 1590.0, "tf_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                smax = float(r[1])
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_step_seconds(cfg, x_host, step, state):
+    from oracle import toma_oracle as O
+    t0 = time.perf_counter()
+    O.block_step(x_host, step, state, grid_h=cfg.grid_h, grid_w=cfg.grid_w, tile_h=cfg.tile_h, tile_w=cfg.tile_w,
+                 merge_ratio=cfg.merge_ratio, tau=cfg.tau, n_heads=cfg.n_heads, reuse_interval=cfg.reuse_interval,
+                 n_extra=cfg.n_extra)
+    return time.perf_counter() - t0
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([i.get("num_threads", 1) for i in threadpool_info()] or [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(cfg):
+    """The oracle as it stands, timed on this machine's host cores on batch item 0: one refresh
+    step and one reuse step, combined with the schedule's 2:8 mix."""
+    import gen
+    from oracle import toma_oracle as O
+    seq = list(gen.feature_sequence(cfg, 2))
+    st = O.BlockState()
+    t_refresh = oracle_step_seconds(cfg, seq[0][:1], 0, st)
+    t_reuse = oracle_step_seconds(cfg, seq[1][:1], 1, st)
+    k = cfg.reuse_interval
+    per_cycle = t_refresh + (k - 1) * t_reuse
+    tokens = k * (cfg.n_tokens + cfg.n_extra)
+    return {"value": tokens / per_cycle, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": f"batch item 0 of {cfg.batch}: one refresh step ({t_refresh:.2f} s) and one reuse step "
+                      f"({t_reuse:.2f} s), weighted 1:{k - 1} as in the schedule",
+            "refresh_s": t_refresh, "reuse_s": t_reuse}
+
+
+def run_reference(args, cfg):
+    """The CPU oracle as the reference arm: each step is schedule step t on batch item 0."""
+    import gen
+    from oracle import toma_oracle as O
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    seq = list(gen.feature_sequence(cfg, cfg.steps))
+    st = O.BlockState()
+    cycle = cfg.steps
+    for t in range(args.warmup):
+        oracle_step_seconds(cfg, seq[t % cycle][:1], t % cycle, st)
+    t0 = time.perf_counter()
+    for t in range(args.steps):
+        oracle_step_seconds(cfg, seq[t % cycle][:1], t % cycle, st)
+    dt = time.perf_counter() - t0
+    tokens = cfg.n_tokens + cfg.n_extra
+    value = tokens * args.steps / dt
+    sample = f"batch item 0 of {cfg.batch} per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def workload_config(cfg):
+    return {"workload": f"{cfg.name}: SDXL-like high-resolution block, batch {cfg.batch}, {cfg.grid_h}x{cfg.grid_w} "
+                        f"tokens, d={cfg.dim} {cfg.dtype}, {cfg.n_heads}x{cfg.head_dim} heads, tiles "
+                        f"{cfg.tile_h}x{cfg.tile_w}, merge ratio {cfg.merge_ratio}, reuse interval "
+                        f"{cfg.reuse_interval} over a {cfg.steps}-step drifting sequence",
+            "global_batch": cfg.batch, "seq_len": cfg.n_tokens + cfg.n_extra, "l2": "flushed between steps",
+            "parallelism": "independent batches per GPU, no collective"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="toma", choices=["toma", "reference"])
+    ap.add_argument("--workload", default="cfg3")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "toma" else args.warmup
+
+    import gen
+    cfg = gen.config(args.workload)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import numpy as np
+    import torch
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2509_10918_b200 as toma
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the ToMA path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    peaks = load_peaks()
+    cfg_rank = cfg.with_(seed=cfg.seed + rank)          # weak scaling: every rank has its own batch
+    desc = toma.desc_from_config(cfg_rank)
+    tdt = toma.torch_dtype(desc)
+    cycle = cfg.steps
+    xs_host = [torch.from_numpy(x).to(tdt).pin_memory() for x in gen.feature_sequence(cfg_rank, cycle)]
+    xs = [x.cuda() for x in xs_host]
+    out = torch.empty_like(xs[0])
+    out_host = torch.empty_like(xs_host[0]).pin_memory()
+    idx = toma.alloc_idx(desc)
+    w = toma.alloc_weights(desc)
+    ws = toma.alloc_workspace(desc)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    B, N, d = cfg.batch, cfg.n_tokens + cfg.n_extra, cfg.dim
+    Lm = cfg.n_merged + cfg.n_extra
+
+    def block(t):
+        toma.toma_block(desc, t % cycle, xs[t % cycle], out, idx, w, ws, status)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup):
+        for t in range(warmup):
+            fn(t)
+        sync_all()
+        evs = []
+        for t in range(steps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn(t)
+            e1.record()
+            evs.append((e0, e1))
+        sync_all()
+        return [a.elapsed_time(b) for a, b in evs]
+
+    # ---- the timed region: K toma_block steps -------------------------------------------------
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = toma.toma_launch_counter()
+    for t in range(args.warmup):
+        block(t)
+    launches_warm = toma.toma_launch_counter() - launches0
+    step_ms = timed(block, args.steps, 0)
+    gpu_launches = toma.toma_launch_counter() - launches0 - launches_warm
+    clocks = sampler.stop()
+    assert int(status.item()) == 0, "a kernel reported a device-side timeout"
+    total_ms = sum(step_ms)
+    t_local = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t_local, op=dist.ReduceOp.MAX)
+    total_ms = float(t_local.item())
+    ms_per_step = total_ms / args.steps
+    value = world * B * N / (ms_per_step * 1e-3)
+    refresh_ms = [m for t, m in enumerate(step_ms) if (t % cycle) % cfg.reuse_interval == 0]
+    reuse_ms = [m for t, m in enumerate(step_ms) if (t % cycle) % cfg.reuse_interval != 0]
+
+    # ---- full-token attention with the same kernel at length N --------------------------------
+    o_full = torch.empty_like(xs[0])
+
+    def full_attention(t):
+        x = xs[t % cycle]
+        toma.toma_attention(B, N, cfg.n_heads, cfg.head_dim, cfg.dtype, x, x, x, o_full, status)
+
+    full_ms = timed(full_attention, min(args.steps, 20), 3)
+
+    # ---- per-stage breakdown (same calls toma_block makes, events in between) -------------------
+    xm = torch.empty((B, Lm, d), dtype=tdt, device="cuda")
+    att = torch.empty_like(xm)
+    stages = {"select": [], "weights": [], "merge": [], "attention": [], "unmerge": []}
+    reps = min(args.steps, 20)
+    for t in range(3 + reps):
+        x = xs[t % cycle]
+        flush.zero_()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+        ev[0].record()
+        toma.toma_select(desc, x, idx, ws, status)
+        ev[1].record()
+        toma.toma_merge_weights(desc, x, idx, w, ws, status)
+        ev[2].record()
+        toma.toma_merge(desc, w, x, xm, status)
+        ev[3].record()
+        toma.toma_attention(B, Lm, cfg.n_heads, cfg.head_dim, cfg.dtype, xm, xm, xm, att, status)
+        ev[4].record()
+        toma.toma_unmerge(desc, w, att, out, status)
+        ev[5].record()
+        torch.cuda.synchronize()
+        if t >= 3:
+            for i, name in enumerate(stages):
+                stages[name].append(ev[i].elapsed_time(ev[i + 1]))
+    stage_ms = {k: statistics.mean(v) for k, v in stages.items()}
+    esz = 2 if cfg.dtype == "bf16" else 4
+    att_flops = 4.0 * B * Lm * Lm * d
+    att_tf = att_flops / (stage_ms["attention"] * 1e-3) / 1e12
+    mrg_bytes = B * (cfg.n_tokens * d * esz + cfg.n_merged * d * esz + cfg.n_tiles * cfg.n_loc * cfg.d_loc * esz)
+    roofline = {"kernel": "attention over merged tokens", "bound": "tensor", "achieved": att_tf,
+                "peak": peaks["tf_burst"], "unit": "TFLOP/s", "frac": att_tf / peaks["tf_burst"], "traffic": None,
+                "peak_source": peaks["source"] + " bf16 burst",
+                "merge_gbs": mrg_bytes / (stage_ms["merge"] * 1e-3) / 1e9,
+                "unmerge_gbs": mrg_bytes / (stage_ms["unmerge"] * 1e-3) / 1e9,
+                "hbm_peak_gbs": peaks["hbm_gbs"]}
+
+    # ---- end to end: pinned host input -> device -> block -> host output, every step ----------
+    x_dev = torch.empty_like(xs[0])
+
+    def e2e_step(t):
+        x_dev.copy_(xs_host[t % cycle], non_blocking=True)
+        toma.toma_block(desc, t % cycle, x_dev, out, idx, w, ws, status)
+        out_host.copy_(out, non_blocking=True)
+
+    for t in range(3):
+        e2e_step(t)
+    sync_all()
+    t0 = time.perf_counter()
+    for t in range(args.steps):
+        e2e_step(t)
+    sync_all()
+    e2e_s = time.perf_counter() - t0
+    t_local = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t_local, op=dist.ReduceOp.MAX)
+    e2e_value = world * B * N * args.steps / float(t_local.item())
+    xbytes = xs[0].numel() * xs[0].element_size()
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": cfg.dtype, "data": "synthetic", "config": workload_config(cfg),
+        "block_latency_us": {"mean": 1e3 * ms_per_step, "refresh_median": 1e3 * statistics.median(refresh_ms) if refresh_ms else None,
+                             "reuse_median": 1e3 * statistics.median(reuse_ms) if reuse_ms else None},
+        "full_attention_latency_us": 1e3 * statistics.median(full_ms),
+        "speedup_vs_full_attention": statistics.median(full_ms) / ms_per_step,
+        "stage_us": {k: 1e3 * v for k, v in stage_ms.items()},
+        "roofline": roofline,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": xbytes, "d2h_bytes_per_step": xbytes},
+        "gpu_launches": int(gpu_launches),
+        "clocks": clocks,
+        "paper_context": "paper reports -24%/-23% SDXL/Flux generation latency on RTX6000/V100/RTX8000 (other hardware)",
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = cpu_baseline(cfg)
+    if rank == 0:
+        print(json.dumps(result))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -118,7 +118,7 @@ class TomaConfig:
 
     @property
     def d_loc(self) -> int:
-        return self.n_loc - int(round(self.merge_ratio * self.n_loc))
+        return self.n_loc - int(np.floor(float(np.float32(self.merge_ratio)) * self.n_loc + 0.5))
 
     @property
     def n_merged(self) -> int:

@@ -1,0 +1,140 @@
+/*
+ * toma.h -- C ABI of the B200 (sm_100a) ToMA token-reduction library.
+ *
+ * The library implements, per transformer block, the locality-aware ToMA path
+ * of "ToMA: Token Merge with Attention for Diffusion Models" (Algorithm 3):
+ * split the H x W token grid into equal tiles, pick destination tokens in every
+ * tile by greedy facility-location maximisation (Algorithm 2), build the
+ * attention-like merge weights (Sec. 4.2.1), merge N tokens to D, run the core
+ * attention over the D merged tokens (Eq. 1), and unmerge with the transposed
+ * weights (Sec. 4.2.2).  Selection and weights are reused between refresh
+ * steps (Sec. 4.3.2).
+ *
+ * Conventions that hold for every entry point
+ *   - Every data pointer is DEVICE memory owned by the caller, 16-byte aligned,
+ *     dense row-major.  `desc` is HOST memory.  The library never allocates,
+ *     frees or synchronises; work is enqueued on `stream` (a cudaStream_t
+ *     passed as void*; NULL is the default stream).
+ *   - Errors the host can detect (null pointers, shapes that do not divide,
+ *     unsupported sizes, a workspace that is too small) are returned before
+ *     anything is launched.  Conditions only the device can see (a bounded wait
+ *     inside a kernel that ran out) are OR-ed into `*dev_status`, a caller-owned
+ *     device word that the caller zeroes and reads after synchronising; the
+ *     kernels still exit cleanly.  `dev_status` may be NULL.
+ *   - There is no CPU fallback: without a CUDA device the calls fail with
+ *     TOMA_ERR_CUDA.
+ *
+ * Token layout.  X is [batch][grid_h*grid_w + n_extra][dim].  Image token
+ * n = y*grid_w + x lies in tile p = (y/tile_h)*(grid_w/tile_w) + x/tile_w at
+ * local slot l = (y%tile_h)*tile_w + x%tile_w.  N_loc = tile_h*tile_w,
+ * P = tiles per image, D_loc = N_loc - round(merge_ratio*N_loc) destinations
+ * per tile, D = P*D_loc.  Merged tensors are [batch][D + n_extra][dim] with row
+ * p*D_loc + k holding destination k (greedy pick order) of tile p; the n_extra
+ * trailing (text) tokens are never merged and follow the D merged rows.
+ */
+#ifndef TOMA_H_
+#define TOMA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define TOMA_API __attribute__((visibility("default")))
+#else
+#define TOMA_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  TOMA_OK = 0,
+  TOMA_ERR_NULL = 1,        /* a required pointer is NULL */
+  TOMA_ERR_SHAPE = 2,       /* tiles do not divide the grid, dim not a multiple of 8, heads*head_dim != dim ... */
+  TOMA_ERR_DTYPE = 3,
+  TOMA_ERR_RATIO = 4,       /* merge_ratio outside [0,1) or leaving no destination */
+  TOMA_ERR_TAU = 5,         /* tau <= 0 or not finite */
+  TOMA_ERR_WORKSPACE = 6,   /* workspace missing or smaller than toma_workspace_bytes() */
+  TOMA_ERR_UNSUPPORTED = 7, /* N_loc > 1024, head_dim not 64/128 in bf16 mode, dim > 4096 ... */
+  TOMA_ERR_CUDA = 8,        /* a CUDA runtime call or launch failed */
+  TOMA_ERR_TIMEOUT = 9      /* only ever reported through *dev_status (bit 0) */
+} toma_status;
+
+typedef enum { TOMA_BF16 = 0, TOMA_F32 = 1 } toma_dtype;
+
+/* Problem statement of Algorithm 3 (token tensor shape, region layout, merge
+ * ratio, temperature) plus the reuse schedule of Sec. 4.3.2.  Plain data. */
+typedef struct {
+  int32_t batch, grid_h, grid_w, dim;
+  int32_t tile_h, tile_w;          /* must divide grid_h / grid_w; a stripe is tile_h x grid_w */
+  float merge_ratio;               /* fraction of tokens REMOVED, in [0, 1) */
+  float tau;                       /* merge temperature; logits are <d_i, x_k> / (tau * sqrt(dim)) */
+  int32_t reuse_interval;          /* k >= 1: toma_block refreshes selection when step % k == 0 */
+  int32_t weight_reuse_interval;   /* 0: same as reuse_interval; else weights are refreshed when
+                                      step % weight_reuse_interval == 0 from the cached selection */
+  int32_t n_heads, head_dim;       /* n_heads*head_dim == dim (attention inside toma_block) */
+  int32_t n_extra;                 /* trailing un-merged tokens */
+  int32_t dtype;                   /* toma_dtype of x / merged / out tensors */
+} toma_desc;
+
+/* Host-only helpers.  Return 0 / negative on an invalid descriptor. */
+TOMA_API size_t toma_workspace_bytes(const toma_desc* desc);   /* scratch needed by select / merge_weights / block */
+TOMA_API size_t toma_weights_bytes(const toma_desc* desc);     /* size of one weight buffer `w` */
+TOMA_API int32_t toma_dest_per_tile(const toma_desc* desc);    /* D_loc */
+TOMA_API toma_status toma_validate(const toma_desc* desc);
+TOMA_API const char* toma_status_str(toma_status s);
+/* Total number of kernels this library has launched in this process (monotonic; for benchmarks). */
+TOMA_API uint64_t toma_launch_counter(void);
+
+/* Destination selection (Sec. 4.1, Algorithm 2) inside every tile.
+ *   x   [batch][N + n_extra][dim]  in
+ *   idx [batch][P][D_loc] int32    out: tile-local indices (0..N_loc-1) in greedy pick order
+ * Similarity is the fixed-point cosine: each token is scaled to length 0.99,
+ * quantised to a bf16-representable grid of 2^-12 steps, the Gram matrix is
+ * accumulated exactly and rounded to int16 units of 2^-12 (diagonal forced to
+ * 4014).  Gains are exact integers; ties go to the lowest index; selected
+ * tokens are excluded from later rounds.  Uses `ws` as scratch. */
+TOMA_API toma_status toma_select(const toma_desc* desc, const void* x, int32_t* idx, void* ws, size_t ws_bytes,
+                        uint32_t* dev_status, void* stream);
+
+/* Merge weights (Sec. 4.2.1).  For each tile: logits between the D_loc selected
+ * tokens and all N_loc tokens, softmax over the destination axis per source
+ * token, then each destination row normalised to sum 1.
+ *   w: opaque buffer of toma_weights_bytes(); holds A~^T as [batch][P][N_loc][D_loc]
+ *      (fp16 in bf16 mode, fp32 in f32 mode).  Uses `ws` as scratch. */
+TOMA_API toma_status toma_merge_weights(const toma_desc* desc, const void* x, const int32_t* idx, void* w, void* ws,
+                               size_t ws_bytes, uint32_t* dev_status, void* stream);
+
+/* Merge X_m = A~ X per tile (Sec. 4.2.1).  xm [batch][D + n_extra][dim] out; extra tokens copied. */
+TOMA_API toma_status toma_merge(const toma_desc* desc, const void* w, const void* x, void* xm, uint32_t* dev_status,
+                       void* stream);
+
+/* Multi-head attention core softmax(Q K^T / sqrt(head_dim)) V (Eq. 1 with tau = 1), no mask.
+ *   q, k, v, o: [batch][len][n_heads][head_dim]. */
+TOMA_API toma_status toma_attention(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim, int32_t dtype,
+                           const void* q, const void* k, const void* v, void* o, uint32_t* dev_status,
+                           void* stream);
+
+/* Unmerge out = A~^T y per tile, written back in spatial order (Sec. 4.2.2, Algorithm 3 step 3).
+ *   y [batch][D + n_extra][dim] in; out [batch][N + n_extra][dim]; extra tokens copied. */
+TOMA_API toma_status toma_unmerge(const toma_desc* desc, const void* w, const void* y, void* out, uint32_t* dev_status,
+                         void* stream);
+
+/* One ToMA-wrapped attention call (Algorithm 3) with pattern reuse (Sec. 4.3.2):
+ * refresh idx_state / w_state when the schedule says so, then merge, attention
+ * with Q = K = V = merged tokens, unmerge.  idx_state [batch][P][D_loc] and
+ * w_state (toma_weights_bytes()) persist between calls and are caller-owned. */
+TOMA_API toma_status toma_block(const toma_desc* desc, int32_t step, const void* x, void* out, int32_t* idx_state,
+                       void* w_state, void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream);
+
+/* Conversions between the opaque weight buffer and dense fp32 A~ [batch][P][D_loc][N_loc]
+ * (device pointers).  For tests and for callers that bring their own weights (a
+ * one-hot matrix makes merge a hard ToMeSD-style merge, Sec. 4.2). */
+TOMA_API toma_status toma_weights_export(const toma_desc* desc, const void* w, float* dense, void* stream);
+TOMA_API toma_status toma_weights_import(const toma_desc* desc, const float* dense, void* w, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TOMA_H_ */

@@ -48,7 +48,8 @@ def dest_count(n_loc: int, merge_ratio: float) -> int:
     """Destinations per region.  `merge_ratio` is the fraction of tokens REMOVED
     (the reading under which the paper's tables get faster as the ratio grows,
     App. F: D = (1 - r) N)."""
-    d_loc = n_loc - int(round(merge_ratio * n_loc))
+    # half-way cases round up; the ratio is taken at float32 precision like the C descriptor field
+    d_loc = n_loc - int(np.floor(float(np.float32(merge_ratio)) * n_loc + 0.5))
     if d_loc < 1 or d_loc > n_loc:
         raise ValueError("merge ratio leaves no destination")
     return d_loc

@@ -1,0 +1,200 @@
+"""ctypes binding of libtoma_b200.so: the same names as the C ABI, argument
+marshalling only.  Tensors are torch CUDA tensors; their data pointers and the
+current stream handle are passed straight through.  There is no fallback: if the
+shared library has not been built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, c_char_p, c_float, c_int32, c_size_t, c_void_p
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtoma_b200.so")
+
+TOMA_BF16, TOMA_F32 = 0, 1
+STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_RATIO", "ERR_TAU", "ERR_WORKSPACE",
+                "ERR_UNSUPPORTED", "ERR_CUDA", "ERR_TIMEOUT"]
+
+EXPORTS = ["toma_launch_counter", "toma_workspace_bytes", "toma_weights_bytes", "toma_dest_per_tile", "toma_validate", "toma_status_str",
+           "toma_select", "toma_merge_weights", "toma_merge", "toma_attention", "toma_unmerge", "toma_block",
+           "toma_weights_export", "toma_weights_import"]
+
+
+class TomaDesc(Structure):
+    _fields_ = [
+        ("batch", c_int32), ("grid_h", c_int32), ("grid_w", c_int32), ("dim", c_int32),
+        ("tile_h", c_int32), ("tile_w", c_int32),
+        ("merge_ratio", c_float), ("tau", c_float),
+        ("reuse_interval", c_int32), ("weight_reuse_interval", c_int32),
+        ("n_heads", c_int32), ("head_dim", c_int32), ("n_extra", c_int32), ("dtype", c_int32),
+    ]
+
+
+class TomaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{where}: TOMA_{name}")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2509_10918_b200.build` "
+            "(there is no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    P = POINTER(TomaDesc)
+    lib.toma_workspace_bytes.restype = c_size_t
+    lib.toma_workspace_bytes.argtypes = [P]
+    lib.toma_weights_bytes.restype = c_size_t
+    lib.toma_weights_bytes.argtypes = [P]
+    lib.toma_dest_per_tile.restype = c_int32
+    lib.toma_dest_per_tile.argtypes = [P]
+    lib.toma_launch_counter.restype = ctypes.c_uint64
+    lib.toma_launch_counter.argtypes = []
+    lib.toma_validate.restype = c_int32
+    lib.toma_validate.argtypes = [P]
+    lib.toma_status_str.restype = c_char_p
+    lib.toma_status_str.argtypes = [c_int32]
+    lib.toma_select.restype = c_int32
+    lib.toma_select.argtypes = [P, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
+    lib.toma_merge_weights.restype = c_int32
+    lib.toma_merge_weights.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
+    lib.toma_merge.restype = c_int32
+    lib.toma_merge.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.toma_unmerge.restype = c_int32
+    lib.toma_unmerge.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.toma_attention.restype = c_int32
+    lib.toma_attention.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
+                                   c_void_p, c_void_p, c_void_p]
+    lib.toma_block.restype = c_int32
+    lib.toma_block.argtypes = [P, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p,
+                               c_void_p]
+    lib.toma_weights_export.restype = c_int32
+    lib.toma_weights_export.argtypes = [P, c_void_p, c_void_p, c_void_p]
+    lib.toma_weights_import.restype = c_int32
+    lib.toma_weights_import.argtypes = [P, c_void_p, c_void_p, c_void_p]
+    return lib
+
+
+lib = _load()
+
+
+def make_desc(*, batch, grid_h, grid_w, dim, tile_h, tile_w, merge_ratio, tau, n_heads, head_dim, dtype,
+              reuse_interval=1, weight_reuse_interval=0, n_extra=0) -> TomaDesc:
+    code = {"bf16": TOMA_BF16, "f32": TOMA_F32, TOMA_BF16: TOMA_BF16, TOMA_F32: TOMA_F32}[dtype]
+    return TomaDesc(batch, grid_h, grid_w, dim, tile_h, tile_w, merge_ratio, tau, reuse_interval,
+                    weight_reuse_interval, n_heads, head_dim, n_extra, code)
+
+
+def desc_from_config(cfg, **overrides) -> TomaDesc:
+    """Descriptor from a gen.TomaConfig-like object (duck-typed attributes)."""
+    kw = dict(batch=cfg.batch, grid_h=cfg.grid_h, grid_w=cfg.grid_w, dim=cfg.dim, tile_h=cfg.tile_h,
+              tile_w=cfg.tile_w, merge_ratio=cfg.merge_ratio, tau=cfg.tau, n_heads=cfg.n_heads,
+              head_dim=cfg.head_dim, dtype=cfg.dtype, reuse_interval=cfg.reuse_interval, n_extra=cfg.n_extra)
+    kw.update(overrides)
+    return make_desc(**kw)
+
+
+def torch_dtype(desc: TomaDesc):
+    return torch.float32 if desc.dtype == TOMA_F32 else torch.bfloat16
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("tensor must live on a CUDA device (no CPU path exists)")
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise TomaError(status, where)
+
+
+def toma_validate(desc: TomaDesc) -> int:
+    return lib.toma_validate(ctypes.byref(desc))
+
+
+def toma_workspace_bytes(desc: TomaDesc) -> int:
+    return lib.toma_workspace_bytes(ctypes.byref(desc))
+
+
+def toma_weights_bytes(desc: TomaDesc) -> int:
+    return lib.toma_weights_bytes(ctypes.byref(desc))
+
+
+def toma_dest_per_tile(desc: TomaDesc) -> int:
+    return lib.toma_dest_per_tile(ctypes.byref(desc))
+
+
+def toma_launch_counter() -> int:
+    return int(lib.toma_launch_counter())
+
+
+def toma_status_str(status: int) -> str:
+    return lib.toma_status_str(status).decode()
+
+
+def toma_select(desc, x, idx, ws, dev_status=None):
+    _check(lib.toma_select(ctypes.byref(desc), _ptr(x), _ptr(idx), _ptr(ws), ws.numel() * ws.element_size(),
+                           _ptr(dev_status), _stream()), "toma_select")
+
+
+def toma_merge_weights(desc, x, idx, w, ws, dev_status=None):
+    _check(lib.toma_merge_weights(ctypes.byref(desc), _ptr(x), _ptr(idx), _ptr(w), _ptr(ws),
+                                  ws.numel() * ws.element_size(), _ptr(dev_status), _stream()), "toma_merge_weights")
+
+
+def toma_merge(desc, w, x, xm, dev_status=None):
+    _check(lib.toma_merge(ctypes.byref(desc), _ptr(w), _ptr(x), _ptr(xm), _ptr(dev_status), _stream()), "toma_merge")
+
+
+def toma_unmerge(desc, w, y, out, dev_status=None):
+    _check(lib.toma_unmerge(ctypes.byref(desc), _ptr(w), _ptr(y), _ptr(out), _ptr(dev_status), _stream()),
+           "toma_unmerge")
+
+
+def toma_attention(batch, length, n_heads, head_dim, dtype, q, k, v, o, dev_status=None):
+    code = {"bf16": TOMA_BF16, "f32": TOMA_F32, TOMA_BF16: TOMA_BF16, TOMA_F32: TOMA_F32}[dtype]
+    _check(lib.toma_attention(batch, length, n_heads, head_dim, code, _ptr(q), _ptr(k), _ptr(v), _ptr(o),
+                              _ptr(dev_status), _stream()), "toma_attention")
+
+
+def toma_block(desc, step, x, out, idx_state, w_state, ws, dev_status=None):
+    _check(lib.toma_block(ctypes.byref(desc), step, _ptr(x), _ptr(out), _ptr(idx_state), _ptr(w_state), _ptr(ws),
+                          ws.numel() * ws.element_size(), _ptr(dev_status), _stream()), "toma_block")
+
+
+def toma_weights_export(desc, w, dense):
+    _check(lib.toma_weights_export(ctypes.byref(desc), _ptr(w), _ptr(dense), _stream()), "toma_weights_export")
+
+
+def toma_weights_import(desc, dense, w):
+    _check(lib.toma_weights_import(ctypes.byref(desc), _ptr(dense), _ptr(w), _stream()), "toma_weights_import")
+
+
+# ---- allocation helpers (torch owns the memory; the library never allocates) ----
+
+def alloc_workspace(desc, device="cuda") -> torch.Tensor:
+    return torch.empty(max(toma_workspace_bytes(desc), 16), dtype=torch.uint8, device=device)
+
+
+def alloc_weights(desc, device="cuda") -> torch.Tensor:
+    return torch.empty(max(toma_weights_bytes(desc), 16), dtype=torch.uint8, device=device)
+
+
+def alloc_idx(desc, device="cuda") -> torch.Tensor:
+    tiles = (desc.grid_h // desc.tile_h) * (desc.grid_w // desc.tile_w)
+    return torch.empty((desc.batch, tiles, toma_dest_per_tile(desc)), dtype=torch.int32, device=device)

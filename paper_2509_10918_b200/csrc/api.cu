@@ -1,0 +1,250 @@
+// extern "C" boundary of the ToMA library: descriptor validation, workspace
+// carve-up and kernel sequencing.  Argument marshalling only; all arithmetic is in
+// the kernels.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace toma {
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+toma_status make_geom(const toma_desc* desc, Geom* g) {
+  if (!desc) return TOMA_ERR_NULL;
+  if (desc->dtype != TOMA_BF16 && desc->dtype != TOMA_F32) return TOMA_ERR_DTYPE;
+  if (desc->batch < 1 || desc->grid_h < 1 || desc->grid_w < 1 || desc->dim < 8 || desc->dim % 8) return TOMA_ERR_SHAPE;
+  if (desc->tile_h < 1 || desc->tile_w < 1 || desc->grid_h % desc->tile_h || desc->grid_w % desc->tile_w)
+    return TOMA_ERR_SHAPE;
+  if (desc->n_extra < 0) return TOMA_ERR_SHAPE;
+  if (desc->n_heads < 1 || desc->head_dim < 1 || (long long)desc->n_heads * desc->head_dim != desc->dim)
+    return TOMA_ERR_SHAPE;
+  if (!(desc->merge_ratio >= 0.f) || !(desc->merge_ratio < 1.f)) return TOMA_ERR_RATIO;
+  if (!(desc->tau > 0.f) || !isfinite(desc->tau)) return TOMA_ERR_TAU;
+  if (desc->reuse_interval < 1 || desc->weight_reuse_interval < 0) return TOMA_ERR_SHAPE;
+  const long long nloc = (long long)desc->tile_h * desc->tile_w;
+  if (nloc > kMaxNloc || desc->dim > kMaxDim) return TOMA_ERR_UNSUPPORTED;
+  const long long ntok = (long long)desc->grid_h * desc->grid_w;
+  if ((ntok + desc->n_extra) * (long long)desc->batch > (1ll << 30)) return TOMA_ERR_UNSUPPORTED;
+  const int dloc = (int)nloc - (int)lround((double)desc->merge_ratio * (double)nloc);
+  if (dloc < 1 || dloc > nloc) return TOMA_ERR_RATIO;
+  g->B = desc->batch; g->H = desc->grid_h; g->W = desc->grid_w; g->d = desc->dim;
+  g->th = desc->tile_h; g->tw = desc->tile_w;
+  g->tiles_x = desc->grid_w / desc->tile_w;
+  g->P = g->tiles_x * (desc->grid_h / desc->tile_h);
+  g->N = (int)ntok; g->Nloc = (int)nloc; g->Dloc = dloc; g->D = g->P * dloc;
+  g->n_extra = desc->n_extra; g->Lm = g->D + g->n_extra;
+  g->heads = desc->n_heads; g->dh = desc->head_dim;
+  g->f32 = desc->dtype == TOMA_F32;
+  g->logit_scale = (float)(1.0 / ((double)desc->tau * sqrt((double)desc->dim)));
+  return TOMA_OK;
+}
+
+WsLayout ws_layout(const Geom& g) {
+  WsLayout l;
+  const size_t tiles = (size_t)g.B * g.P;
+  const size_t esz = g.f32 ? 4 : 2;
+  size_t off = 0;
+  l.y_off = off;      off = align_up(off + tiles * g.Nloc * g.d * sizeof(__nv_bfloat16), 256);
+  l.sq_off = off;     off = align_up(off + tiles * g.Nloc * g.Nloc * sizeof(int16_t), 256);
+  l.logits_off = off; off = align_up(off + tiles * g.Dloc * g.Nloc * sizeof(float), 256);
+  l.xm_off = off;     off = align_up(off + (size_t)g.B * g.Lm * g.d * esz, 256);
+  l.att_off = off;    off = align_up(off + (size_t)g.B * g.Lm * g.d * esz, 256);
+  l.total = off;
+  return l;
+}
+
+static bool attention_supported_simt(int dh) { return dh == 16 || dh == 32 || dh == 64 || dh == 128; }
+
+static toma_status check_ws(const Geom& g, const void* ws, size_t ws_bytes) {
+  if (!ws) return TOMA_ERR_WORKSPACE;
+  if (((uintptr_t)ws & 15) != 0) return TOMA_ERR_WORKSPACE;
+  return ws_bytes >= ws_layout(g).total ? TOMA_OK : TOMA_ERR_WORKSPACE;
+}
+
+static toma_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? TOMA_OK : TOMA_ERR_CUDA; }
+
+static bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
+
+// --- step sequencing shared by the public entry points -------------------------------
+
+static cudaError_t do_select(const Geom& g, const void* x, int32_t* idx, char* ws, uint32_t* dev_status,
+                             cudaStream_t s) {
+  const WsLayout l = ws_layout(g);
+  __nv_bfloat16* y = (__nv_bfloat16*)(ws + l.y_off);
+  int16_t* sq = (int16_t*)(ws + l.sq_off);
+  cudaError_t e = launch_quantise(g, x, y, s);
+  if (e != cudaSuccess) return e;
+  e = launch_gram_ffma(g, y, sq, s);
+  if (e != cudaSuccess) return e;
+  return launch_greedy(g, sq, idx, s);
+}
+
+static cudaError_t do_weights(const Geom& g, const void* x, const int32_t* idx, void* w, char* ws,
+                              uint32_t* dev_status, cudaStream_t s) {
+  const WsLayout l = ws_layout(g);
+  return launch_weights_simt(g, x, idx, w, (float*)(ws + l.logits_off), s);
+}
+
+static cudaError_t do_merge(const Geom& g, const void* w, const void* x, void* xm, uint32_t* dev_status,
+                            cudaStream_t s) {
+  return launch_merge_simt(g, w, x, xm, s);
+}
+
+static cudaError_t do_unmerge(const Geom& g, const void* w, const void* y, void* out, uint32_t* dev_status,
+                              cudaStream_t s) {
+  return launch_unmerge_simt(g, w, y, out, s);
+}
+
+static cudaError_t do_attention(int B, int L, int heads, int dh, bool f32, const void* q, const void* k,
+                                const void* v, void* o, uint32_t* dev_status, cudaStream_t s) {
+  return launch_attention_simt(B, L, heads, dh, f32, q, k, v, o, s);
+}
+
+}  // namespace toma
+
+using namespace toma;
+
+extern "C" {
+
+toma_status toma_validate(const toma_desc* desc) {
+  Geom g;
+  return make_geom(desc, &g);
+}
+
+size_t toma_workspace_bytes(const toma_desc* desc) {
+  Geom g;
+  if (make_geom(desc, &g) != TOMA_OK) return 0;
+  return ws_layout(g).total;
+}
+
+size_t toma_weights_bytes(const toma_desc* desc) {
+  Geom g;
+  if (make_geom(desc, &g) != TOMA_OK) return 0;
+  return (size_t)g.B * g.P * g.Nloc * g.Dloc * (g.f32 ? 4 : 2);
+}
+
+int32_t toma_dest_per_tile(const toma_desc* desc) {
+  Geom g;
+  if (make_geom(desc, &g) != TOMA_OK) return -1;
+  return g.Dloc;
+}
+
+const char* toma_status_str(toma_status s) {
+  switch (s) {
+    case TOMA_OK: return "ok";
+    case TOMA_ERR_NULL: return "null pointer";
+    case TOMA_ERR_SHAPE: return "bad shape";
+    case TOMA_ERR_DTYPE: return "bad dtype";
+    case TOMA_ERR_RATIO: return "bad merge ratio";
+    case TOMA_ERR_TAU: return "bad temperature";
+    case TOMA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case TOMA_ERR_UNSUPPORTED: return "unsupported size";
+    case TOMA_ERR_CUDA: return "CUDA error";
+    case TOMA_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown";
+}
+
+toma_status toma_select(const toma_desc* desc, const void* x, int32_t* idx, void* ws, size_t ws_bytes,
+                        uint32_t* dev_status, void* stream) {
+  Geom g;
+  toma_status st = make_geom(desc, &g);
+  if (st != TOMA_OK) return st;
+  if (!x || !idx) return TOMA_ERR_NULL;
+  if (misaligned(x)) return TOMA_ERR_SHAPE;
+  if ((st = check_ws(g, ws, ws_bytes)) != TOMA_OK) return st;
+  return cuda_ok(do_select(g, x, idx, (char*)ws, dev_status, (cudaStream_t)stream));
+}
+
+toma_status toma_merge_weights(const toma_desc* desc, const void* x, const int32_t* idx, void* w, void* ws,
+                               size_t ws_bytes, uint32_t* dev_status, void* stream) {
+  Geom g;
+  toma_status st = make_geom(desc, &g);
+  if (st != TOMA_OK) return st;
+  if (!x || !idx || !w) return TOMA_ERR_NULL;
+  if (misaligned(x) || misaligned(w)) return TOMA_ERR_SHAPE;
+  if ((st = check_ws(g, ws, ws_bytes)) != TOMA_OK) return st;
+  return cuda_ok(do_weights(g, x, idx, w, (char*)ws, dev_status, (cudaStream_t)stream));
+}
+
+toma_status toma_merge(const toma_desc* desc, const void* w, const void* x, void* xm, uint32_t* dev_status,
+                       void* stream) {
+  Geom g;
+  toma_status st = make_geom(desc, &g);
+  if (st != TOMA_OK) return st;
+  if (!w || !x || !xm) return TOMA_ERR_NULL;
+  if (misaligned(x) || misaligned(w) || misaligned(xm)) return TOMA_ERR_SHAPE;
+  return cuda_ok(do_merge(g, w, x, xm, dev_status, (cudaStream_t)stream));
+}
+
+toma_status toma_unmerge(const toma_desc* desc, const void* w, const void* y, void* out, uint32_t* dev_status,
+                         void* stream) {
+  Geom g;
+  toma_status st = make_geom(desc, &g);
+  if (st != TOMA_OK) return st;
+  if (!w || !y || !out) return TOMA_ERR_NULL;
+  if (misaligned(y) || misaligned(w) || misaligned(out)) return TOMA_ERR_SHAPE;
+  return cuda_ok(do_unmerge(g, w, y, out, dev_status, (cudaStream_t)stream));
+}
+
+toma_status toma_attention(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim, int32_t dtype,
+                           const void* q, const void* k, const void* v, void* o, uint32_t* dev_status,
+                           void* stream) {
+  if (dtype != TOMA_BF16 && dtype != TOMA_F32) return TOMA_ERR_DTYPE;
+  if (batch < 1 || len < 1 || n_heads < 1 || head_dim < 1) return TOMA_ERR_SHAPE;
+  if (!q || !k || !v || !o) return TOMA_ERR_NULL;
+  if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(o)) return TOMA_ERR_SHAPE;
+  if (!attention_supported_simt(head_dim)) return TOMA_ERR_UNSUPPORTED;
+  return cuda_ok(do_attention(batch, len, n_heads, head_dim, dtype == TOMA_F32, q, k, v, o, dev_status,
+                              (cudaStream_t)stream));
+}
+
+toma_status toma_block(const toma_desc* desc, int32_t step, const void* x, void* out, int32_t* idx_state,
+                       void* w_state, void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream) {
+  Geom g;
+  toma_status st = make_geom(desc, &g);
+  if (st != TOMA_OK) return st;
+  if (!x || !out || !idx_state || !w_state) return TOMA_ERR_NULL;
+  if (step < 0) return TOMA_ERR_SHAPE;
+  if (misaligned(x) || misaligned(out) || misaligned(w_state)) return TOMA_ERR_SHAPE;
+  if (!attention_supported_simt(g.dh)) return TOMA_ERR_UNSUPPORTED;
+  if ((st = check_ws(g, ws, ws_bytes)) != TOMA_OK) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  char* wsb = (char*)ws;
+  const WsLayout l = ws_layout(g);
+  const int kw = desc->weight_reuse_interval > 0 ? desc->weight_reuse_interval : desc->reuse_interval;
+  const bool refresh_sel = step % desc->reuse_interval == 0;
+  const bool refresh_w = refresh_sel || step % kw == 0;
+  cudaError_t e = cudaSuccess;
+  if (refresh_sel) e = do_select(g, x, idx_state, wsb, dev_status, s);
+  if (e == cudaSuccess && refresh_w) e = do_weights(g, x, idx_state, w_state, wsb, dev_status, s);
+  void* xm = wsb + l.xm_off;
+  void* att = wsb + l.att_off;
+  if (e == cudaSuccess) e = do_merge(g, w_state, x, xm, dev_status, s);
+  if (e == cudaSuccess) e = do_attention(g.B, g.Lm, g.heads, g.dh, g.f32, xm, xm, xm, att, dev_status, s);
+  if (e == cudaSuccess) e = do_unmerge(g, w_state, att, out, dev_status, s);
+  return cuda_ok(e);
+}
+
+toma_status toma_weights_export(const toma_desc* desc, const void* w, float* dense, void* stream) {
+  Geom g;
+  toma_status st = make_geom(desc, &g);
+  if (st != TOMA_OK) return st;
+  if (!w || !dense) return TOMA_ERR_NULL;
+  return cuda_ok(launch_weights_export(g, w, dense, (cudaStream_t)stream));
+}
+
+toma_status toma_weights_import(const toma_desc* desc, const float* dense, void* w, void* stream) {
+  Geom g;
+  toma_status st = make_geom(desc, &g);
+  if (st != TOMA_OK) return st;
+  if (!w || !dense) return TOMA_ERR_NULL;
+  return cuda_ok(launch_weights_import(g, dense, w, (cudaStream_t)stream));
+}
+
+}  // extern "C"
+
+namespace toma {
+std::atomic<unsigned long long> g_launches{0};
+}
+extern "C" uint64_t toma_launch_counter(void) { return (uint64_t)toma::g_launches.load(); }

@@ -1,0 +1,71 @@
+// Shared declarations of the ToMA sm_100a library: derived problem geometry,
+// launch prototypes between translation units, small device helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "../../include/toma.h"
+
+namespace toma {
+
+// Fixed-point cosine similarity constants (see toma_select in toma.h).
+constexpr double kCosScaleTimesOne = 0.99 * 4096.0;  // token length 0.99 in units of 2^-12
+constexpr int kDiagQ = 4014;                          // rint(0.99^2 * 4096)
+constexpr int kMaxNloc = 1024;
+constexpr int kMaxDim = 4096;
+
+// Geometry derived from a validated descriptor.
+struct Geom {
+  int B, H, W, d, th, tw, tiles_x, P, N, Nloc, Dloc, D, n_extra, Lm;  // Lm = D + n_extra
+  int heads, dh;
+  bool f32;
+  float logit_scale;  // 1 / (tau * sqrt(d))
+  long long tokens_all() const { return (long long)N + n_extra; }
+};
+
+toma_status make_geom(const toma_desc* desc, Geom* g);
+
+// Workspace carve-up (all offsets 256-byte aligned).
+struct WsLayout {
+  size_t y_off, sq_off, logits_off, xm_off, att_off, total;
+};
+WsLayout ws_layout(const Geom& g);
+
+// Process-wide count of kernel launches (reported by toma_launch_counter()).
+extern std::atomic<unsigned long long> g_launches;
+inline void count_launch(int n = 1) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+// ---- launchers (each returns cudaGetLastError() of its launches) ----
+cudaError_t launch_quantise(const Geom& g, const void* x, __nv_bfloat16* y, cudaStream_t s);
+cudaError_t launch_gram_ffma(const Geom& g, const __nv_bfloat16* y, int16_t* sq, cudaStream_t s);
+cudaError_t launch_greedy(const Geom& g, const int16_t* sq, int32_t* idx, cudaStream_t s);
+cudaError_t launch_weights_simt(const Geom& g, const void* x, const int32_t* idx, void* w, float* logits,
+                                cudaStream_t s);
+cudaError_t launch_merge_simt(const Geom& g, const void* w, const void* x, void* xm, cudaStream_t s);
+cudaError_t launch_unmerge_simt(const Geom& g, const void* w, const void* y, void* out, cudaStream_t s);
+cudaError_t launch_attention_simt(int B, int L, int heads, int dh, bool f32, const void* q, const void* k,
+                                  const void* v, void* o, cudaStream_t s);
+cudaError_t launch_weights_export(const Geom& g, const void* w, float* dense, cudaStream_t s);
+cudaError_t launch_weights_import(const Geom& g, const float* dense, void* w, cudaStream_t s);
+
+// ---- device helpers ----
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float to_f32(__half v) { return __half2float(v); }
+__device__ __forceinline__ void from_f32(float& o, float v) { o = v; }
+__device__ __forceinline__ void from_f32(__nv_bfloat16& o, float v) { o = __float2bfloat16_rn(v); }
+__device__ __forceinline__ void from_f32(__half& o, float v) { o = __float2half_rn(v); }
+
+// Global row of image token (tile p, local slot l) inside one batch item.
+__device__ __forceinline__ int tile_token(int p, int l, int tiles_x, int th, int tw, int W) {
+  const int ty = p / tiles_x, tx = p - ty * tiles_x;
+  const int ly = l / tw, lx = l - ly * tw;
+  return (ty * th + ly) * W + tx * tw + lx;
+}
+
+}  // namespace toma

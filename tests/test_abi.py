@@ -1,0 +1,85 @@
+"""Host-only checks of the C-ABI library: it loads, exports every declared symbol, and
+rejects bad descriptors before launching anything.  No compute calls (no GPU needed)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import __graft_entry__ as entry
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def toma():
+    entry.build()
+    import paper_2509_10918_b200 as t
+    return t
+
+
+def test_every_declared_symbol_is_exported(toma):
+    header = open(os.path.join(ROOT, "include", "toma.h")).read()
+    declared = set(re.findall(r"TOMA_API[^;(]*?\b(toma_\w+)\s*\(", header))
+    assert declared, "no declarations found"
+    lib = ctypes.CDLL(toma.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), f"{name} is declared but not exported"
+    assert declared == set(toma.EXPORTS)
+
+
+def _desc(toma, **kw):
+    base = dict(batch=2, grid_h=64, grid_w=64, dim=640, tile_h=16, tile_w=16, merge_ratio=0.5, tau=0.1, n_heads=10,
+                head_dim=64, dtype="bf16")
+    base.update(kw)
+    return toma.make_desc(**base)
+
+
+def test_descriptor_validation(toma):
+    OK, SHAPE, DTYPE, RATIO, TAU, UNSUP = 0, 2, 3, 4, 5, 7
+    assert toma.toma_validate(_desc(toma)) == OK
+    assert toma.toma_validate(_desc(toma, tile_h=24)) == SHAPE          # does not divide the grid
+    assert toma.toma_validate(_desc(toma, dim=644, n_heads=7, head_dim=92)) == SHAPE  # dim % 8
+    assert toma.toma_validate(_desc(toma, n_heads=9)) == SHAPE
+    assert toma.toma_validate(_desc(toma, merge_ratio=1.0)) == RATIO
+    assert toma.toma_validate(_desc(toma, merge_ratio=-0.1)) == RATIO
+    assert toma.toma_validate(_desc(toma, merge_ratio=0.999)) == RATIO   # leaves no destination
+    assert toma.toma_validate(_desc(toma, tau=0.0)) == TAU
+    assert toma.toma_validate(_desc(toma, tau=float("nan"))) == TAU
+    assert toma.toma_validate(_desc(toma, tile_h=64, tile_w=32)) == UNSUP  # N_loc = 2048
+    assert toma.toma_validate(_desc(toma, reuse_interval=0)) == SHAPE
+    d = _desc(toma)
+    d.dtype = 5
+    assert toma.toma_validate(d) == DTYPE
+
+
+def test_sizes(toma):
+    d = _desc(toma)
+    assert toma.toma_dest_per_tile(d) == 128
+    assert toma.toma_weights_bytes(d) == 2 * 16 * 256 * 128 * 2
+    assert toma.toma_workspace_bytes(d) > 0
+    assert toma.toma_dest_per_tile(_desc(toma, merge_ratio=0.25)) == 192
+    assert toma.toma_dest_per_tile(_desc(toma, merge_ratio=0.75)) == 64
+    assert toma.toma_workspace_bytes(_desc(toma, tau=-1.0)) == 0
+    assert toma.toma_status_str(6).startswith("workspace")
+
+
+def test_null_and_workspace_errors_are_returned_before_any_launch(toma):
+    d = _desc(toma)
+    lib = toma.lib
+    NULL, WS = 1, 6
+    assert lib.toma_select(ctypes.byref(d), None, None, None, 0, None, None) == NULL
+    fake = ctypes.c_void_p(0x1000)  # never dereferenced: validation fails first
+    assert lib.toma_select(ctypes.byref(d), fake, fake, None, 0, None, None) == WS
+    assert lib.toma_select(ctypes.byref(d), fake, fake, fake, 16, None, None) == WS
+    assert lib.toma_merge(ctypes.byref(d), None, fake, fake, None, None) == NULL
+    assert lib.toma_attention(1, 0, 1, 64, 0, fake, fake, fake, fake, None, None) == 2
+    assert lib.toma_attention(1, 8, 1, 48, 0, fake, fake, fake, fake, None, None) == 7
+
+
+def test_binding_refuses_cpu_tensors(toma):
+    import torch
+    d = _desc(toma)
+    x = torch.zeros(4)
+    with pytest.raises(ValueError):
+        toma.toma_merge(d, x, x, x)

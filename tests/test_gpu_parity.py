@@ -1,0 +1,300 @@
+"""GPU-vs-oracle parity of every step of the ToMA block path, called through the C ABI.
+
+Tolerances (written here, as the target states them): selected indices bit-exact;
+bf16 tensors max-abs <= 2e-2 and relative Frobenius <= 1e-2; fp32 tensors max-abs <= 1e-4.
+"""
+import numpy as np
+import pytest
+import torch
+
+import gen
+from oracle import toma_oracle as O
+from tests._util import assert_close, sample_tiles, tile_tokens, to_dev, to_host64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def toma():
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2509_10918_b200 as t
+    return t
+
+
+class Run:
+    """Device buffers of one configuration plus the entry points bound to them."""
+
+    def __init__(self, toma, cfg, x_host, **desc_over):
+        self.t, self.cfg = toma, cfg
+        self.desc = toma.desc_from_config(cfg, **desc_over)
+        self.x = to_dev(x_host, cfg.dtype)
+        self.idx = toma.alloc_idx(self.desc)
+        self.w = toma.alloc_weights(self.desc)
+        self.ws = toma.alloc_workspace(self.desc)
+        self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        self.lm = cfg.n_merged + cfg.n_extra
+        self.xm = torch.empty((cfg.batch, self.lm, cfg.dim), dtype=self.x.dtype, device="cuda")
+
+    def ok(self):
+        torch.cuda.synchronize()
+        assert int(self.status.item()) == 0
+
+    def select(self):
+        self.t.toma_select(self.desc, self.x, self.idx, self.ws, self.status)
+        self.ok()
+        return self.idx.cpu().numpy().astype(np.int64)
+
+    def weights(self):
+        self.t.toma_merge_weights(self.desc, self.x, self.idx, self.w, self.ws, self.status)
+        self.ok()
+        c = self.cfg
+        dense = torch.empty((c.batch, c.n_tiles, c.d_loc, c.n_loc), dtype=torch.float32, device="cuda")
+        self.t.toma_weights_export(self.desc, self.w, dense)
+        torch.cuda.synchronize()
+        return dense.cpu().numpy().astype(np.float64)
+
+    def merge(self):
+        self.t.toma_merge(self.desc, self.w, self.x, self.xm, self.status)
+        self.ok()
+        return to_host64(self.xm)
+
+    def attend(self):
+        """Attention over the merged tokens (Q = K = V = merged), as toma_block does."""
+        c = self.cfg
+        att = torch.empty_like(self.xm)
+        self.t.toma_attention(c.batch, self.lm, c.n_heads, c.head_dim, c.dtype, self.xm, self.xm, self.xm, att,
+                              self.status)
+        self.ok()
+        return att
+
+    def unmerge(self, y):
+        out = torch.empty_like(self.x)
+        self.t.toma_unmerge(self.desc, self.w, y, out, self.status)
+        self.ok()
+        return to_host64(out)
+
+
+CASES = [
+    # name, overrides, number of tiles the oracle checks
+    ("cfg1", {}, 16),
+    ("cfg2", {}, 32),
+    ("cfg3", {"merge_ratio": 0.25}, 8),
+    ("cfg3", {"merge_ratio": 0.5}, 32),
+    ("cfg3", {"merge_ratio": 0.75}, 8),
+    ("cfg4", {}, 6),
+    ("cfg5a", {}, 8),
+    ("cfg5b", {}, 2),
+]
+
+
+@pytest.mark.parametrize("name,over,n_check", CASES, ids=[f"{n}-{'-'.join(map(str, o.values())) or 'base'}" for n, o, _ in CASES])
+def test_select_weights_merge_unmerge_parity(toma, name, over, n_check):
+    cfg = gen.config(name, **over)
+    x_host = gen.features(cfg)
+    run = Run(toma, cfg, x_host)
+    idx = run.select()
+    # properties that hold for every tile at full size
+    assert idx.min() >= 0 and idx.max() < cfg.n_loc
+    srt = np.sort(idx, axis=-1)
+    assert np.all(srt[..., 1:] != srt[..., :-1]), "a tile selected the same token twice"
+    dense = run.weights()
+    assert np.all(dense >= 0)
+    tol_rows = 1e-5 if cfg.dtype == "f32" else 2e-3
+    assert np.abs(dense.sum(-1) - 1.0).max() < tol_rows, "merge rows must sum to 1"
+    merged = run.merge()
+    # the unmerge input is what the block feeds it: the attention output over the merged tokens
+    # (already in storage dtype; the oracle unmerges this same tensor)
+    y_dev = run.attend()
+    unmerged = run.unmerge(y_dev)
+    y_host = to_host64(y_dev)
+    D = cfg.n_merged
+    if cfg.n_extra:
+        assert np.array_equal(merged[:, D:], x_host[:, cfg.n_tokens:].astype(np.float64))
+        assert np.array_equal(unmerged[:, cfg.n_tokens:], y_host[:, D:])
+    ids = O.tile_token_ids(cfg.grid_h, cfg.grid_w, cfg.tile_h, cfg.tile_w)
+    # fp32 logits up to ~512 carry a half-ulp of 3e-5, i.e. <= 1.5e-5 on a softmax share; fp16 storage adds 2^-11
+    w_abs = 2e-5 if cfg.dtype == "f32" else 6e-4
+    got_m, want_m, got_u, want_u = [], [], [], []
+    for b, p in sample_tiles(cfg, n_check):
+        xt = tile_tokens(cfg, x_host, b, p)
+        want_idx, margin = O.select_tile(xt, cfg.d_loc)
+        assert margin > O.FRAGILE_MARGIN, "input sits on a quantisation boundary; choose another seed"
+        assert np.array_equal(idx[b, p], want_idx), f"selection differs in tile ({b},{p})"
+        w = O.merge_weights(xt, want_idx, cfg.tau)
+        assert np.abs(dense[b, p] - w).max() <= w_abs, f"weights differ in tile ({b},{p})"
+        got_m.append(merged[b, p * cfg.d_loc:(p + 1) * cfg.d_loc])
+        want_m.append(O.merge(w, xt))
+        got_u.append(unmerged[b, ids[p]])
+        want_u.append(O.unmerge(w, y_host[b, p * cfg.d_loc:(p + 1) * cfg.d_loc]))
+    assert_close(np.stack(got_m), np.stack(want_m), cfg.dtype, "merge")
+    assert_close(np.stack(got_u), np.stack(want_u), cfg.dtype, "unmerge")
+
+
+ATT_CASES = [
+    ("f32", 1, 512, 10, 64, None),
+    ("bf16", 2, 512, 20, 64, None),
+    ("bf16", 2, 2048, 10, 64, 96),
+    ("bf16", 1, 2560, 24, 128, 64),
+    ("bf16", 2, 1000, 3, 64, None),   # ragged length
+    ("bf16", 1, 77, 2, 128, None),    # shorter than one tile
+    ("bf16", 4, 8192, 10, 64, 24),
+]
+
+
+@pytest.mark.parametrize("dtype,B,L,h,dh,n_rows", ATT_CASES)
+def test_attention_parity(toma, dtype, B, L, h, dh, n_rows):
+    rng_tag = (L * 131 + h * 7 + dh) % 1000
+    host = [gen.round_to_dtype(gen.normal(0, (77, rng_tag, i), B * L * h * dh).reshape(B, L, h * dh).astype(np.float32),
+                               dtype) for i in range(3)]
+    q, k, v = (to_dev(a, dtype) for a in host)
+    o = torch.empty_like(q)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    toma.toma_attention(B, L, h, dh, dtype, q, k, v, o, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    got = to_host64(o)
+    rows = None if n_rows is None else np.unique(np.concatenate(
+        [[0, L - 1], np.random.default_rng(L).choice(L, size=n_rows, replace=False)]))
+    for b in range(B):
+        want = O.attention(host[0][b], host[1][b], host[2][b], h, query_rows=rows)
+        assert_close(got[b] if rows is None else got[b][rows], want, dtype, f"attention b={b}")
+
+
+BLOCK_CASES = [
+    ("cfg1", {}, None),
+    ("cfg2", {}, None),
+    ("cfg3", {"steps": 6}, None),
+    ("cfg4", {}, None),
+]
+
+
+@pytest.mark.parametrize("name,over,_", BLOCK_CASES, ids=[c[0] for c in BLOCK_CASES])
+def test_block_sequence_parity(toma, name, over, _):
+    cfg = gen.config(name, **over)
+    desc = toma.desc_from_config(cfg)
+    idx = toma.alloc_idx(desc)
+    w = toma.alloc_weights(desc)
+    ws = toma.alloc_workspace(desc)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    st = O.BlockState()
+    kw = dict(grid_h=cfg.grid_h, grid_w=cfg.grid_w, tile_h=cfg.tile_h, tile_w=cfg.tile_w, merge_ratio=cfg.merge_ratio,
+              tau=cfg.tau, n_heads=cfg.n_heads, reuse_interval=cfg.reuse_interval, n_extra=cfg.n_extra)
+    for step, x_host in enumerate(gen.feature_sequence(cfg)):
+        x = to_dev(x_host, cfg.dtype)
+        out = torch.empty_like(x)
+        toma.toma_block(desc, step, x, out, idx, w, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        want, _, _ = O.block_step(x_host, step, st, **kw)
+        assert min(st.margins) > O.FRAGILE_MARGIN
+        assert np.array_equal(idx.cpu().numpy().astype(np.int64), st.idx), f"selection differs at step {step}"
+        assert_close(to_host64(out), want, cfg.dtype, f"block step {step}")
+
+
+def test_block_long_sequence_schedule_and_sampled_parity(toma):
+    """The 28-step stress sequence: selection may only change on refresh steps, and sampled
+    tiles of every refresh match the oracle exactly."""
+    cfg = gen.config("cfg5a", batch=1, steps=12)
+    desc = toma.desc_from_config(cfg)
+    idx = toma.alloc_idx(desc)
+    w = toma.alloc_weights(desc)
+    ws = toma.alloc_workspace(desc)
+    prev = None
+    tiles = sample_tiles(cfg, 4)
+    for step, x_host in enumerate(gen.feature_sequence(cfg)):
+        x = to_dev(x_host, cfg.dtype)
+        out = torch.empty_like(x)
+        toma.toma_block(desc, step, x, out, idx, w, ws, None)
+        torch.cuda.synchronize()
+        cur = idx.cpu().numpy().astype(np.int64)
+        if step % cfg.reuse_interval == 0:
+            for b, p in tiles:
+                want, margin = O.select_tile(tile_tokens(cfg, x_host, b, p), cfg.d_loc)
+                assert margin > O.FRAGILE_MARGIN
+                assert np.array_equal(cur[b, p], want)
+        else:
+            assert np.array_equal(cur, prev), "selection changed on a reuse step"
+        prev = cur
+        assert torch.isfinite(out.float()).all()
+
+
+def test_identity_weights_round_trip_is_bit_exact(toma):
+    for dtype in ("bf16", "f32"):
+        cfg = gen.config("cfg2", batch=1, grid_h=16, grid_w=16, dim=128, n_heads=2, merge_ratio=0.0, dtype=dtype)
+        assert cfg.d_loc == cfg.n_loc
+        x_host = gen.features(cfg)
+        run = Run(toma, cfg, x_host)
+        eye = torch.eye(cfg.n_loc, dtype=torch.float32, device="cuda").repeat(cfg.batch, cfg.n_tiles, 1, 1).contiguous()
+        toma.toma_weights_import(run.desc, eye, run.w)
+        merged = run.merge()
+        ids = O.tile_token_ids(cfg.grid_h, cfg.grid_w, cfg.tile_h, cfg.tile_w)
+        assert np.array_equal(merged[0], x_host[0][ids.reshape(-1)].astype(np.float64))
+        back = run.unmerge(run.xm)
+        assert np.array_equal(back, x_host.astype(np.float64))
+
+
+EDGE = [
+    dict(grid_h=12, grid_w=12, tile_h=6, tile_w=6, dim=64, n_heads=1, merge_ratio=0.5),      # N_loc = 36, not a warp multiple
+    dict(grid_h=16, grid_w=32, tile_h=2, tile_w=32, dim=128, n_heads=2, merge_ratio=0.5),    # stripes
+    dict(grid_h=16, grid_w=16, tile_h=8, tile_w=16, dim=64, n_heads=1, merge_ratio=0.99),    # one destination per tile
+    dict(grid_h=16, grid_w=16, tile_h=16, tile_w=8, dim=72, n_heads=1, head_dim=72, merge_ratio=0.3),  # odd dim, ragged D_loc
+    dict(grid_h=8, grid_w=8, tile_h=8, tile_w=8, dim=64, n_heads=1, merge_ratio=0.0),        # keep everything
+    dict(grid_h=16, grid_w=16, tile_h=8, tile_w=8, dim=64, n_heads=1, merge_ratio=0.5, n_extra=7),
+]
+
+
+@pytest.mark.parametrize("over", EDGE, ids=[str(i) for i in range(len(EDGE))])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_edge_shapes(toma, over, dtype):
+    cfg = gen.config("cfg2", batch=2, dtype=dtype, **over)
+    x_host = gen.features(cfg)
+    run = Run(toma, cfg, x_host)
+    idx = run.select()
+    dense = run.weights()
+    merged = run.merge()
+    # unmerge input: the merged tokens scaled by 1/4 (exact in both dtypes).  A source token that is
+    # split between destinations whose rows carry little mass has unmerge weights summing above 1, and
+    # values >= 8 cannot be stored in bf16 within 2e-2 by anyone; the scaling keeps them below that.
+    y_dev = (run.xm.float() * 0.25).to(run.xm.dtype)
+    unmerged = run.unmerge(y_dev)
+    y_host = to_host64(y_dev)
+    ids = O.tile_token_ids(cfg.grid_h, cfg.grid_w, cfg.tile_h, cfg.tile_w)
+    for b in range(cfg.batch):
+        for p in range(cfg.n_tiles):
+            xt = tile_tokens(cfg, x_host, b, p)
+            want_idx, margin = O.select_tile(xt, cfg.d_loc)
+            assert margin > O.FRAGILE_MARGIN
+            assert np.array_equal(idx[b, p], want_idx)
+            w = O.merge_weights(xt, want_idx, cfg.tau)
+            assert np.abs(dense[b, p] - w).max() <= (2e-5 if dtype == "f32" else 6e-4)
+            sl = slice(p * cfg.d_loc, (p + 1) * cfg.d_loc)
+            assert_close(merged[b, sl], O.merge(w, xt), dtype, "merge")
+            assert_close(unmerged[b, ids[p]], O.unmerge(w, y_host[b, sl]), dtype, "unmerge")
+
+
+def test_degenerate_inputs_identical_and_zero_tokens(toma):
+    cfg = gen.config("cfg2", batch=1, grid_h=8, grid_w=16, tile_h=8, tile_w=8, dim=64, n_heads=1)
+    x_host = np.zeros((1, 128, 64), dtype=np.float32)
+    x_host[0, :, :] = np.linspace(-1, 1, 64, dtype=np.float32)[None, :]   # all tokens identical
+    ids = O.tile_token_ids(8, 16, 8, 8)
+    x_host[0, ids[1][5]] = 0.0                                             # one zero-norm token in tile 1
+    x_host = gen.round_to_dtype(x_host, "bf16")
+    run = Run(toma, cfg, x_host)
+    idx = run.select()
+    assert list(idx[0, 0]) == list(range(32))                              # ties resolve to the lowest index
+    for p in range(2):
+        want, _ = O.select_tile(tile_tokens(cfg, x_host, 0, p), cfg.d_loc)
+        assert np.array_equal(idx[0, p], want)
+
+
+def test_results_are_deterministic(toma):
+    cfg = gen.config("cfg3", batch=1)
+    x_host = gen.features(cfg)
+    a = Run(toma, cfg, x_host)
+    b = Run(toma, cfg, x_host)
+    ia, ib = a.select(), b.select()
+    assert np.array_equal(ia, ib)
+    wa, wb = a.weights(), b.weights()
+    assert np.array_equal(wa, wb)
+    assert np.array_equal(a.merge(), b.merge())
