@@ -97,6 +97,7 @@ static cudaError_t do_unmerge(const Geom& g, const void* w, const void* y, void*
 
 static cudaError_t do_attention(int B, int L, int heads, int dh, bool f32, const void* q, const void* k,
                                 const void* v, void* o, uint32_t* dev_status, cudaStream_t s) {
+  if (!f32 && (dh == 64 || dh == 128)) return launch_attention_tc(B, L, heads, dh, q, k, v, o, dev_status, s);
   return launch_attention_simt(B, L, heads, dh, f32, q, k, v, o, s);
 }
 
