@@ -87,11 +87,19 @@ static cudaError_t do_weights(const Geom& g, const void* x, const int32_t* idx, 
 
 static cudaError_t do_merge(const Geom& g, const void* w, const void* x, void* xm, uint32_t* dev_status,
                             cudaStream_t s) {
+  if (linear_tc_supported(g)) {
+    cudaError_t e = launch_merge_tc(g, w, x, xm, dev_status, s);
+    return e != cudaSuccess ? e : launch_copy_extra(g, x, xm, true, s);
+  }
   return launch_merge_simt(g, w, x, xm, s);
 }
 
 static cudaError_t do_unmerge(const Geom& g, const void* w, const void* y, void* out, uint32_t* dev_status,
                               cudaStream_t s) {
+  if (linear_tc_supported(g)) {
+    cudaError_t e = launch_unmerge_tc(g, w, y, out, dev_status, s);
+    return e != cudaSuccess ? e : launch_copy_extra(g, y, out, false, s);
+  }
   return launch_unmerge_simt(g, w, y, out, s);
 }
 
@@ -121,7 +129,7 @@ size_t toma_workspace_bytes(const toma_desc* desc) {
 size_t toma_weights_bytes(const toma_desc* desc) {
   Geom g;
   if (make_geom(desc, &g) != TOMA_OK) return 0;
-  return (size_t)g.B * g.P * g.Nloc * g.Dloc * (g.f32 ? 4 : 2);
+  return (size_t)g.B * g.P * g.Nloc * g.Dloc * 4;  // one fp32 plane, or a hi and a lo bf16 plane
 }
 
 int32_t toma_dest_per_tile(const toma_desc* desc) {

@@ -85,7 +85,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     bar->abort_flag = 0;
     mbar_fence_init();
   }
-  if (warp == 1) tmem_alloc<C::kTmemCols>(&bar->tmem_base);
+  if (warp == 1) tmem_alloc(&bar->tmem_base, C::kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -254,7 +254,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc<C::kTmemCols>(tmem);
+    tmem_dealloc(tmem, C::kTmemCols);
   }
 }
 

@@ -50,6 +50,11 @@ cudaError_t launch_merge_simt(const Geom& g, const void* w, const void* x, void*
 cudaError_t launch_unmerge_simt(const Geom& g, const void* w, const void* y, void* out, cudaStream_t s);
 cudaError_t launch_attention_simt(int B, int L, int heads, int dh, bool f32, const void* q, const void* k,
                                   const void* v, void* o, cudaStream_t s);
+bool linear_tc_supported(const Geom& g);
+cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* xm, uint32_t* dev_status, cudaStream_t s);
+cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void* out, uint32_t* dev_status,
+                              cudaStream_t s);
+cudaError_t launch_copy_extra(const Geom& g, const void* src, void* dst, bool merging, cudaStream_t s);
 cudaError_t launch_attention_tc(int B, int L, int heads, int dh, const void* q, const void* k, const void* v, void* o,
                                 uint32_t* dev_status, cudaStream_t s);
 cudaError_t launch_weights_export(const Geom& g, const void* w, float* dense, cudaStream_t s);

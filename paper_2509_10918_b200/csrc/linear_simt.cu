@@ -62,6 +62,26 @@ struct TileMap {
   }
 };
 
+// Stored weights A~^T of one tile: fp32 mode keeps one fp32 plane [N_loc][D_loc]; bf16 mode keeps
+// the value split into two bf16 planes, hi = bf16(v) and lo = bf16(v - hi), hi plane first, so that
+// the tensor-core kernels can feed both planes as bf16 operands and still carry ~16 mantissa bits.
+__device__ __forceinline__ float w_load(const float* w, int batch, size_t off, size_t plane) {
+  return w[(size_t)batch * plane + off];
+}
+__device__ __forceinline__ float w_load(const __nv_bfloat16* w, int batch, size_t off, size_t plane) {
+  const __nv_bfloat16* t = w + (size_t)batch * 2 * plane;
+  return __bfloat162float(t[off]) + __bfloat162float(t[plane + off]);
+}
+__device__ __forceinline__ void w_store(float* w, int batch, size_t off, size_t plane, float v) {
+  w[(size_t)batch * plane + off] = v;
+}
+__device__ __forceinline__ void w_store(__nv_bfloat16* w, int batch, size_t off, size_t plane, float v) {
+  __nv_bfloat16* t = w + (size_t)batch * 2 * plane;
+  const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+  t[off] = hi;
+  t[plane + off] = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
 static TileMap make_map(const Geom& g) {
   return TileMap{g.P, g.tiles_x, g.th, g.tw, g.W, g.Nloc, g.Dloc, g.d, (int)g.tokens_all(), g.Lm};
 }
@@ -96,7 +116,7 @@ struct MergeOp {
   const T* x;
   T* xm;
   __device__ __forceinline__ float a(int batch, int i, int k) const {
-    return to_f32(w[((size_t)batch * tm.Nloc + k) * tm.Dloc + i]);
+    return w_load(w, batch, (size_t)k * tm.Dloc + i, (size_t)tm.Nloc * tm.Dloc);
   }
   __device__ __forceinline__ float b(int batch, int k, int c) const { return to_f32(x[tm.x_row(batch, k) * tm.d + c]); }
   __device__ __forceinline__ void store(int batch, int i, int c, float v) const {
@@ -114,7 +134,7 @@ struct UnmergeOp {
   const T* y;
   T* out;
   __device__ __forceinline__ float a(int batch, int k, int i) const {
-    return to_f32(w[((size_t)batch * tm.Nloc + k) * tm.Dloc + i]);
+    return w_load(w, batch, (size_t)k * tm.Dloc + i, (size_t)tm.Nloc * tm.Dloc);
   }
   __device__ __forceinline__ float b(int batch, int i, int c) const { return to_f32(y[tm.m_row(batch, i) * tm.d + c]); }
   __device__ __forceinline__ void store(int batch, int k, int c, float v) const {
@@ -161,8 +181,8 @@ __global__ void __launch_bounds__(256) rownorm_kernel(const float* __restrict__ 
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
   const float inv = z > 0.f ? 1.f / z : 0.f;
-  WT* wt = w + (size_t)batch * Nloc * Dloc + i;
-  for (int k = lane; k < Nloc; k += 32) from_f32(wt[(size_t)k * Dloc], a[k] * inv);
+  const size_t plane = (size_t)Nloc * Dloc;
+  for (int k = lane; k < Nloc; k += 32) w_store(w, batch, (size_t)k * Dloc + i, plane, a[k] * inv);
 }
 
 cudaError_t launch_weights_simt(const Geom& g, const void* x, const int32_t* idx, void* w, float* logits,
@@ -182,7 +202,7 @@ cudaError_t launch_weights_simt(const Geom& g, const void* x, const int32_t* idx
   if (g.f32)
     rownorm_kernel<float><<<blocks, 256, 0, s>>>(logits, (float*)w, g.Nloc, g.Dloc, rows);
   else
-    rownorm_kernel<__half><<<blocks, 256, 0, s>>>(logits, (__half*)w, g.Nloc, g.Dloc, rows);
+    rownorm_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(logits, (__nv_bfloat16*)w, g.Nloc, g.Dloc, rows);
   count_launch();
   return cudaGetLastError();
 }
@@ -211,6 +231,12 @@ static void copy_extra(const Geom& g, const T* src, T* dst, bool merging, cudaSt
   count_launch();
 }
 
+cudaError_t launch_copy_extra(const Geom& g, const void* src, void* dst, bool merging, cudaStream_t s) {
+  if (g.f32) copy_extra<float>(g, (const float*)src, (float*)dst, merging, s);
+  else copy_extra<__nv_bfloat16>(g, (const __nv_bfloat16*)src, (__nv_bfloat16*)dst, merging, s);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_merge_simt(const Geom& g, const void* w, const void* x, void* xm, cudaStream_t s) {
   const int batches = g.B * g.P;
   if (g.f32) {
@@ -218,9 +244,9 @@ cudaError_t launch_merge_simt(const Geom& g, const void* w, const void* x, void*
     run_gemm<MergeOp<float, float>, float>(op, batches, s);
     copy_extra<float>(g, (const float*)x, (float*)xm, true, s);
   } else {
-    MergeOp<__nv_bfloat16, __half> op{g.Dloc, g.d, g.Nloc, make_map(g), (const __half*)w, (const __nv_bfloat16*)x,
+    MergeOp<__nv_bfloat16, __nv_bfloat16> op{g.Dloc, g.d, g.Nloc, make_map(g), (const __nv_bfloat16*)w, (const __nv_bfloat16*)x,
                                       (__nv_bfloat16*)xm};
-    run_gemm<MergeOp<__nv_bfloat16, __half>, float>(op, batches, s);
+    run_gemm<MergeOp<__nv_bfloat16, __nv_bfloat16>, float>(op, batches, s);
     copy_extra<__nv_bfloat16>(g, (const __nv_bfloat16*)x, (__nv_bfloat16*)xm, true, s);
   }
   return cudaGetLastError();
@@ -233,9 +259,9 @@ cudaError_t launch_unmerge_simt(const Geom& g, const void* w, const void* y, voi
     run_gemm<UnmergeOp<float, float>, float>(op, batches, s);
     copy_extra<float>(g, (const float*)y, (float*)out, false, s);
   } else {
-    UnmergeOp<__nv_bfloat16, __half> op{g.Nloc, g.d, g.Dloc, make_map(g), (const __half*)w, (const __nv_bfloat16*)y,
+    UnmergeOp<__nv_bfloat16, __nv_bfloat16> op{g.Nloc, g.d, g.Dloc, make_map(g), (const __nv_bfloat16*)w, (const __nv_bfloat16*)y,
                                         (__nv_bfloat16*)out};
-    run_gemm<UnmergeOp<__nv_bfloat16, __half>, float>(op, batches, s);
+    run_gemm<UnmergeOp<__nv_bfloat16, __nv_bfloat16>, float>(op, batches, s);
     copy_extra<__nv_bfloat16>(g, (const __nv_bfloat16*)y, (__nv_bfloat16*)out, false, s);
   }
   return cudaGetLastError();
@@ -250,14 +276,14 @@ __global__ void weights_convert_kernel(WT* __restrict__ w, float* __restrict__ d
   const size_t batch = e / per, r = e - batch * per;
   const int k = (int)(r / Dloc), i = (int)(r - (size_t)k * Dloc);
   float* dp = dense + batch * per + (size_t)i * Nloc + k;
-  if (kExport) *dp = to_f32(w[e]); else from_f32(w[e], *dp);
+  if (kExport) *dp = w_load(w, (int)batch, r, per); else w_store(w, (int)batch, r, per, *dp);
 }
 
 cudaError_t launch_weights_export(const Geom& g, const void* w, float* dense, cudaStream_t s) {
   const size_t total = (size_t)g.B * g.P * g.Nloc * g.Dloc;
   const unsigned blocks = (unsigned)((total + 255) / 256);
   if (g.f32) weights_convert_kernel<float, true><<<blocks, 256, 0, s>>>((float*)w, dense, g.Nloc, g.Dloc, total);
-  else weights_convert_kernel<__half, true><<<blocks, 256, 0, s>>>((__half*)w, dense, g.Nloc, g.Dloc, total);
+  else weights_convert_kernel<__nv_bfloat16, true><<<blocks, 256, 0, s>>>((__nv_bfloat16*)w, dense, g.Nloc, g.Dloc, total);
   count_launch();
   return cudaGetLastError();
 }
@@ -266,7 +292,7 @@ cudaError_t launch_weights_import(const Geom& g, const float* dense, void* w, cu
   const size_t total = (size_t)g.B * g.P * g.Nloc * g.Dloc;
   const unsigned blocks = (unsigned)((total + 255) / 256);
   if (g.f32) weights_convert_kernel<float, false><<<blocks, 256, 0, s>>>((float*)w, (float*)dense, g.Nloc, g.Dloc, total);
-  else weights_convert_kernel<__half, false><<<blocks, 256, 0, s>>>((__half*)w, (float*)dense, g.Nloc, g.Dloc, total);
+  else weights_convert_kernel<__nv_bfloat16, false><<<blocks, 256, 0, s>>>((__nv_bfloat16*)w, (float*)dense, g.Nloc, g.Dloc, total);
   count_launch();
   return cudaGetLastError();
 }

@@ -1,0 +1,308 @@
+// Merge X_m = A~ X (Sec. 4.2.1) and unmerge A~^T X' (Sec. 4.2.2) per tile on the sm_100a
+// tensor cores: bf16 tokens, weights as a hi + lo pair of bf16 planes (two MMAs per step, ~16
+// mantissa bits), fp32 accumulation in tensor memory.
+//
+// Both are computed transposed, with 128 feature channels on the MMA M dimension:
+//   merge:    X_m^T [ch x D_loc] = X^T  [ch x N_loc] * A~^T [N_loc x D_loc]
+//   unmerge:  Y^T   [ch x N_loc] = X'^T [ch x D_loc] * A~   [D_loc x N_loc]
+// so the one stored weight layout A~^T [N_loc][D_loc] is the B operand of both (MN-major for the
+// merge, K-major for the unmerge) and the token tensors are MN-major A operands that TMA fetches
+// straight from their row-major [token][channel] storage: a spatial tile is one 4-D box of the
+// (channel, x, y, batch) view of X, so no gather/reshape pass exists.
+// One CTA = one (tile, 128-channel chunk, block of <= 256 output columns); warp 0 TMA, warp 1
+// MMA, warps 2..5 epilogue (one thread per channel).
+#include "common.cuh"
+#include "tc.cuh"
+
+namespace toma {
+
+using namespace tc;
+
+namespace {
+
+constexpr int kKC = 64;           // contraction elements per pipeline stage
+constexpr int kSlab = kKC * 128;  // bytes of a 64-row x 128-byte slab
+constexpr int kMaxCols = 256;     // output columns (MMA N) per CTA
+
+struct PipeBars {
+  uint64_t full[4], empty[4], done;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct LinParams {
+  int P, tiles_x, th, tw, W, Nloc, Dloc, d, n_all, Lm;
+  int stages;  // pipeline depth
+};
+
+__device__ __forceinline__ uint32_t tmem_cols_for(int n) { return n > 128 ? 256u : n > 64 ? 128u : 64u; }
+
+__device__ __forceinline__ void pipe_init(PipeBars* bar, int stages) {
+  for (int s = 0; s < stages; ++s) {
+    mbar_init(&bar->full[s], 1);
+    mbar_init(&bar->empty[s], 1);
+  }
+  mbar_init(&bar->done, 1);
+  bar->abort_flag = 0;
+  mbar_fence_init();
+}
+
+// ------------------------------------------------------------------------------------------------
+// merge: grid (tile, channel chunk, destination block); K loop over the tile's tokens.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(192, 1)
+merge_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+                __nv_bfloat16* __restrict__ xm, const LinParams p, uint32_t* dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int batch = blockIdx.x, c0 = blockIdx.y * 128, i_base = blockIdx.z * kMaxCols;
+  const int n_dest = min(kMaxCols, p.Dloc - i_base);  // destinations this CTA produces
+  const int slabs = (n_dest + 63) / 64;               // 64-destination slabs per weight plane
+  const int n_mma = slabs * 64;                       // MMA N (zero padded by TMA)
+  const int stage_bytes = (2 + 2 * slabs) * kSlab;
+  PipeBars* bar = reinterpret_cast<PipeBars*>(smem + p.stages * stage_bytes);
+  const int b = batch / p.P, tile = batch - b * p.P;
+  const int ty = tile / p.tiles_x, tx = tile - ty * p.tiles_x;
+  const int rows_per_chunk = kKC / p.tw;
+  const int nk = p.Nloc / kKC;
+  const uint32_t ncols = tmem_cols_for(n_mma);
+
+  if (threadIdx.x == 0) pipe_init(bar, p.stages);
+  if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bar->tmem_base;
+  volatile int* abort_flag = &bar->abort_flag;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tmap(&tm_x);
+      prefetch_tmap(&tm_w);
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % p.stages;
+        if (k >= p.stages && !mbar_wait(&bar->empty[s], ((k / p.stages) - 1) & 1, dev_status, abort_flag)) break;
+        uint8_t* sx = smem + s * stage_bytes;
+        uint8_t* sw = sx + 2 * kSlab;
+        mbar_expect_tx(&bar->full[s], stage_bytes);
+        for (int c = 0; c < 2; ++c)
+          tma_load_4d(sx + c * kSlab, &tm_x, &bar->full[s], c0 + c * 64, tx * p.tw, ty * p.th + k * rows_per_chunk, b);
+        for (int pl = 0; pl < 2; ++pl)
+          for (int c = 0; c < slabs; ++c)
+            tma_load_3d(sw + (pl * slabs + c) * kSlab, &tm_w, &bar->full[s], i_base + c * 64, k * kKC, 2 * batch + pl);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = idesc_f16(kFmtBF16, kFmtBF16, true, true, 128, n_mma);
+      bool ok = true;
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % p.stages;
+        if (!mbar_wait(&bar->full[s], (k / p.stages) & 1, dev_status, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t xa = smem_u32(smem + s * stage_bytes), wa = xa + 2 * kSlab;
+#pragma unroll
+        for (int kk = 0; kk < kKC / 16; ++kk) {  // 16 tokens per MMA: 16 rows of 128 B in every slab
+          const uint64_t xd = smem_desc_sw128(xa + kk * 2048, kSlab, 1024);
+          mma_ss(tmem, xd, smem_desc_sw128(wa + kk * 2048, kSlab, 1024), idesc, k > 0 || kk > 0);
+          mma_ss(tmem, xd, smem_desc_sw128(wa + slabs * kSlab + kk * 2048, kSlab, 1024), idesc, true);
+        }
+        mma_commit(&bar->empty[s]);
+      }
+      if (ok) mma_commit(&bar->done);
+    }
+  } else {
+    const int quarter = warp & 3;
+    const int ch = c0 + quarter * 32 + lane;
+    const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16);
+    if (mbar_wait(&bar->done, 0, dev_status, abort_flag)) {
+      tc_fence_after();
+      __nv_bfloat16* dst = xm + ((size_t)b * p.Lm + (size_t)tile * p.Dloc + i_base) * p.d + ch;
+      for (int i0 = 0; i0 < n_dest; i0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + i0, r);
+        tmem_wait_ld();
+        if (ch < p.d) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            if (i0 + e < n_dest) dst[(size_t)(i0 + e) * p.d] = __float2bfloat16_rn(__uint_as_float(r[e]));
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, ncols);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// unmerge: grid (tile, channel chunk, token block); K loop over the tile's destinations.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(192, 1)
+unmerge_tc_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_w,
+                  __nv_bfloat16* __restrict__ out, const LinParams p, int n_tok, uint32_t* dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int w_plane = n_tok * 128;  // bytes of one [n_tok tokens][64 destinations] weight block
+  const int stage_bytes = 2 * kSlab + 2 * w_plane;
+  PipeBars* bar = reinterpret_cast<PipeBars*>(smem + p.stages * stage_bytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int batch = blockIdx.x, c0 = blockIdx.y * 128, t0 = blockIdx.z * n_tok;
+  const int b = batch / p.P, tile = batch - b * p.P;
+  const int nk = (p.Dloc + kKC - 1) / kKC;
+  const uint32_t ncols = tmem_cols_for(n_tok);
+
+  if (threadIdx.x == 0) pipe_init(bar, p.stages);
+  if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bar->tmem_base;
+  volatile int* abort_flag = &bar->abort_flag;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tmap(&tm_y);
+      prefetch_tmap(&tm_w);
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % p.stages;
+        if (k >= p.stages && !mbar_wait(&bar->empty[s], ((k / p.stages) - 1) & 1, dev_status, abort_flag)) break;
+        uint8_t* sy = smem + s * stage_bytes;
+        uint8_t* sw = sy + 2 * kSlab;
+        mbar_expect_tx(&bar->full[s], stage_bytes);
+        for (int c = 0; c < 2; ++c)
+          tma_load_3d(sy + c * kSlab, &tm_y, &bar->full[s], c0 + c * 64, tile * p.Dloc + k * kKC, b);
+        for (int pl = 0; pl < 2; ++pl) tma_load_3d(sw + pl * w_plane, &tm_w, &bar->full[s], k * kKC, t0, 2 * batch + pl);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = idesc_f16(kFmtBF16, kFmtBF16, true, false, 128, n_tok);
+      bool ok = true;
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % p.stages;
+        if (!mbar_wait(&bar->full[s], (k / p.stages) & 1, dev_status, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t ya = smem_u32(smem + s * stage_bytes), wa = ya + 2 * kSlab;
+        const int ksteps = min(kKC, p.Dloc - k * kKC + 15) / 16;  // 16 destinations per MMA
+        for (int kk = 0; kk < ksteps; ++kk) {
+          const uint64_t yd = smem_desc_sw128(ya + kk * 2048, kSlab, 1024);
+          mma_ss(tmem, yd, smem_desc_sw128(wa + kk * 32, 16, 1024), idesc, k > 0 || kk > 0);
+          mma_ss(tmem, yd, smem_desc_sw128(wa + w_plane + kk * 32, 16, 1024), idesc, true);
+        }
+        mma_commit(&bar->empty[s]);
+      }
+      if (ok) mma_commit(&bar->done);
+    }
+  } else {
+    const int quarter = warp & 3;
+    const int ch = c0 + quarter * 32 + lane;
+    const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16);
+    if (mbar_wait(&bar->done, 0, dev_status, abort_flag)) {
+      tc_fence_after();
+      __nv_bfloat16* base = out + (size_t)b * p.n_all * p.d + ch;
+      for (int l0 = 0; l0 < n_tok; l0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + l0, r);
+        tmem_wait_ld();
+        if (ch < p.d) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const int tok = tile_token(tile, t0 + l0 + e, p.tiles_x, p.th, p.tw, p.W);
+            base[(size_t)tok * p.d] = __float2bfloat16_rn(__uint_as_float(r[e]));
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, ncols);
+  }
+}
+
+LinParams make_params(const Geom& g) {
+  LinParams p;
+  p.P = g.P; p.tiles_x = g.tiles_x; p.th = g.th; p.tw = g.tw; p.W = g.W; p.Nloc = g.Nloc; p.Dloc = g.Dloc;
+  p.d = g.d; p.n_all = (int)g.tokens_all(); p.Lm = g.Lm; p.stages = 2;
+  return p;
+}
+
+// Weight planes as a 3-D tensor (destination, token, plane): plane 2*tile is hi, 2*tile + 1 is lo.
+bool encode_w(const Geom& g, const void* w, CUtensorMap* tm, uint32_t box_tokens) {
+  const uint64_t dims[3] = {(uint64_t)g.Dloc, (uint64_t)g.Nloc, (uint64_t)g.B * g.P * 2};
+  const uint64_t strides[2] = {(uint64_t)g.Dloc * 2, (uint64_t)g.Nloc * g.Dloc * 2};
+  const uint32_t box[3] = {64, box_tokens, 1};
+  return encode_tmap_16bit(tm, w, 3, dims, strides, box);
+}
+
+cudaError_t raise_smem_limit(const void* fn, bool* done) {
+  if (*done) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e == cudaSuccess) *done = true;
+  return e;
+}
+
+}  // namespace
+
+// Shapes the tensor-core merge / unmerge cover; everything else runs on the FFMA kernels.
+bool linear_tc_supported(const Geom& g) {
+  if (g.f32) return false;
+  if (g.tw > 64 || (64 % g.tw) != 0 || (g.th % (64 / g.tw)) != 0) return false;  // 64 tokens = whole tile rows
+  if (g.Nloc % 64 != 0 || g.Dloc % 8 != 0) return false;
+  if (g.Nloc > kMaxCols && g.Nloc % kMaxCols != 0) return false;  // unmerge token blocks
+  return true;
+}
+
+cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* xm, uint32_t* dev_status,
+                            cudaStream_t s) {
+  CUtensorMap tx, tw;
+  const uint64_t dims[4] = {(uint64_t)g.d, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.B};
+  const uint64_t strides[3] = {(uint64_t)g.d * 2, (uint64_t)g.W * g.d * 2, (uint64_t)g.tokens_all() * g.d * 2};
+  const uint32_t box[4] = {64, (uint32_t)g.tw, (uint32_t)(64 / g.tw), 1};
+  if (!encode_tmap_16bit(&tx, x, 4, dims, strides, box) || !encode_w(g, w, &tw, 64)) return cudaErrorInvalidValue;
+  LinParams p = make_params(g);
+  const int slabs = ((g.Dloc < kMaxCols ? g.Dloc : kMaxCols) + 63) / 64;
+  const int stage_bytes = (2 + 2 * slabs) * kSlab;
+  p.stages = stage_bytes <= 48 * 1024 ? 4 : 2;
+  if (p.stages > g.Nloc / kKC) p.stages = g.Nloc / kKC;
+  const int smem = 1024 + p.stages * stage_bytes + 256;
+  static bool attr = false;
+  cudaError_t e = raise_smem_limit((const void*)merge_tc_kernel, &attr);
+  if (e != cudaSuccess) return e;
+  dim3 grid(g.B * g.P, (g.d + 127) / 128, (g.Dloc + kMaxCols - 1) / kMaxCols);
+  merge_tc_kernel<<<grid, 192, smem, s>>>(tx, tw, (__nv_bfloat16*)xm, p, dev_status);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void* out, uint32_t* dev_status,
+                              cudaStream_t s) {
+  CUtensorMap ty, tw;
+  const int n_tok = g.Nloc > kMaxCols ? kMaxCols : g.Nloc;
+  const uint64_t dims[3] = {(uint64_t)g.d, (uint64_t)g.Lm, (uint64_t)g.B};
+  const uint64_t strides[2] = {(uint64_t)g.d * 2, (uint64_t)g.Lm * g.d * 2};
+  const uint32_t box[3] = {64, 64, 1};
+  if (!encode_tmap_16bit(&ty, y, 3, dims, strides, box) || !encode_w(g, w, &tw, (uint32_t)n_tok))
+    return cudaErrorInvalidValue;
+  LinParams p = make_params(g);
+  const int stage_bytes = 2 * kSlab + 2 * n_tok * 128;
+  p.stages = stage_bytes <= 48 * 1024 ? 4 : 2;
+  if (p.stages > (g.Dloc + kKC - 1) / kKC) p.stages = (g.Dloc + kKC - 1) / kKC;
+  const int smem = 1024 + p.stages * stage_bytes + 256;
+  static bool attr = false;
+  cudaError_t e = raise_smem_limit((const void*)unmerge_tc_kernel, &attr);
+  if (e != cudaSuccess) return e;
+  dim3 grid(g.B * g.P, (g.d + 127) / 128, g.Nloc / n_tok);
+  unmerge_tc_kernel<<<grid, 192, smem, s>>>(ty, tw, (__nv_bfloat16*)out, p, n_tok, dev_status);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace toma

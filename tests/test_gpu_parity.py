@@ -113,7 +113,7 @@ def test_select_weights_merge_unmerge_parity(toma, name, over, n_check):
         assert np.array_equal(merged[:, D:], x_host[:, cfg.n_tokens:].astype(np.float64))
         assert np.array_equal(unmerged[:, cfg.n_tokens:], y_host[:, D:])
     ids = O.tile_token_ids(cfg.grid_h, cfg.grid_w, cfg.tile_h, cfg.tile_w)
-    # fp32 logits up to ~512 carry a half-ulp of 3e-5, i.e. <= 1.5e-5 on a softmax share; fp16 storage adds 2^-11
+    # fp32 logits up to ~512 carry a half-ulp of 3e-5, i.e. <= 1.5e-5 on a softmax share; bf16 mode: fp32 accumulation over d terms perturbs a logit of ~400 by up to ~1e-3, i.e. 2.5e-4 on a share
     w_abs = 2e-5 if cfg.dtype == "f32" else 6e-4
     got_m, want_m, got_u, want_u = [], [], [], []
     for b, p in sample_tiles(cfg, n_check):
