@@ -74,7 +74,7 @@ static cudaError_t do_select(const Geom& g, const void* x, int32_t* idx, char* w
   int16_t* sq = (int16_t*)(ws + l.sq_off);
   cudaError_t e = launch_quantise(g, x, y, s);
   if (e != cudaSuccess) return e;
-  e = launch_gram_ffma(g, y, sq, s);
+  e = gram_tc_supported(g) ? launch_gram_tc(g, y, sq, dev_status, s) : launch_gram_ffma(g, y, sq, s);
   if (e != cudaSuccess) return e;
   return launch_greedy(g, sq, idx, s);
 }

@@ -43,6 +43,8 @@ inline void count_launch(int n = 1) { g_launches.fetch_add((unsigned long long)n
 // ---- launchers (each returns cudaGetLastError() of its launches) ----
 cudaError_t launch_quantise(const Geom& g, const void* x, __nv_bfloat16* y, cudaStream_t s);
 cudaError_t launch_gram_ffma(const Geom& g, const __nv_bfloat16* y, int16_t* sq, cudaStream_t s);
+bool gram_tc_supported(const Geom& g);
+cudaError_t launch_gram_tc(const Geom& g, const __nv_bfloat16* y, int16_t* sq, uint32_t* dev_status, cudaStream_t s);
 cudaError_t launch_greedy(const Geom& g, const int16_t* sq, int32_t* idx, cudaStream_t s);
 cudaError_t launch_weights_simt(const Geom& g, const void* x, const int32_t* idx, void* w, float* logits,
                                 cudaStream_t s);

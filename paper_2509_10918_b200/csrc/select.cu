@@ -54,7 +54,8 @@ cudaError_t launch_quantise(const Geom& g, const void* x, __nv_bfloat16* y, cuda
 // Gram, FFMA version: S_q[i][j] = rint(<y_i, y_j> * 4096), diag = 4014.
 // 64x64 output block per CTA, 4x4 per thread, 32-channel chunks in shared memory.
 // The fp32 sum is exact in any order (every partial sum is a multiple of 2^-24
-// below 1), so this equals the integer definition.
+// below 1), so this equals the integer definition.  Used for tile sizes the
+// tensor-core version does not cover.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) gram_ffma_kernel(const __nv_bfloat16* __restrict__ y,
                                                         int16_t* __restrict__ sq, int Nloc, int d) {
@@ -94,7 +95,8 @@ __global__ void __launch_bounds__(256) gram_ffma_kernel(const __nv_bfloat16* __r
 #pragma unroll
     for (int v = 0; v < 4; ++v) {
       const int i = i0 + ty * 4 + u, j = j0 + tx * 4 + v;
-      if (i < Nloc && j < Nloc) S[(size_t)i * Nloc + j] = (i == j) ? (int16_t)kDiagQ : (int16_t)__float2int_rn(acc[u][v] * 4096.f);
+      if (i < Nloc && j < Nloc)
+        S[(size_t)i * Nloc + j] = (i == j) ? (int16_t)kDiagQ : (int16_t)__float2int_rn(acc[u][v] * 4096.f);
     }
 }
 
@@ -114,7 +116,12 @@ cudaError_t launch_gram_ffma(const Geom& g, const __nv_bfloat16* y, int16_t* sq,
 // All quantities are integers, so this equals recomputing
 //   g_i = sum_j relu(S[i][j] - m[j])
 // from scratch every round.  S is symmetric; it is always read as S[j][i] with
-// i = thread index so that a warp reads consecutive int16.
+// i = thread index so that a warp reads consecutive int16.  Thread i also owns
+// m[i] in a register.  For N_loc <= 256 the tile's S_q (<= 128 KB) is first
+// copied to shared memory so that the two dependent reads of every round cost a
+// shared-memory latency instead of an L2 round trip.
+// Two block barriers per round: after the per-warp argmax partials are posted,
+// and after the changed-column list is posted (both double buffered).
 // Ties: lowest index.  Selected tokens are excluded from the argmax.
 // ---------------------------------------------------------------------------
 struct ArgMax {
@@ -123,34 +130,41 @@ struct ArgMax {
 __device__ __forceinline__ ArgMax better(ArgMax a, ArgMax b) {
   return (b.g > a.g || (b.g == a.g && b.i < a.i)) ? b : a;
 }
-__device__ __forceinline__ ArgMax block_argmax(ArgMax v, ArgMax* red, int nwarps) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+__device__ __forceinline__ ArgMax warp_argmax(ArgMax v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     ArgMax other{__shfl_xor_sync(0xffffffffu, v.g, o), __shfl_xor_sync(0xffffffffu, v.i, o)};
     v = better(v, other);
   }
+  return v;
+}
+// Posts this warp's best into red[], one barrier, then every warp reduces the partials itself.
+__device__ __forceinline__ ArgMax block_argmax(ArgMax v, ArgMax* red, int nwarps) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  v = warp_argmax(v);
   if (lane == 0) red[warp] = v;
   __syncthreads();
-  ArgMax r = red[lane < nwarps ? lane : 0];
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    ArgMax other{__shfl_xor_sync(0xffffffffu, r.g, o), __shfl_xor_sync(0xffffffffu, r.i, o)};
-    r = better(r, other);
-  }
-  __syncthreads();  // red[] may be rewritten by the next call
-  return r;
+  return warp_argmax(red[lane < nwarps ? lane : 0]);
 }
 
+template <bool kSmemS>
 __global__ void __launch_bounds__(1024) greedy_kernel(const int16_t* __restrict__ sq, int32_t* __restrict__ idx,
                                                       int Nloc, int Dloc) {
-  __shared__ int m[kMaxNloc];
-  __shared__ int ch_j[kMaxNloc];
-  __shared__ int ch_old[kMaxNloc];
-  __shared__ int ch_new[kMaxNloc];
-  __shared__ ArgMax red[32];
-  __shared__ int n_changed;
-  const int16_t* S = sq + (size_t)blockIdx.x * Nloc * Nloc;
+  extern __shared__ __align__(16) uint8_t greedy_smem[];
+  __shared__ int2 changed[2][kMaxNloc];  // (column j, new << 16 | old & 0xffff)
+  __shared__ ArgMax red[2][32];
+  __shared__ int n_changed[2];
+  const int16_t* Sg = sq + (size_t)blockIdx.x * Nloc * Nloc;
+  const int16_t* S = Sg;
+  if (threadIdx.x == 0) n_changed[0] = n_changed[1] = 0;
+  if (kSmemS) {
+    const int n16 = Nloc * Nloc / 8;  // 16-byte packets
+    const uint4* src = reinterpret_cast<const uint4*>(Sg);
+    uint4* dst = reinterpret_cast<uint4*>(greedy_smem);
+    for (int e = threadIdx.x; e < n16; e += blockDim.x) dst[e] = src[e];
+    S = reinterpret_cast<const int16_t*>(greedy_smem);
+  }
+  __syncthreads();
   int32_t* out = idx + (size_t)blockIdx.x * Dloc;
   const int i = threadIdx.x;
   const bool live = i < Nloc;
@@ -161,51 +175,69 @@ __global__ void __launch_bounds__(1024) greedy_kernel(const int16_t* __restrict_
   int sum = 0;
   if (live)
     for (int j = 0; j < Nloc; ++j) sum += S[(size_t)j * Nloc + i];
-  ArgMax pick = block_argmax(ArgMax{live ? sum : kNever, i}, red, nwarps);
+  ArgMax pick = block_argmax(ArgMax{live ? sum : kNever, i}, red[0], nwarps);
   bool selected = false;
   if (i == pick.i) {
     selected = true;
     out[0] = pick.i;
   }
-  if (live) m[i] = S[(size_t)pick.i * Nloc + i];
-  __syncthreads();
+  // cached maximum m[j] = S[t1][j]; thread i keeps m[i]; the full row is needed once for the initial gains
+  int m_own = live ? S[(size_t)pick.i * Nloc + i] : 0;
   int gain = 0;
-  if (live)
-    for (int j = 0; j < Nloc; ++j) gain += max((int)S[(size_t)j * Nloc + i] - m[j], 0);
+  if (live) {
+    const int16_t* mrow = S + (size_t)pick.i * Nloc;
+    for (int j = 0; j < Nloc; ++j) gain += max((int)S[(size_t)j * Nloc + i] - (int)mrow[j], 0);
+  }
 
   for (int r = 1; r < Dloc; ++r) {
-    if (threadIdx.x == 0) n_changed = 0;
-    pick = block_argmax(ArgMax{(live && !selected) ? gain : kNever, i}, red, nwarps);
+    const int pb = r & 1;
+    pick = block_argmax(ArgMax{(live && !selected) ? gain : kNever, i}, red[pb], nwarps);
     if (i == pick.i) {
       selected = true;
       out[r] = pick.i;
     }
-    if (live) {
-      const int s_new = S[(size_t)pick.i * Nloc + i];
-      const int s_old = m[i];
-      if (s_new > s_old) {
-        const int slot = atomicAdd(&n_changed, 1);
-        ch_j[slot] = i;
-        ch_old[slot] = s_old;
-        ch_new[slot] = s_new;
-        m[i] = s_new;
+    // columns whose cached maximum improves
+    const int s_new = live ? (int)S[(size_t)pick.i * Nloc + i] : 0;
+    const bool ch = live && s_new > m_own;
+    const unsigned mask = __ballot_sync(0xffffffffu, ch);
+    if (mask) {
+      const int lane = threadIdx.x & 31;
+      int base = 0;
+      if (lane == 0) base = atomicAdd(&n_changed[pb], __popc(mask));
+      base = __shfl_sync(0xffffffffu, base, 0);
+      if (ch) {
+        changed[pb][base + __popc(mask & ((1u << lane) - 1u))] = make_int2(i, (int)(((unsigned)s_new << 16) | ((unsigned)m_own & 0xFFFFu)));
+        m_own = s_new;
       }
     }
     __syncthreads();
+    const int n = n_changed[pb];
+    if (threadIdx.x == 0) n_changed[pb ^ 1] = 0;  // last read one full round ago
     if (live) {
-      const int n = n_changed;
       for (int e = 0; e < n; ++e) {
-        const int s = S[(size_t)ch_j[e] * Nloc + i];
-        gain += max(s - ch_new[e], 0) - max(s - ch_old[e], 0);
+        const int2 c = changed[pb][e];
+        const int s = S[(size_t)c.x * Nloc + i];
+        gain += max(s - (c.y >> 16), 0) - max(s - (int)(short)(c.y & 0xFFFF), 0);
       }
     }
-    __syncthreads();
   }
 }
 
 cudaError_t launch_greedy(const Geom& g, const int16_t* sq, int32_t* idx, cudaStream_t s) {
   const int threads = ((g.Nloc + 31) / 32) * 32;
-  greedy_kernel<<<g.B * g.P, threads, 0, s>>>(sq, idx, g.Nloc, g.Dloc);
+  const size_t s_bytes = (size_t)g.Nloc * g.Nloc * 2;
+  const bool smem_s = g.Nloc <= 256 && (g.Nloc * g.Nloc) % 8 == 0;
+  if (smem_s) {
+    static bool attr = false;
+    if (!attr) {
+      cudaError_t e = cudaFuncSetAttribute(greedy_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * 256 * 2);
+      if (e != cudaSuccess) return e;
+      attr = true;
+    }
+    greedy_kernel<true><<<g.B * g.P, threads, s_bytes, s>>>(sq, idx, g.Nloc, g.Dloc);
+  } else {
+    greedy_kernel<false><<<g.B * g.P, threads, 0, s>>>(sq, idx, g.Nloc, g.Dloc);
+  }
   count_launch();
   return cudaGetLastError();
 }
