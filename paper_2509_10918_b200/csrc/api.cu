@@ -47,6 +47,7 @@ WsLayout ws_layout(const Geom& g) {
   l.y_off = off;      off = align_up(off + tiles * g.Nloc * g.d * sizeof(__nv_bfloat16), 256);
   l.sq_off = off;     off = align_up(off + tiles * g.Nloc * g.Nloc * sizeof(int16_t), 256);
   l.logits_off = off; off = align_up(off + tiles * g.Dloc * g.Nloc * sizeof(float), 256);
+  l.wts_off = off;    off = align_up(off + (weights_tc_supported(g) ? weights_tc_scratch_bytes(g) : 0), 256);
   l.xm_off = off;     off = align_up(off + (size_t)g.B * g.Lm * g.d * esz, 256);
   l.att_off = off;    off = align_up(off + (size_t)g.B * g.Lm * g.d * esz, 256);
   l.total = off;
@@ -82,6 +83,8 @@ static cudaError_t do_select(const Geom& g, const void* x, int32_t* idx, char* w
 static cudaError_t do_weights(const Geom& g, const void* x, const int32_t* idx, void* w, char* ws,
                               uint32_t* dev_status, cudaStream_t s) {
   const WsLayout l = ws_layout(g);
+  if (weights_tc_supported(g))
+    return launch_weights_tc(g, x, idx, w, (float*)(ws + l.logits_off), ws + l.wts_off, dev_status, s);
   return launch_weights_simt(g, x, idx, w, (float*)(ws + l.logits_off), s);
 }
 

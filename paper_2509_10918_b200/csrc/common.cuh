@@ -32,7 +32,7 @@ toma_status make_geom(const toma_desc* desc, Geom* g);
 
 // Workspace carve-up (all offsets 256-byte aligned).
 struct WsLayout {
-  size_t y_off, sq_off, logits_off, xm_off, att_off, total;
+  size_t y_off, sq_off, logits_off, wts_off, xm_off, att_off, total;
 };
 WsLayout ws_layout(const Geom& g);
 
@@ -52,6 +52,10 @@ cudaError_t launch_merge_simt(const Geom& g, const void* w, const void* x, void*
 cudaError_t launch_unmerge_simt(const Geom& g, const void* w, const void* y, void* out, cudaStream_t s);
 cudaError_t launch_attention_simt(int B, int L, int heads, int dh, bool f32, const void* q, const void* k,
                                   const void* v, void* o, cudaStream_t s);
+bool weights_tc_supported(const Geom& g);
+size_t weights_tc_scratch_bytes(const Geom& g);
+cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, void* w, float* shares, void* scratch,
+                              uint32_t* dev_status, cudaStream_t s);
 bool linear_tc_supported(const Geom& g);
 cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* xm, uint32_t* dev_status, cudaStream_t s);
 cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void* out, uint32_t* dev_status,

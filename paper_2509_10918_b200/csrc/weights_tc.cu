@@ -1,0 +1,286 @@
+// Merge weights (Sec. 4.2.1) on the tensor cores, bf16 mode.
+//
+//   1. gather_dest_kernel: copies the D_loc selected tokens of every tile into a dense
+//      [tile][D_loc][d] buffer so that TMA can feed them as an MMA operand.
+//   2. weights_logits_kernel: L^T [source k][destination i] = <X_k, X_idx_i> with 128 source
+//      tokens on the MMA M dimension, so each epilogue thread owns one source token and the softmax
+//      over the DESTINATION axis (a source token's shares sum to 1) is a private register
+//      reduction over its tensor-memory row.  Writes the shares A_ik (fp32) and, per 128-source
+//      block, the partial row sums sum_k A_ik.
+//   3. weights_normalise_kernel: A~_ik = A_ik / sum_k' A_ik' with the partial sums added in a
+//      fixed order, stored as A~^T [N_loc][D_loc] split into a hi and a lo bf16 plane.
+#include "common.cuh"
+#include "tc.cuh"
+
+namespace toma {
+
+using namespace tc;
+
+namespace {
+
+constexpr int kKC = 64;
+
+struct WBars {
+  uint64_t full[4], empty[4], done;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct WParams {
+  int P, tiles_x, th, tw, W, Nloc, Dloc, d, n_all;
+  int m_tok;    // source tokens per CTA (128, or N_loc when the tile is smaller)
+  int stages;
+  float scale_log2;  // log2(e) / (tau * sqrt(d))
+};
+
+__global__ void __launch_bounds__(256)
+gather_dest_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ idx, __nv_bfloat16* __restrict__ dg,
+                   WParams p, int rows_total) {
+  const int vec_per_row = p.d / 8;  // 16-byte packets
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= (long long)rows_total * vec_per_row) return;
+  const int row = (int)(e / vec_per_row), v = (int)(e - (long long)row * vec_per_row);
+  const int batch = row / p.Dloc;
+  const int b = batch / p.P, tile = batch - b * p.P;
+  const int tok = tile_token(tile, idx[row], p.tiles_x, p.th, p.tw, p.W);
+  const uint4* src = reinterpret_cast<const uint4*>(x + ((size_t)b * p.n_all + tok) * p.d) + v;
+  reinterpret_cast<uint4*>(dg + (size_t)row * p.d)[v] = *src;
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__global__ void __launch_bounds__(192, 1)
+weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_d,
+                      float* __restrict__ shares, float* __restrict__ zpart, const WParams p, uint32_t* dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int n_mma = (p.Dloc + 15) & ~15;          // MMA N: destinations padded to 16
+  const int n0 = n_mma > 256 ? 256 : n_mma, n1 = n_mma - n0;
+  const int a_bytes = 128 * 128;
+  const int b_rows = p.Dloc > 256 ? 512 : ((p.Dloc + 7) & ~7);  // rows the swizzled operand tile spans
+  const int b_bytes = ((b_rows * 128 + 1023) / 1024) * 1024;
+  const int b_load_bytes = p.Dloc > 256 ? 512 * 128 : p.Dloc * 128;  // what the TMA boxes deliver
+  const int stage_bytes = a_bytes + b_bytes;
+  WBars* bar = reinterpret_cast<WBars*>(smem + p.stages * stage_bytes);
+  float* zw = reinterpret_cast<float*>(bar + 1);  // [4 warps][D_loc] partial row sums
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int batch = blockIdx.x, mblk = blockIdx.y, k_base = mblk * p.m_tok;
+  const int b = batch / p.P, tile = batch - b * p.P;
+  const int ty = tile / p.tiles_x, tx = tile - ty * p.tiles_x;
+  const int rows_per_box = p.m_tok / p.tw;
+  const int nk = (p.d + kKC - 1) / kKC;
+  const uint32_t ncols = n_mma > 256 ? 512u : n_mma > 128 ? 256u : n_mma > 64 ? 128u : n_mma > 32 ? 64u : 32u;
+  const int box_bytes_a = p.m_tok * 128;
+  const int box_d0 = p.Dloc > 256 ? 256 : p.Dloc, box_d1 = p.Dloc - box_d0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&bar->full[s], 1);
+      mbar_init(&bar->empty[s], 1);
+    }
+    mbar_init(&bar->done, 1);
+    bar->abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bar->tmem_base;
+  volatile int* abort_flag = &bar->abort_flag;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tmap(&tm_x);
+      prefetch_tmap(&tm_d);
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % p.stages;
+        if (k >= p.stages && !mbar_wait(&bar->empty[s], ((k / p.stages) - 1) & 1, dev_status, abort_flag)) break;
+        uint8_t* sa = smem + s * stage_bytes;
+        mbar_expect_tx(&bar->full[s], box_bytes_a + b_load_bytes);
+        tma_load_4d(sa, &tm_x, &bar->full[s], k * kKC, tx * p.tw, ty * p.th + mblk * rows_per_box, b);
+        tma_load_3d(sa + a_bytes, &tm_d, &bar->full[s], k * kKC, 0, batch);
+        if (box_d1 > 0) tma_load_3d(sa + a_bytes + 256 * 128, &tm_d, &bar->full[s], k * kKC, 256, batch);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc0 = idesc_f16(kFmtBF16, kFmtBF16, false, false, 128, n0);
+      const uint32_t idesc1 = idesc_f16(kFmtBF16, kFmtBF16, false, false, 128, n1 > 0 ? n1 : 16);
+      bool ok = true;
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % p.stages;
+        if (!mbar_wait(&bar->full[s], (k / p.stages) & 1, dev_status, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t aa = smem_u32(smem + s * stage_bytes), ba = aa + a_bytes;
+#pragma unroll
+        for (int kk = 0; kk < kKC / 16; ++kk) {
+          const uint64_t ad = smem_desc_sw128(aa + kk * 32, 16, 1024);
+          mma_ss(tmem, ad, smem_desc_sw128(ba + kk * 32, 16, 1024), idesc0, k > 0 || kk > 0);
+          if (n1 > 0) mma_ss(tmem + 256, ad, smem_desc_sw128(ba + 256 * 128 + kk * 32, 16, 1024), idesc1, k > 0 || kk > 0);
+        }
+        mma_commit(&bar->empty[s]);
+      }
+      if (ok) mma_commit(&bar->done);
+    }
+  } else {
+    const int quarter = warp & 3;
+    const int k_loc = quarter * 32 + lane;              // source row inside this CTA
+    const bool valid = k_loc < p.m_tok;
+    const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16);
+    float* zrow = zw + quarter * p.Dloc;
+    if (mbar_wait(&bar->done, 0, dev_status, abort_flag)) {
+      tc_fence_after();
+      // pass 1: maximum logit over the destinations
+      float mx = -INFINITY;
+      for (int i0 = 0; i0 < p.Dloc; i0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + i0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if (i0 + e < p.Dloc) mx = fmaxf(mx, __uint_as_float(r[e]));
+      }
+      const float neg_m = -mx * p.scale_log2;
+      // pass 2: denominator
+      float sum = 0.f;
+      for (int i0 = 0; i0 < p.Dloc; i0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + i0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if (i0 + e < p.Dloc) sum += fast_exp2(fmaf(__uint_as_float(r[e]), p.scale_log2, neg_m));
+      }
+      const float inv = valid ? 1.f / sum : 0.f;
+      // pass 3: shares, their store, and the per-warp column sums
+      float* dst = shares + ((size_t)batch * p.Nloc + k_base + (valid ? k_loc : 0)) * p.Dloc;
+      for (int i0 = 0; i0 < p.Dloc; i0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + i0, r);
+        tmem_wait_ld();
+        float a[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const float v = fast_exp2(fmaf(__uint_as_float(r[e]), p.scale_log2, neg_m)) * inv;
+          a[e] = (valid && i0 + e < p.Dloc) ? v : 0.f;
+        }
+        if (valid) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 4)
+            if (i0 + e < p.Dloc) *reinterpret_cast<float4*>(dst + i0 + e) = make_float4(a[e], a[e + 1], a[e + 2], a[e + 3]);
+        }
+        // transpose-reduce: afterwards lane c holds the sum over the warp's 32 rows of column i0 + c
+#pragma unroll
+        for (int off = 16, n = 32; off >= 1; off >>= 1, n >>= 1) {
+          const bool upper = (lane & off) != 0;
+#pragma unroll
+          for (int c = 0; c < n / 2; ++c) {
+            const float send = upper ? a[c] : a[c + n / 2];
+            const float keep = upper ? a[c + n / 2] : a[c];
+            a[c] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+          }
+        }
+        if (i0 + lane < p.Dloc) zrow[i0 + lane] = a[0];
+      }
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");  // the four epilogue warps
+    const int t = threadIdx.x - 64;
+    float* zout = zpart + ((size_t)batch * gridDim.y + mblk) * p.Dloc;
+    for (int i = t; i < p.Dloc; i += 128) zout[i] = (zw[i] + zw[p.Dloc + i]) + (zw[2 * p.Dloc + i] + zw[3 * p.Dloc + i]);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, ncols);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+weights_normalise_kernel(const float* __restrict__ shares, const float* __restrict__ zpart, __nv_bfloat16* __restrict__ w,
+                         int Nloc, int Dloc, int mblocks, size_t total) {
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= total) return;
+  const size_t plane = (size_t)Nloc * Dloc;
+  const size_t batch = e / plane, r = e - batch * plane;
+  const int i = (int)(r % Dloc);
+  float z = 0.f;
+  for (int mb = 0; mb < mblocks; ++mb) z += zpart[(batch * mblocks + mb) * Dloc + i];
+  const float v = z > 0.f ? shares[e] / z : 0.f;
+  __nv_bfloat16* t = w + batch * 2 * plane;
+  const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+  t[r] = hi;
+  t[plane + r] = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
+}  // namespace
+
+bool weights_tc_supported(const Geom& g) {
+  if (g.f32) return false;
+  const int m_tok = g.Nloc < 128 ? g.Nloc : 128;
+  if (g.Nloc % m_tok != 0 || m_tok % 8 != 0) return false;
+  if (g.tw > m_tok || m_tok % g.tw != 0 || g.th % (m_tok / g.tw) != 0 || g.tw > 256 || m_tok / g.tw > 256) return false;
+  if (g.Dloc % 4 != 0 || g.Dloc > 512) return false;
+  return true;
+}
+
+size_t weights_tc_scratch_bytes(const Geom& g) {  // gathered destinations + partial row sums
+  const size_t tiles = (size_t)g.B * g.P;
+  const int m_tok = g.Nloc < 128 ? g.Nloc : 128;
+  return tiles * g.Dloc * g.d * 2 + 256 + tiles * (g.Nloc / m_tok) * g.Dloc * 4 + 256;
+}
+
+cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, void* w, float* shares, void* scratch,
+                              uint32_t* dev_status, cudaStream_t s) {
+  const size_t tiles = (size_t)g.B * g.P;
+  WParams p;
+  p.P = g.P; p.tiles_x = g.tiles_x; p.th = g.th; p.tw = g.tw; p.W = g.W; p.Nloc = g.Nloc; p.Dloc = g.Dloc; p.d = g.d;
+  p.n_all = (int)g.tokens_all();
+  p.m_tok = g.Nloc < 128 ? g.Nloc : 128;
+  p.scale_log2 = g.logit_scale * 1.4426950408889634f;
+  const int mblocks = g.Nloc / p.m_tok;
+  __nv_bfloat16* dg = (__nv_bfloat16*)scratch;
+  float* zpart = (float*)((char*)scratch + ((tiles * g.Dloc * g.d * 2 + 255) / 256) * 256);
+
+  const int rows_total = (int)(tiles * g.Dloc);
+  const long long vecs = (long long)rows_total * (g.d / 8);
+  gather_dest_kernel<<<(unsigned)((vecs + 255) / 256), 256, 0, s>>>((const __nv_bfloat16*)x, idx, dg, p, rows_total);
+  count_launch();
+
+  CUtensorMap tx, td;
+  const uint64_t xdims[4] = {(uint64_t)g.d, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.B};
+  const uint64_t xstr[3] = {(uint64_t)g.d * 2, (uint64_t)g.W * g.d * 2, (uint64_t)g.tokens_all() * g.d * 2};
+  const uint32_t xbox[4] = {64, (uint32_t)g.tw, (uint32_t)(p.m_tok / g.tw), 1};
+  const uint64_t ddims[3] = {(uint64_t)g.d, (uint64_t)g.Dloc, (uint64_t)tiles};
+  const uint64_t dstr[2] = {(uint64_t)g.d * 2, (uint64_t)g.Dloc * g.d * 2};
+  const uint32_t dbox[3] = {64, (uint32_t)(g.Dloc > 256 ? 256 : g.Dloc), 1};
+  if (!encode_tmap_16bit(&tx, x, 4, xdims, xstr, xbox) || !encode_tmap_16bit(&td, dg, 3, ddims, dstr, dbox))
+    return cudaErrorInvalidValue;
+  const int b_rows = g.Dloc > 256 ? 512 : ((g.Dloc + 7) & ~7);
+  const int stage_bytes = 128 * 128 + ((b_rows * 128 + 1023) / 1024) * 1024;
+  p.stages = stage_bytes <= 48 * 1024 ? 4 : 2;
+  const int nk = (g.d + kKC - 1) / kKC;
+  if (p.stages > nk) p.stages = nk;
+  const int smem = 1024 + p.stages * stage_bytes + (int)sizeof(WBars) + 4 * g.Dloc * 4 + 64;
+  static bool attr = false;
+  if (!attr) {
+    cudaError_t e = cudaFuncSetAttribute(weights_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    attr = true;
+  }
+  dim3 grid((unsigned)tiles, mblocks);
+  weights_logits_kernel<<<grid, 192, smem, s>>>(tx, td, shares, zpart, p, dev_status);
+  count_launch();
+  const size_t total = tiles * g.Nloc * g.Dloc;
+  weights_normalise_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(shares, zpart, (__nv_bfloat16*)w, g.Nloc,
+                                                                           g.Dloc, mblocks, total);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace toma
