@@ -149,6 +149,25 @@ def run_reference(args, cfg):
     }))
 
 
+def rank_config(cfg, rank: int):
+    """Weak scaling: every rank works on its own batch of the same shape (its own random stream)."""
+    return cfg.with_(seed=cfg.seed + rank)
+
+
+def max_over_ranks(value: float, dist, device) -> float:
+    """Slowest rank's time (the job is as slow as its slowest rank)."""
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(total_ms: float, steps: int, tokens_per_rank_step: int, world: int) -> float:
+    """Whole-job tokens/s: all ranks' tokens over the slowest rank's time."""
+    return world * tokens_per_rank_step * steps / (total_ms * 1e-3)
+
+
 def workload_config(cfg):
     return {"workload": f"{cfg.name}: SDXL-like high-resolution block, batch {cfg.batch}, {cfg.grid_h}x{cfg.grid_w} "
                         f"tokens, d={cfg.dim} {cfg.dtype}, {cfg.n_heads}x{cfg.head_dim} heads, tiles "
@@ -193,7 +212,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     peaks = load_peaks()
-    cfg_rank = cfg.with_(seed=cfg.seed + rank)          # weak scaling: every rank has its own batch
+    cfg_rank = rank_config(cfg, rank)
     desc = toma.desc_from_config(cfg_rank)
     tdt = toma.torch_dtype(desc)
     cycle = cfg.steps
@@ -244,13 +263,9 @@ def main():
     gpu_launches = toma.toma_launch_counter() - launches0 - launches_warm
     clocks = sampler.stop()
     assert int(status.item()) == 0, "a kernel reported a device-side timeout"
-    total_ms = sum(step_ms)
-    t_local = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(t_local, op=dist.ReduceOp.MAX)
-    total_ms = float(t_local.item())
+    total_ms = max_over_ranks(sum(step_ms), dist, "cuda")
     ms_per_step = total_ms / args.steps
-    value = world * B * N / (ms_per_step * 1e-3)
+    value = job_throughput(total_ms, args.steps, B * N, world)
     refresh_ms = [m for t, m in enumerate(step_ms) if (t % cycle) % cfg.reuse_interval == 0]
     reuse_ms = [m for t, m in enumerate(step_ms) if (t % cycle) % cfg.reuse_interval != 0]
 
@@ -315,10 +330,7 @@ def main():
         e2e_step(t)
     sync_all()
     e2e_s = time.perf_counter() - t0
-    t_local = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(t_local, op=dist.ReduceOp.MAX)
-    e2e_value = world * B * N * args.steps / float(t_local.item())
+    e2e_value = job_throughput(1e3 * max_over_ranks(e2e_s, dist, "cuda"), args.steps, B * N, world)
     xbytes = xs[0].numel() * xs[0].element_size()
 
     result = {

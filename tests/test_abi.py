@@ -56,7 +56,7 @@ def test_descriptor_validation(toma):
 def test_sizes(toma):
     d = _desc(toma)
     assert toma.toma_dest_per_tile(d) == 128
-    assert toma.toma_weights_bytes(d) == 2 * 16 * 256 * 128 * 2
+    assert toma.toma_weights_bytes(d) == 2 * 16 * 256 * 128 * 4  # hi + lo bf16 planes
     assert toma.toma_workspace_bytes(d) > 0
     assert toma.toma_dest_per_tile(_desc(toma, merge_ratio=0.25)) == 192
     assert toma.toma_dest_per_tile(_desc(toma, merge_ratio=0.75)) == 64
