@@ -58,8 +58,12 @@ typedef enum {
   TOMA_ERR_WORKSPACE = 6,   /* workspace missing or smaller than toma_workspace_bytes() */
   TOMA_ERR_UNSUPPORTED = 7, /* N_loc > 1024, head_dim not 64/128 in bf16 mode, dim > 4096 ... */
   TOMA_ERR_CUDA = 8,        /* a CUDA runtime call or launch failed */
-  TOMA_ERR_TIMEOUT = 9      /* only ever reported through *dev_status (bit 0) */
+  TOMA_ERR_TIMEOUT = 9,     /* only ever reported through *dev_status (bit 0) */
+  TOMA_ERR_SCRATCH_LIMIT = 10 /* toma_select_static: the problem needs more than TOMA_STATIC_SCRATCH_BYTES */
 } toma_status;
+
+/* Size of the fixed scratch array built into the library for toma_select_static (16 MiB). */
+#define TOMA_STATIC_SCRATCH_BYTES (16u << 20)
 
 typedef enum { TOMA_BF16 = 0, TOMA_F32 = 1 } toma_dtype;
 
@@ -97,6 +101,25 @@ TOMA_API uint64_t toma_launch_counter(void);
  * tokens are excluded from later rounds.  Uses `ws` as scratch. */
 TOMA_API toma_status toma_select(const toma_desc* desc, const void* x, int32_t* idx, void* ws, size_t ws_bytes,
                         uint32_t* dev_status, void* stream);
+
+/* toma_select for callers that have no workspace to give and may not allocate one.
+ * (No counterpart in the paper: this exists for integration, not for the method.)
+ * Meant for code that only receives its tensors and a stream -- a runtime's per-layer hook, a
+ * plug-in inside another program's step loop -- where cudaMalloc is off the table because it
+ * synchronises the device, is illegal during stream capture and sidesteps the host's memory pool.
+ * Same inputs, outputs and results as toma_select; the scratch is a static device array of
+ * TOMA_STATIC_SCRATCH_BYTES inside the library, so:
+ *   - it occupies that much memory on every GPU that loads the library, until process exit;
+ *   - a problem whose scratch, batch*P*N_loc*(dim + N_loc)*2 bytes plus padding, exceeds it is
+ *     refused with TOMA_ERR_SCRATCH_LIMIT before any launch;
+ *   - all calls on a device share it and it keeps the previous call's contents (nothing needs
+ *     zeroing: every byte read is written earlier in the same call); calls that can overlap on
+ *     the GPU race on it, so the caller must serialise them;
+ *   - the first call on each device resolves the array's device address; make that call before
+ *     starting any stream capture.
+ * The call never allocates or frees memory. */
+TOMA_API toma_status toma_select_static(const toma_desc* desc, const void* x, int32_t* idx, uint32_t* dev_status,
+                                        void* stream);
 
 /* Merge weights (Sec. 4.2.1).  For each tile: logits between the D_loc selected
  * tokens and all N_loc tokens, softmax over the destination axis per source

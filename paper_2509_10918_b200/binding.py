@@ -17,9 +17,9 @@ LIB_PATH = os.path.join(_HERE, "libtoma_b200.so")
 
 TOMA_BF16, TOMA_F32 = 0, 1
 STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_RATIO", "ERR_TAU", "ERR_WORKSPACE",
-                "ERR_UNSUPPORTED", "ERR_CUDA", "ERR_TIMEOUT"]
+                "ERR_UNSUPPORTED", "ERR_CUDA", "ERR_TIMEOUT", "ERR_SCRATCH_LIMIT"]
 
-EXPORTS = ["toma_launch_counter", "toma_workspace_bytes", "toma_weights_bytes", "toma_dest_per_tile", "toma_validate", "toma_status_str",
+EXPORTS = ["toma_select_static", "toma_launch_counter", "toma_workspace_bytes", "toma_weights_bytes", "toma_dest_per_tile", "toma_validate", "toma_status_str",
            "toma_select", "toma_merge_weights", "toma_merge", "toma_attention", "toma_unmerge", "toma_block",
            "toma_weights_export", "toma_weights_import"]
 
@@ -62,6 +62,8 @@ def _load() -> ctypes.CDLL:
     lib.toma_status_str.argtypes = [c_int32]
     lib.toma_select.restype = c_int32
     lib.toma_select.argtypes = [P, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
+    lib.toma_select_static.restype = c_int32
+    lib.toma_select_static.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.toma_merge_weights.restype = c_int32
     lib.toma_merge_weights.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
     lib.toma_merge.restype = c_int32
@@ -150,6 +152,13 @@ def toma_status_str(status: int) -> str:
 def toma_select(desc, x, idx, ws, dev_status=None):
     _check(lib.toma_select(ctypes.byref(desc), _ptr(x), _ptr(idx), _ptr(ws), ws.numel() * ws.element_size(),
                            _ptr(dev_status), _stream()), "toma_select")
+
+
+def toma_select_static(desc, x, idx, dev_status=None):
+    """toma_select without a workspace argument: the scratch is a fixed array inside the library
+    (see include/toma.h for who this is for and what sharing that array implies)."""
+    _check(lib.toma_select_static(ctypes.byref(desc), _ptr(x), _ptr(idx), _ptr(dev_status), _stream()),
+           "toma_select_static")
 
 
 def toma_merge_weights(desc, x, idx, w, ws, dev_status=None):

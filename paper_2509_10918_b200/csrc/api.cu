@@ -153,6 +153,7 @@ const char* toma_status_str(toma_status s) {
     case TOMA_ERR_UNSUPPORTED: return "unsupported size";
     case TOMA_ERR_CUDA: return "CUDA error";
     case TOMA_ERR_TIMEOUT: return "device-side wait timed out";
+    case TOMA_ERR_SCRATCH_LIMIT: return "problem does not fit the built-in static scratch";
   }
   return "unknown";
 }
