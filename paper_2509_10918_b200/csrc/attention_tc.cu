@@ -1,15 +1,25 @@
 // Attention core softmax(Q K^T / sqrt(dh)) V (Eq. 1 with tau = 1) on the sm_100a tensor
 // cores, bf16 in / bf16 out, fp32 softmax and accumulation.
 //
-// One CTA per (batch, head, 128 queries).  Warp 0 feeds K/V tiles of 128 keys through a TMA
-// ring, warp 1 issues tcgen05 MMAs, warps 2..5 (one thread per query row) run the online
-// softmax straight out of tensor memory:
-//   S_j = Q K_j^T          -> tensor memory, double buffered, issued one tile ahead
-//   P_j = 2^(S_j*c - m)    -> written back over S_j's columns as bf16 (A operand from tensor memory)
-//   O  += P_j V_j          -> tensor memory accumulator; rescaled only when the running maximum
-//                             grew by more than 2^8 (the final division by the row sum makes the
-//                             stale maximum exact)
-// Keys past the sequence end are zero-filled by TMA and masked to -inf.
+// One CTA per (batch, head, 128 queries), keys in tiles of 64; two CTAs are resident per SM.
+// Warp 4 feeds K and V tiles through separate TMA rings, warp 5 issues tcgen05 MMAs, warps 0..3
+// (one thread per query row) run the online softmax straight out of tensor memory:
+//   S_j = Q K_j^T          -> tensor memory, two 64-column buffers; S_{j+1} is issued before the
+//                             softmax of tile j has finished, so the softmax warps never wait for a
+//                             round trip through the MMA warp
+//   P_j = 2^(S_j*c - m)    -> written back over S_j's first 32 columns as bf16 and used as the
+//                             A operand (from tensor memory) of  O += P_j V_j
+//   row sums (head_dim 64) -> a second tiny MMA, P_j x ones[64 x 16], accumulates sum_k P_jk in
+//                             tensor memory: exactly the bf16 P that multiplies V, so P can be
+//                             produced by truncation (one byte-permute per pair, no conversion on
+//                             the XU pipe) without biasing the normalised result
+//   running maximum        -> O (and the row sums) are rescaled only when the maximum grew by more
+//                             than 2^8; the final division by the row sum makes a stale maximum exact
+//   exponentials           -> a quarter of them are a degree-3 polynomial on the FMA pipe (relative
+//                             error 7.5e-5, far below bf16 resolution of P), the rest MUFU ex2
+// The whole S row of a tile (64 fp32) is fetched with one tensor-memory round trip and kept in
+// registers for both the maximum and the exponentials.
+// Keys past the sequence end are zero-filled by TMA and masked out.
 #include "common.cuh"
 #include "tc.cuh"
 
@@ -20,41 +30,164 @@ using namespace tc;
 namespace {
 
 constexpr int kBM = 128;  // queries per CTA
-constexpr int kBN = 128;  // keys per tile
+constexpr int kBN = 64;   // keys per tile
 constexpr float kRescaleThreshold = 8.0f;
 
 template <int DH>
 struct AttCfg {
-  static constexpr int kStages = DH == 64 ? 3 : 2;
-  static constexpr int kChunks = DH / 64;                 // 64-column (128-byte) slabs per row
-  static constexpr int kSlabBytes = 128 * 128;            // 128 rows x 128 B
-  static constexpr int kTileBytes = kChunks * kSlabBytes; // one Q, K or V tile
-  static constexpr int kSmemBytes = 1024 + kTileBytes * (1 + 2 * kStages) + 256;
-  static constexpr int kTmemCols = 512;
-  static constexpr int kColS0 = 0, kColS1 = 128, kColO = 256;
+  static constexpr int kStages = DH == 64 ? 4 : 2;         // K ring depth = V ring depth
+  static constexpr int kChunks = DH / 64;                  // 64-column (128-byte) slabs per row
+  static constexpr int kQSlab = kBM * 128;                 // 128 query rows x 128 B
+  static constexpr int kKvSlab = kBN * 128;                // 64 key rows x 128 B
+  static constexpr int kQBytes = kChunks * kQSlab;
+  static constexpr int kKvBytes = kChunks * kKvSlab;       // one K or V tile
+  static constexpr int kOnesBytes = 2048;                  // [16][64] bf16 ones, K-major
+  static constexpr int kSmemBytes = 1024 + kQBytes + 2 * kStages * kKvBytes + kOnesBytes + 256;
+  static constexpr bool kSumMma = DH == 64;                // row sums on the tensor pipe, truncated P
+  static constexpr int kTmemCols = 256;
+  static constexpr int kColS = 0, kColO = 128, kColL = 128 + DH;  // S buffers at 0 and 64
 };
 
 struct Barriers {
   uint64_t q_full;
-  uint64_t k_full[3], v_full[3], kv_empty[3];
-  uint64_t s_full[2], p_full[2];
-  uint64_t o_done;
+  uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
+  uint64_t s_full[2], p_full[2], pv_done, o_done;
   uint32_t tmem_base;
   int abort_flag;
 };
 
-__device__ __forceinline__ float fast_exp2(float x) {
+__device__ __forceinline__ float ex2_mufu(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+// 2^x for x <= ~9 on the FMA pipe: round to nearest integer with the 1.5*2^23 trick, degree-3
+// near-minimax polynomial for 2^f on [-0.5, 0.5], exponent patched in with an integer add.
+__device__ __forceinline__ float ex2_poly(float x) {
+  x = fmaxf(x, -126.f);
+  const float t = x + 12582912.f;
+  const float f = x - (t - 12582912.f);
+  float p = fmaf(0.0551716648f, f, 0.2426111251f);
+  p = fmaf(p, f, 0.6932609677f);
+  p = fmaf(p, f, 0.9999280572f);
+  return __int_as_float(__float_as_int(p) + (int)((unsigned)__float_as_int(t) << 23));
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_bf16_rn(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
+__device__ __forceinline__ uint32_t pack_bf16_trunc(float lo, float hi) {  // upper halves of both words
+  return __byte_perm(__float_as_uint(lo), __float_as_uint(hi), 0x7632);
+}
+
+// View of 32 consecutive registers of a larger per-thread array (all indices are compile-time).
+template <int kOff, int kN>
+__device__ __forceinline__ uint32_t (&sub32(uint32_t (&r)[kN]))[32] {
+  return *reinterpret_cast<uint32_t(*)[32]>(&r[kOff]);
+}
+
+// Maximum of 32 tensor-memory words (columns first .. first+31 of this row; columns >= valid ignored).
+template <bool kMask>
+__device__ __forceinline__ float chunk_max(const uint32_t (&r)[32], float mx, int first, int valid) {
+  if (kMask) {
+#pragma unroll
+    for (int e = 0; e < 32; ++e) mx = fmaxf(mx, (first + e < valid) ? __uint_as_float(r[e]) : -INFINITY);
+  } else {
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) mx = max3(mx, __uint_as_float(r[e]), __uint_as_float(r[e + 1]));
+  }
+  return mx;
+}
+
+// P for 32 columns as packed bf16 pairs in pk[16]; returns their fp32 sum when sums stay in registers.
+template <bool kMask, bool kRegSum>
+__device__ __forceinline__ float chunk_exp(const uint32_t (&r)[32], uint32_t (&pk)[16], float scale, float neg_m,
+                                           int first, int valid) {
+  float l = 0.f;
+#pragma unroll
+  for (int e = 0; e < 32; e += 2) {
+    const float x0 = fmaf(__uint_as_float(r[e]), scale, neg_m);
+    const float x1 = fmaf(__uint_as_float(r[e + 1]), scale, neg_m);
+    float p0 = ex2_mufu(x0);
+    float p1 = (e & 2) ? ex2_poly(x1) : ex2_mufu(x1);  // every fourth exponential on the FMA pipe
+    if (kMask) {
+      if (first + e >= valid) p0 = 0.f;
+      if (first + e + 1 >= valid) p1 = 0.f;
+    }
+    if (kRegSum) {
+      l += p0 + p1;
+      pk[e >> 1] = pack_bf16_rn(p0, p1);
+    } else {
+      pk[e >> 1] = pack_bf16_trunc(p0, p1);
+    }
+  }
+  return l;
+}
+
+// One 64-key tile of the online softmax for one query row.
+template <int DH, bool kMask>
+__device__ __forceinline__ bool softmax_tile(uint32_t sb, uint32_t ob, float scale_log2, int valid, int j, float& m_used,
+                                             float& l, uint64_t* pv_done, uint32_t* dev_status, volatile int* abort_flag) {
+  using C = AttCfg<DH>;
+  uint32_t sr[64];
+  tmem_ld32(sb, sub32<0>(sr));
+  tmem_ld32(sb + 32, sub32<32>(sr));
+  tmem_wait_ld();
+  float mx = -INFINITY;
+  mx = chunk_max<kMask>(sub32<0>(sr), mx, 0, valid);
+  mx = chunk_max<kMask>(sub32<32>(sr), mx, 32, valid);
+  mx *= scale_log2;
+  float factor = 1.f;
+  bool rescale = false;
+  if (j == 0) {
+    m_used = mx;
+  } else if (mx > m_used + kRescaleThreshold) {
+    factor = ex2_mufu(m_used - mx);
+    m_used = mx;
+    rescale = true;
+  }
+  if (__any_sync(0xffffffffu, rescale)) {
+    // O holds every PV product issued so far; the last one (tile j-1) must have landed
+    if (!mbar_wait(pv_done, (j - 1) & 1, dev_status, abort_flag)) return false;
+    tc_fence_after();
+    l *= factor;
+#pragma unroll
+    for (int c = 0; c < DH / 32; ++c) {
+      uint32_t t[32];
+      tmem_ld32(ob + c * 32, t);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 32; ++e) t[e] = __float_as_uint(__uint_as_float(t[e]) * factor);
+      tmem_st32(ob + c * 32, t);
+    }
+    if (C::kSumMma) {
+      uint32_t rs[16];
+      tmem_ld16(ob + DH, rs);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 16; ++e) rs[e] = __float_as_uint(__uint_as_float(rs[e]) * factor);
+      tmem_st16(ob + DH, rs);
+    }
+  }
+  // P = 2^(S*c - m) as packed bf16 over the first 32 columns of this S buffer
+  const float neg_m = -m_used;
+  constexpr bool kRegSum = !C::kSumMma;
+  uint32_t pk[16];
+  l += chunk_exp<kMask, kRegSum>(sub32<0>(sr), pk, scale_log2, neg_m, 0, valid);
+  tmem_st16(sb, pk);
+  l += chunk_exp<kMask, kRegSum>(sub32<32>(sr), pk, scale_log2, neg_m, 32, valid);
+  tmem_st16(sb + 16, pk);
+  tmem_wait_st();
+  return true;
+}
 
 template <int DH>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(192, 2)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, int L, int heads,
                     float scale_log2, uint32_t* dev_status) {
@@ -62,9 +195,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = smem;
-  uint8_t* sK = sQ + C::kTileBytes;
-  uint8_t* sV = sK + C::kStages * C::kTileBytes;
-  Barriers* bar = reinterpret_cast<Barriers*>(sV + C::kStages * C::kTileBytes);
+  uint8_t* sK = sQ + C::kQBytes;
+  uint8_t* sV = sK + C::kStages * C::kKvBytes;
+  uint8_t* sOnes = sV + C::kStages * C::kKvBytes;
+  Barriers* bar = reinterpret_cast<Barriers*>(sOnes + C::kOnesBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q0 = blockIdx.x * kBM, h = blockIdx.y, b = blockIdx.z;
@@ -74,58 +208,76 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     mbar_init(&bar->q_full, 1);
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&bar->k_full[s], 1);
+      mbar_init(&bar->k_empty[s], 1);
       mbar_init(&bar->v_full[s], 1);
-      mbar_init(&bar->kv_empty[s], 1);
+      mbar_init(&bar->v_empty[s], 1);
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bar->s_full[s], 1);
       mbar_init(&bar->p_full[s], 128);
     }
+    mbar_init(&bar->pv_done, 1);
     mbar_init(&bar->o_done, 1);
     bar->abort_flag = 0;
     mbar_fence_init();
   }
-  if (warp == 1) tmem_alloc(&bar->tmem_base, C::kTmemCols);
+  if (C::kSumMma) {  // bf16 1.0 everywhere: the layout's swizzle is irrelevant for a constant tile
+    for (int e = threadIdx.x; e < C::kOnesBytes / 4; e += blockDim.x) reinterpret_cast<uint32_t*>(sOnes)[e] = 0x3F803F80u;
+    fence_proxy_async();
+  }
+  if (warp == 5) tmem_alloc(&bar->tmem_base, C::kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bar->tmem_base;
   volatile int* abort_flag = &bar->abort_flag;
 
-  if (warp == 0) {
+  if (warp == 4) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       prefetch_tmap(&tm_q);
       prefetch_tmap(&tm_k);
       prefetch_tmap(&tm_v);
-      mbar_expect_tx(&bar->q_full, C::kTileBytes);
-      for (int c = 0; c < C::kChunks; ++c) tma_load_3d(sQ + c * C::kSlabBytes, &tm_q, &bar->q_full, h * DH + c * 64, q0, b);
+      mbar_expect_tx(&bar->q_full, C::kQBytes);
+      for (int c = 0; c < C::kChunks; ++c) tma_load_3d(sQ + c * C::kQSlab, &tm_q, &bar->q_full, h * DH + c * 64, q0, b);
       for (int j = 0; j < nblk; ++j) {
         const int s = j % C::kStages;
-        if (j >= C::kStages && !mbar_wait(&bar->kv_empty[s], ((j / C::kStages) - 1) & 1, dev_status, abort_flag)) break;
-        mbar_expect_tx(&bar->k_full[s], C::kTileBytes);
+        const uint32_t par = ((j / C::kStages) - 1) & 1;
+        if (j >= C::kStages && !mbar_wait(&bar->k_empty[s], par, dev_status, abort_flag)) break;
+        mbar_expect_tx(&bar->k_full[s], C::kKvBytes);
         for (int c = 0; c < C::kChunks; ++c)
-          tma_load_3d(sK + s * C::kTileBytes + c * C::kSlabBytes, &tm_k, &bar->k_full[s], h * DH + c * 64, j * kBN, b);
-        mbar_expect_tx(&bar->v_full[s], C::kTileBytes);
+          tma_load_3d(sK + s * C::kKvBytes + c * C::kKvSlab, &tm_k, &bar->k_full[s], h * DH + c * 64, j * kBN, b);
+        if (j >= C::kStages && !mbar_wait(&bar->v_empty[s], par, dev_status, abort_flag)) break;
+        mbar_expect_tx(&bar->v_full[s], C::kKvBytes);
         for (int c = 0; c < C::kChunks; ++c)
-          tma_load_3d(sV + s * C::kTileBytes + c * C::kSlabBytes, &tm_v, &bar->v_full[s], h * DH + c * 64, j * kBN, b);
+          tma_load_3d(sV + s * C::kKvBytes + c * C::kKvSlab, &tm_v, &bar->v_full[s], h * DH + c * 64, j * kBN, b);
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 5) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc_s = idesc_f16(kFmtBF16, kFmtBF16, false, false, kBM, kBN);
       constexpr uint32_t idesc_o = idesc_f16(kFmtBF16, kFmtBF16, false, true, kBM, DH);
-      auto issue_s = [&](int j) {  // S_j = Q K_j^T
+      constexpr uint32_t idesc_l = idesc_f16(kFmtBF16, kFmtBF16, false, false, kBM, 16);
+      // Descriptors are built once and advanced by adding a constant to the 14-bit start-address
+      // field (no carry: all tiles live below 256 KB).
+      const uint64_t q_desc = smem_desc_sw128(smem_u32(sQ), 16, 1024);
+      const uint64_t k_desc0 = smem_desc_sw128(smem_u32(sK), 16, 1024);
+      const uint64_t v_desc0 = smem_desc_sw128(smem_u32(sV), C::kKvSlab, 1024);
+      const uint64_t ones_desc = smem_desc_sw128(smem_u32(sOnes), 16, 1024);
+      const uint32_t t_o = tmem + C::kColO, t_l = tmem + C::kColL;
+      auto issue_s = [&](int j) {  // S_j = Q K_j^T into buffer j&1, then the K slot is free again
         const int s = j % C::kStages;
-        const uint32_t d = tmem + ((j & 1) ? C::kColS1 : C::kColS0);
-        const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + s * C::kTileBytes);
+        const uint64_t kb = k_desc0 + (uint64_t)((s * C::kKvBytes) >> 4);
+        const uint32_t t_s = tmem + C::kColS + (j & 1) * kBN;
 #pragma unroll
         for (int kk = 0; kk < DH / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * C::kSlabBytes + (kk & 3) * 32;
-          mma_ss(d, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024), idesc_s, kk > 0);
+          const uint64_t qoff = (uint64_t)(((kk >> 2) * C::kQSlab + (kk & 3) * 32) >> 4);
+          const uint64_t koff = (uint64_t)(((kk >> 2) * C::kKvSlab + (kk & 3) * 32) >> 4);
+          mma_ss(t_s, q_desc + qoff, kb + koff, idesc_s, kk > 0);
         }
         mma_commit(&bar->s_full[j & 1]);
+        mma_commit(&bar->k_empty[s]);
       };
       bool ok = mbar_wait(&bar->q_full, 0, dev_status, abort_flag) && mbar_wait(&bar->k_full[0], 0, dev_status, abort_flag);
       if (ok) {
@@ -134,116 +286,73 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
       for (int j = 0; ok && j < nblk; ++j) {
         const int s = j % C::kStages;
-        if (j + 1 < nblk) {
+        if (j + 1 < nblk) {  // next S first: it only needs K_{j+1} and the buffer PV_{j-1} has released
           const int s1 = (j + 1) % C::kStages;
           if (!mbar_wait(&bar->k_full[s1], ((j + 1) / C::kStages) & 1, dev_status, abort_flag)) break;
+          // S_{j+1} overwrites the buffer whose P_{j-1} the PV (and row-sum) MMAs of tile j-1 read as
+          // their A operand.  MMAs into different accumulators are not ordered among themselves, so
+          // that read has to be complete before the overwrite is issued.
+          if (j >= 1 && !mbar_wait(&bar->pv_done, (j - 1) & 1, dev_status, abort_flag)) break;
           tc_fence_after();
           issue_s(j + 1);
         }
         if (!mbar_wait(&bar->p_full[j & 1], (j >> 1) & 1, dev_status, abort_flag)) break;
         if (!mbar_wait(&bar->v_full[s], (j / C::kStages) & 1, dev_status, abort_flag)) break;
         tc_fence_after();
-        const uint32_t pa = tmem + ((j & 1) ? C::kColS1 : C::kColS0);
-        const uint32_t va = smem_u32(sV + s * C::kTileBytes);
+        const uint64_t vb = v_desc0 + (uint64_t)((s * C::kKvBytes) >> 4);
+        const uint32_t t_p = tmem + C::kColS + (j & 1) * kBN;
 #pragma unroll
-        for (int kk = 0; kk < kBN / 16; ++kk)  // 16 keys per MMA: 8 packed columns of P, 16 rows of V
-          mma_ts(tmem + C::kColO, pa + kk * 8, smem_desc_sw128(va + kk * 2048, C::kSlabBytes, 1024), idesc_o,
-                 j > 0 || kk > 0);
-        mma_commit(&bar->kv_empty[s]);
-        mma_commit(&bar->o_done);
+        for (int kk = 0; kk < kBN / 16; ++kk) {  // 16 keys per MMA: 8 packed columns of P, 16 rows of V
+          mma_ts(t_o, t_p + kk * 8, vb + (uint64_t)((kk * 2048) >> 4), idesc_o, j > 0 || kk > 0);
+          if (C::kSumMma) mma_ts(t_l, t_p + kk * 8, ones_desc + (uint64_t)((kk * 32) >> 4), idesc_l, j > 0 || kk > 0);
+        }
+        mma_commit(&bar->v_empty[s]);
+        mma_commit(&bar->pv_done);
+        if (j + 1 == nblk) mma_commit(&bar->o_done);  // single-phase barrier: the epilogue cannot mistake an older phase for it
       }
     }
-  } else {
+  } else if (warp < 4) {
     // ------------------------------------------------------------------ softmax / correction / epilogue
-    const int quarter = warp & 3;              // tensor-memory lane quarter this warp may access
-    const int row = quarter * 32 + lane;       // query row inside the tile
-    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const int row = warp * 32 + lane;  // query row inside the tile = tensor-memory lane
+    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+    const uint32_t ob = tmem + lane_addr + C::kColO;
     float m_used = -INFINITY, l = 0.f;
     bool ok = true;
     for (int j = 0; j < nblk; ++j) {
-      const uint32_t sb = tmem + lane_addr + ((j & 1) ? C::kColS1 : C::kColS0);
+      const uint32_t sb = tmem + lane_addr + C::kColS + (j & 1) * kBN;
       if (!mbar_wait(&bar->s_full[j & 1], (j >> 1) & 1, dev_status, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const int valid = min(kBN, L - j * kBN);  // keys of this tile inside the sequence
-      // pass 1: row maximum
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld32(sb + c * 32, r);
-        tmem_wait_ld();
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const float v = __uint_as_float(r[e]);
-          mx = fmaxf(mx, (c * 32 + e < valid) ? v : -INFINITY);
-        }
-      }
-      mx *= scale_log2;
-      float factor = 1.f;
-      bool rescale = false;
-      if (j == 0) {
-        m_used = mx;
-      } else if (mx > m_used + kRescaleThreshold) {
-        factor = fast_exp2(m_used - mx);
-        m_used = mx;
-        rescale = true;
-      }
-      if (__any_sync(0xffffffffu, rescale)) {
-        // O holds every PV product issued so far; wait for the last one before touching it
-        if (!mbar_wait(&bar->o_done, (j - 1) & 1, dev_status, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        l *= factor;
-#pragma unroll
-        for (int c = 0; c < DH / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(tmem + lane_addr + C::kColO + c * 32, r);
-          tmem_wait_ld();
-#pragma unroll
-          for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * factor);
-          tmem_st32(tmem + lane_addr + C::kColO + c * 32, r);
-        }
-      }
-      // pass 2: P = 2^(S*c - m), packed bf16 written over the first 64 columns of S_j
-      const float neg_m = -m_used;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld32(sb + c * 32, r);
-        tmem_wait_ld();
-        uint32_t pk[16];
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(r[e]), scale_log2, neg_m));
-          float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 1]), scale_log2, neg_m));
-          if (c * 32 + e >= valid) p0 = 0.f;
-          if (c * 32 + e + 1 >= valid) p1 = 0.f;
-          l += p0 + p1;
-          pk[e >> 1] = pack_bf16(p0, p1);
-        }
-        tmem_st16(sb + c * 16, pk);
-      }
-      tmem_wait_st();
+      const int valid = L - j * kBN;  // keys of this tile inside the sequence (>= 64: all)
+      if (valid >= kBN) ok = softmax_tile<DH, false>(sb, ob, scale_log2, kBN, j, m_used, l, &bar->pv_done, dev_status, abort_flag);
+      else ok = softmax_tile<DH, true>(sb, ob, scale_log2, valid, j, m_used, l, &bar->pv_done, dev_status, abort_flag);
+      if (!ok) break;
       tc_fence_before();
       mbar_arrive(&bar->p_full[j & 1]);
     }
-    if (ok && mbar_wait(&bar->o_done, (nblk - 1) & 1, dev_status, abort_flag)) {
+    if (ok && mbar_wait(&bar->o_done, 0, dev_status, abort_flag)) {
       tc_fence_after();
+      if (C::kSumMma) {
+        uint32_t rs[16];
+        tmem_ld16(ob + DH, rs);
+        tmem_wait_ld();
+        l = __uint_as_float(rs[0]);
+      }
       const float inv = 1.f / l;
       const int qi = q0 + row;
       __nv_bfloat16* dst = o + ((size_t)b * L + (qi < L ? qi : 0)) * ((size_t)heads * DH) + (size_t)h * DH;
 #pragma unroll
       for (int c = 0; c < DH / 32; ++c) {
         uint32_t r[32];
-        tmem_ld32(tmem + lane_addr + C::kColO + c * 32, r);
+        tmem_ld32(ob + c * 32, r);
         tmem_wait_ld();
         if (qi < L) {
 #pragma unroll
           for (int e = 0; e < 32; e += 8) {
             uint4 v;
-            v.x = pack_bf16(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
-            v.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-            v.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-            v.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+            v.x = pack_bf16_rn(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
+            v.y = pack_bf16_rn(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+            v.z = pack_bf16_rn(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+            v.w = pack_bf16_rn(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
             *reinterpret_cast<uint4*>(dst + c * 32 + e) = v;
           }
         }
@@ -252,7 +361,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == 5) {
     tc_fence_after();
     tmem_dealloc(tmem, C::kTmemCols);
   }
@@ -265,9 +374,10 @@ cudaError_t launch(int B, int L, int heads, const void* q, const void* k, const 
   CUtensorMap tq, tk, tv;
   const uint64_t dims[3] = {(uint64_t)heads * DH, (uint64_t)L, (uint64_t)B};
   const uint64_t strides[2] = {(uint64_t)heads * DH * 2, (uint64_t)L * heads * DH * 2};
-  const uint32_t box[3] = {64, 128, 1};
-  if (!encode_tmap_16bit(&tq, q, 3, dims, strides, box) || !encode_tmap_16bit(&tk, k, 3, dims, strides, box) ||
-      !encode_tmap_16bit(&tv, v, 3, dims, strides, box))
+  const uint32_t box_q[3] = {64, kBM, 1};
+  const uint32_t box_kv[3] = {64, kBN, 1};
+  if (!encode_tmap_16bit(&tq, q, 3, dims, strides, box_q) || !encode_tmap_16bit(&tk, k, 3, dims, strides, box_kv) ||
+      !encode_tmap_16bit(&tv, v, 3, dims, strides, box_kv))
     return cudaErrorInvalidValue;
   static bool attr_set = false;
   if (!attr_set) {
