@@ -132,7 +132,7 @@ __device__ __forceinline__ float chunk_exp(const uint32_t (&r)[32], uint32_t (&p
 // One 64-key tile of the online softmax for one query row.
 template <int DH, bool kMask>
 __device__ __forceinline__ bool softmax_tile(uint32_t sb, uint32_t ob, float scale_log2, int valid, int j, float& m_used,
-                                             float& l, uint64_t* pv_done, uint32_t* dev_status, volatile int* abort_flag) {
+                                             float& l, uint64_t* pv_done, uint32_t pv_parity, uint32_t* dev_status, volatile int* abort_flag) {
   using C = AttCfg<DH>;
   uint32_t sr[64];
   tmem_ld32(sb, sub32<0>(sr));
@@ -153,7 +153,7 @@ __device__ __forceinline__ bool softmax_tile(uint32_t sb, uint32_t ob, float sca
   }
   if (__any_sync(0xffffffffu, rescale)) {
     // O holds every PV product issued so far; the last one (tile j-1) must have landed
-    if (!mbar_wait(pv_done, (j - 1) & 1, dev_status, abort_flag)) return false;
+    if (!mbar_wait(pv_done, pv_parity, dev_status, abort_flag)) return false;
     tc_fence_after();
     l *= factor;
 #pragma unroll
@@ -187,7 +187,7 @@ __device__ __forceinline__ bool softmax_tile(uint32_t sb, uint32_t ob, float sca
 }
 
 template <int DH>
-__global__ void __launch_bounds__(192, 2)
+__global__ void __launch_bounds__(224, 2)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, int L, int heads,
                     float scale_log2, uint32_t* dev_status) {
@@ -214,7 +214,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bar->s_full[s], 1);
-      mbar_init(&bar->p_full[s], 128);
+      mbar_init(&bar->p_full[s], 4);  // one arrival per softmax warp
     }
     mbar_init(&bar->pv_done, 1);
     mbar_init(&bar->o_done, 1);
@@ -243,31 +243,33 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (int j = 0; j < nblk; ++j) {
         const int s = j % C::kStages;
         const uint32_t par = ((j / C::kStages) - 1) & 1;
-        if (j >= C::kStages && !mbar_wait(&bar->k_empty[s], par, dev_status, abort_flag)) break;
-        mbar_expect_tx(&bar->k_full[s], C::kKvBytes);
+        if (j >= C::kStages && !mbar_wait(&bar->v_empty[s], par, dev_status, abort_flag)) break;
+        mbar_expect_tx(&bar->k_full[s], 2 * C::kKvBytes);  // K and V of tile j arrive under one barrier
         for (int c = 0; c < C::kChunks; ++c)
           tma_load_3d(sK + s * C::kKvBytes + c * C::kKvSlab, &tm_k, &bar->k_full[s], h * DH + c * 64, j * kBN, b);
-        if (j >= C::kStages && !mbar_wait(&bar->v_empty[s], par, dev_status, abort_flag)) break;
-        mbar_expect_tx(&bar->v_full[s], C::kKvBytes);
         for (int c = 0; c < C::kChunks; ++c)
-          tma_load_3d(sV + s * C::kKvBytes + c * C::kKvSlab, &tm_v, &bar->v_full[s], h * DH + c * 64, j * kBN, b);
+          tma_load_3d(sV + s * C::kKvBytes + c * C::kKvSlab, &tm_v, &bar->k_full[s], h * DH + c * 64, j * kBN, b);
       }
     }
   } else if (warp == 5) {
-    // ------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------ MMA issuer for S = Q K^T
+    // The two issuers are separate warps so that their waits and commits (each a serial, ~100-cycle
+    // operation for a single thread) proceed in parallel.
     if (lane == 0) {
       constexpr uint32_t idesc_s = idesc_f16(kFmtBF16, kFmtBF16, false, false, kBM, kBN);
-      constexpr uint32_t idesc_o = idesc_f16(kFmtBF16, kFmtBF16, false, true, kBM, DH);
-      constexpr uint32_t idesc_l = idesc_f16(kFmtBF16, kFmtBF16, false, false, kBM, 16);
       // Descriptors are built once and advanced by adding a constant to the 14-bit start-address
       // field (no carry: all tiles live below 256 KB).
       const uint64_t q_desc = smem_desc_sw128(smem_u32(sQ), 16, 1024);
       const uint64_t k_desc0 = smem_desc_sw128(smem_u32(sK), 16, 1024);
-      const uint64_t v_desc0 = smem_desc_sw128(smem_u32(sV), C::kKvSlab, 1024);
-      const uint64_t ones_desc = smem_desc_sw128(smem_u32(sOnes), 16, 1024);
-      const uint32_t t_o = tmem + C::kColO, t_l = tmem + C::kColL;
-      auto issue_s = [&](int j) {  // S_j = Q K_j^T into buffer j&1, then the K slot is free again
+      bool ok = mbar_wait(&bar->q_full, 0, dev_status, abort_flag);
+      for (int j = 0; ok && j < nblk; ++j) {
         const int s = j % C::kStages;
+        if (!mbar_wait(&bar->k_full[s], (j / C::kStages) & 1, dev_status, abort_flag)) break;
+        // S_j overwrites the buffer whose P_{j-2} the PV (and row-sum) MMAs of tile j-2 read as their
+        // A operand.  MMAs into different accumulators are not ordered among themselves, so that read
+        // has to be complete before the overwrite is issued.
+        if (j >= 2 && !mbar_wait(&bar->v_empty[(j - 2) % C::kStages], ((j - 2) / C::kStages) & 1, dev_status, abort_flag)) break;
+        tc_fence_after();
         const uint64_t kb = k_desc0 + (uint64_t)((s * C::kKvBytes) >> 4);
         const uint32_t t_s = tmem + C::kColS + (j & 1) * kBN;
 #pragma unroll
@@ -277,27 +279,19 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           mma_ss(t_s, q_desc + qoff, kb + koff, idesc_s, kk > 0);
         }
         mma_commit(&bar->s_full[j & 1]);
-        mma_commit(&bar->k_empty[s]);
-      };
-      bool ok = mbar_wait(&bar->q_full, 0, dev_status, abort_flag) && mbar_wait(&bar->k_full[0], 0, dev_status, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        issue_s(0);
       }
-      for (int j = 0; ok && j < nblk; ++j) {
+    }
+  } else if (warp == 6) {
+    // ------------------------------------------------------------------ MMA issuer for O += P V
+    if (lane == 0) {
+      constexpr uint32_t idesc_o = idesc_f16(kFmtBF16, kFmtBF16, false, true, kBM, DH);
+      constexpr uint32_t idesc_l = idesc_f16(kFmtBF16, kFmtBF16, false, false, kBM, 16);
+      const uint64_t v_desc0 = smem_desc_sw128(smem_u32(sV), C::kKvSlab, 1024);
+      const uint64_t ones_desc = smem_desc_sw128(smem_u32(sOnes), 16, 1024);
+      const uint32_t t_o = tmem + C::kColO, t_l = tmem + C::kColL;
+      for (int j = 0; j < nblk; ++j) {
         const int s = j % C::kStages;
-        if (j + 1 < nblk) {  // next S first: it only needs K_{j+1} and the buffer PV_{j-1} has released
-          const int s1 = (j + 1) % C::kStages;
-          if (!mbar_wait(&bar->k_full[s1], ((j + 1) / C::kStages) & 1, dev_status, abort_flag)) break;
-          // S_{j+1} overwrites the buffer whose P_{j-1} the PV (and row-sum) MMAs of tile j-1 read as
-          // their A operand.  MMAs into different accumulators are not ordered among themselves, so
-          // that read has to be complete before the overwrite is issued.
-          if (j >= 1 && !mbar_wait(&bar->pv_done, (j - 1) & 1, dev_status, abort_flag)) break;
-          tc_fence_after();
-          issue_s(j + 1);
-        }
-        if (!mbar_wait(&bar->p_full[j & 1], (j >> 1) & 1, dev_status, abort_flag)) break;
-        if (!mbar_wait(&bar->v_full[s], (j / C::kStages) & 1, dev_status, abort_flag)) break;
+        if (!mbar_wait(&bar->p_full[j & 1], (j >> 1) & 1, dev_status, abort_flag)) break;  // implies K/V tile j has landed
         tc_fence_after();
         const uint64_t vb = v_desc0 + (uint64_t)((s * C::kKvBytes) >> 4);
         const uint32_t t_p = tmem + C::kColS + (j & 1) * kBN;
@@ -306,8 +300,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           mma_ts(t_o, t_p + kk * 8, vb + (uint64_t)((kk * 2048) >> 4), idesc_o, j > 0 || kk > 0);
           if (C::kSumMma) mma_ts(t_l, t_p + kk * 8, ones_desc + (uint64_t)((kk * 32) >> 4), idesc_l, j > 0 || kk > 0);
         }
-        mma_commit(&bar->v_empty[s]);
-        mma_commit(&bar->pv_done);
+        mma_commit(&bar->v_empty[s]);  // frees the K/V slot and tells everyone that PV_j has landed
         if (j + 1 == nblk) mma_commit(&bar->o_done);  // single-phase barrier: the epilogue cannot mistake an older phase for it
       }
     }
@@ -323,11 +316,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (!mbar_wait(&bar->s_full[j & 1], (j >> 1) & 1, dev_status, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int valid = L - j * kBN;  // keys of this tile inside the sequence (>= 64: all)
-      if (valid >= kBN) ok = softmax_tile<DH, false>(sb, ob, scale_log2, kBN, j, m_used, l, &bar->pv_done, dev_status, abort_flag);
-      else ok = softmax_tile<DH, true>(sb, ob, scale_log2, valid, j, m_used, l, &bar->pv_done, dev_status, abort_flag);
+      uint64_t* pvb = &bar->v_empty[(j + C::kStages - 1) % C::kStages];  // barrier PV_{j-1} commits to
+      const uint32_t pvp = (uint32_t)(((j - 1) / C::kStages) & 1);
+      if (valid >= kBN) ok = softmax_tile<DH, false>(sb, ob, scale_log2, kBN, j, m_used, l, pvb, pvp, dev_status, abort_flag);
+      else ok = softmax_tile<DH, true>(sb, ob, scale_log2, valid, j, m_used, l, pvb, pvp, dev_status, abort_flag);
       if (!ok) break;
       tc_fence_before();
-      mbar_arrive(&bar->p_full[j & 1]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar->p_full[j & 1]);
     }
     if (ok && mbar_wait(&bar->o_done, 0, dev_status, abort_flag)) {
       tc_fence_after();
@@ -387,7 +383,7 @@ cudaError_t launch(int B, int L, int heads, const void* q, const void* k, const 
   }
   dim3 grid((L + kBM - 1) / kBM, heads, B);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  attention_tc_kernel<DH><<<grid, 192, C::kSmemBytes, s>>>(tq, tk, tv, (__nv_bfloat16*)o, L, heads, scale_log2, dev_status);
+  attention_tc_kernel<DH><<<grid, 224, C::kSmemBytes, s>>>(tq, tk, tv, (__nv_bfloat16*)o, L, heads, scale_log2, dev_status);
   count_launch();
   return cudaGetLastError();
 }
