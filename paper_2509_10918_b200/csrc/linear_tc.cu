@@ -22,7 +22,8 @@ namespace {
 
 constexpr int kKC = 64;           // contraction elements per pipeline stage
 constexpr int kSlab = kKC * 128;  // bytes of a 64-row x 128-byte slab
-constexpr int kMaxCols = 256;     // output columns (MMA N) per CTA
+constexpr int kMaxCols = 256;     // output columns (MMA N) per merge CTA
+constexpr int kUnmergeTok = 128;  // tokens per unmerge CTA: small enough that two CTAs share an SM
 
 struct PipeBars {
   uint64_t full[4], empty[4], done;
@@ -210,10 +211,13 @@ unmerge_tc_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constan
         tmem_ld32(taddr + l0, r);
         tmem_wait_ld();
         if (ch < p.d) {
+          // token of local slot l0 (one division per 32 slots), then walk the tile row by row
+          int lx = (t0 + l0) % p.tw;
+          size_t tok = (size_t)tile_token(tile, t0 + l0, p.tiles_x, p.th, p.tw, p.W);
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
-            const int tok = tile_token(tile, t0 + l0 + e, p.tiles_x, p.th, p.tw, p.W);
-            base[(size_t)tok * p.d] = __float2bfloat16_rn(__uint_as_float(r[e]));
+            base[tok * p.d] = __float2bfloat16_rn(__uint_as_float(r[e]));
+            if (++lx == p.tw) { lx = 0; tok += (size_t)(p.W - p.tw + 1); } else { ++tok; }
           }
         }
       }
@@ -256,7 +260,7 @@ bool linear_tc_supported(const Geom& g) {
   if (g.f32) return false;
   if (g.tw > 64 || (64 % g.tw) != 0 || (g.th % (64 / g.tw)) != 0) return false;  // 64 tokens = whole tile rows
   if (g.Nloc % 64 != 0 || g.Dloc % 8 != 0) return false;
-  if (g.Nloc > kMaxCols && g.Nloc % kMaxCols != 0) return false;  // unmerge token blocks
+  if (g.Nloc > kUnmergeTok && g.Nloc % kUnmergeTok != 0) return false;  // unmerge token blocks
   return true;
 }
 
@@ -270,7 +274,7 @@ cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* x
   LinParams p = make_params(g);
   const int slabs = ((g.Dloc < kMaxCols ? g.Dloc : kMaxCols) + 63) / 64;
   const int stage_bytes = (2 + 2 * slabs) * kSlab;
-  p.stages = stage_bytes <= 48 * 1024 ? 4 : 2;
+  p.stages = 2;  // two stages keep a CTA below ~100 KB so that two or three CTAs share an SM and hide each other's latencies
   if (p.stages > g.Nloc / kKC) p.stages = g.Nloc / kKC;
   const int smem = 1024 + p.stages * stage_bytes + 256;
   static bool attr = false;
@@ -285,7 +289,7 @@ cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* x
 cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void* out, uint32_t* dev_status,
                               cudaStream_t s) {
   CUtensorMap ty, tw;
-  const int n_tok = g.Nloc > kMaxCols ? kMaxCols : g.Nloc;
+  const int n_tok = g.Nloc > kUnmergeTok ? kUnmergeTok : g.Nloc;
   const uint64_t dims[3] = {(uint64_t)g.d, (uint64_t)g.Lm, (uint64_t)g.B};
   const uint64_t strides[2] = {(uint64_t)g.d * 2, (uint64_t)g.Lm * g.d * 2};
   const uint32_t box[3] = {64, 64, 1};
@@ -293,7 +297,7 @@ cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void*
     return cudaErrorInvalidValue;
   LinParams p = make_params(g);
   const int stage_bytes = 2 * kSlab + 2 * n_tok * 128;
-  p.stages = stage_bytes <= 48 * 1024 ? 4 : 2;
+  p.stages = 2;
   if (p.stages > (g.Dloc + kKC - 1) / kKC) p.stages = (g.Dloc + kKC - 1) / kKC;
   const int smem = 1024 + p.stages * stage_bytes + 256;
   static bool attr = false;
