@@ -127,16 +127,11 @@ cudaError_t launch_gram_ffma(const Geom& g, const __nv_bfloat16* y, int16_t* sq,
 struct ArgMax {
   int g, i;
 };
-__device__ __forceinline__ ArgMax better(ArgMax a, ArgMax b) {
-  return (b.g > a.g || (b.g == a.g && b.i < a.i)) ? b : a;
-}
+// Warp argmax with lowest-index ties: two hardware warp reductions (redux.sync).
 __device__ __forceinline__ ArgMax warp_argmax(ArgMax v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    ArgMax other{__shfl_xor_sync(0xffffffffu, v.g, o), __shfl_xor_sync(0xffffffffu, v.i, o)};
-    v = better(v, other);
-  }
-  return v;
+  const int g = __reduce_max_sync(0xffffffffu, v.g);
+  const int i = __reduce_min_sync(0xffffffffu, v.g == g ? v.i : INT_MAX);
+  return ArgMax{g, i};
 }
 // Posts this warp's best into red[], one barrier, then every warp reduces the partials itself.
 __device__ __forceinline__ ArgMax block_argmax(ArgMax v, ArgMax* red, int nwarps) {
@@ -144,14 +139,14 @@ __device__ __forceinline__ ArgMax block_argmax(ArgMax v, ArgMax* red, int nwarps
   v = warp_argmax(v);
   if (lane == 0) red[warp] = v;
   __syncthreads();
-  return warp_argmax(red[lane < nwarps ? lane : 0]);
+  return warp_argmax(lane < nwarps ? red[lane] : ArgMax{INT_MIN, INT_MAX});
 }
 
 template <bool kSmemS>
 __global__ void __launch_bounds__(1024) greedy_kernel(const int16_t* __restrict__ sq, int32_t* __restrict__ idx,
                                                       int Nloc, int Dloc) {
   extern __shared__ __align__(16) uint8_t greedy_smem[];
-  __shared__ int2 changed[2][kMaxNloc];  // (column j, new << 16 | old & 0xffff)
+  __shared__ int2 changed[2][kMaxNloc];  // (column j, new << 16 | old & 0xffff) of columns whose cached maximum improved
   __shared__ ArgMax red[2][32];
   __shared__ int n_changed[2];
   const int16_t* Sg = sq + (size_t)blockIdx.x * Nloc * Nloc;
@@ -167,6 +162,7 @@ __global__ void __launch_bounds__(1024) greedy_kernel(const int16_t* __restrict_
   __syncthreads();
   int32_t* out = idx + (size_t)blockIdx.x * Dloc;
   const int i = threadIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const bool live = i < Nloc;
   const int nwarps = blockDim.x >> 5;
   constexpr int kNever = INT_MIN;
@@ -196,17 +192,17 @@ __global__ void __launch_bounds__(1024) greedy_kernel(const int16_t* __restrict_
       selected = true;
       out[r] = pick.i;
     }
-    // columns whose cached maximum improves
+    // columns whose cached maximum improves, compacted into a list (one shared-memory atomic per warp)
     const int s_new = live ? (int)S[(size_t)pick.i * Nloc + i] : 0;
     const bool ch = live && s_new > m_own;
     const unsigned mask = __ballot_sync(0xffffffffu, ch);
     if (mask) {
-      const int lane = threadIdx.x & 31;
       int base = 0;
       if (lane == 0) base = atomicAdd(&n_changed[pb], __popc(mask));
       base = __shfl_sync(0xffffffffu, base, 0);
       if (ch) {
-        changed[pb][base + __popc(mask & ((1u << lane) - 1u))] = make_int2(i, (int)(((unsigned)s_new << 16) | ((unsigned)m_own & 0xFFFFu)));
+        changed[pb][base + __popc(mask & ((1u << lane) - 1u))] =
+            make_int2(i, (int)(((unsigned)s_new << 16) | ((unsigned)m_own & 0xFFFFu)));
         m_own = s_new;
       }
     }
@@ -214,10 +210,22 @@ __global__ void __launch_bounds__(1024) greedy_kernel(const int16_t* __restrict_
     const int n = n_changed[pb];
     if (threadIdx.x == 0) n_changed[pb ^ 1] = 0;  // last read one full round ago
     if (live) {
-      for (int e = 0; e < n; ++e) {
+      // four entries at a time so that the dependent shared-memory reads overlap
+      int e = 0;
+      for (; e + 4 <= n; e += 4) {
+        int2 c[4];
+        int sv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) c[u] = changed[pb][e + u];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) sv[u] = S[(size_t)c[u].x * Nloc + i];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) gain += max(sv[u] - (c[u].y >> 16), 0) - max(sv[u] - (int)(short)(c[u].y & 0xFFFF), 0);
+      }
+      for (; e < n; ++e) {
         const int2 c = changed[pb][e];
-        const int s = S[(size_t)c.x * Nloc + i];
-        gain += max(s - (c.y >> 16), 0) - max(s - (int)(short)(c.y & 0xFFFF), 0);
+        const int sv = S[(size_t)c.x * Nloc + i];
+        gain += max(sv - (c.y >> 16), 0) - max(sv - (int)(short)(c.y & 0xFFFF), 0);
       }
     }
   }
