@@ -161,6 +161,33 @@ def test_attention_parity(toma, dtype, B, L, h, dh, n_rows):
         assert_close(got[b] if rows is None else got[b][rows], want, dtype, f"attention b={b}")
 
 
+@pytest.mark.parametrize("dh,L", [(64, 1536), (128, 1000)])
+def test_attention_growing_logits_exercise_the_rescale_path(toma, dh, L):
+    """Keys grow along the sequence so that the row maximum rises by far more than the kernel's
+    rescaling threshold many times: the accumulator rescaling and the stale-maximum bookkeeping
+    must still give the exact softmax."""
+    B, h = 1, 2
+    rng = np.random.default_rng(dh)
+    u = rng.normal(size=(h, dh))
+    u /= np.linalg.norm(u, axis=1, keepdims=True)
+    q = rng.normal(size=(B, L, h, dh)) + 6.0 * u[None, None]
+    ramp = (np.arange(L) / L)[None, :, None, None]
+    k = 0.3 * rng.normal(size=(B, L, h, dh)) + 14.0 * np.sqrt(dh) / 3.0 * ramp * u[None, None]
+    v = rng.normal(size=(B, L, h, dh))
+    host = [gen.round_to_dtype(a.reshape(B, L, h * dh).astype(np.float32), "bf16") for a in (q, k, v)]
+    # the logits really do climb by tens of units of log2 over the sequence
+    s = (6.0 * u[0] @ host[1][0, :, :dh].astype(np.float64).T) / np.sqrt(dh) * 1.4427  # a typical query
+    assert s[-64:].max() - s[:64].max() > 30
+    dq, dk, dv = (to_dev(a, "bf16") for a in host)
+    o = torch.empty_like(dq)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    toma.toma_attention(B, L, h, dh, "bf16", dq, dk, dv, o, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    want = O.attention(host[0][0], host[1][0], host[2][0], h)
+    assert_close(to_host64(o)[0], want, "bf16", "attention with growing logits")
+
+
 BLOCK_CASES = [
     ("cfg1", {}, None),
     ("cfg2", {}, None),
