@@ -177,6 +177,50 @@ def workload_config(cfg):
             "parallelism": "independent batches per GPU, no collective"}
 
 
+def other_workloads(toma, torch, flush, peaks):
+    """Block latency vs full-token attention on the other SDXL- and Flux-shaped configurations
+    (one fixed input per workload; refresh and reuse steps timed separately, CUDA events, L2 flushed)."""
+    import gen
+    out = {}
+    # cfg2 states no schedule: the paper's weight interval (5) is used.  cfg4 (Flux) does not reuse across
+    # timesteps but shares one selection among the blocks of a kind within a step (19 joint blocks).
+    for name, reuse in (("cfg2", 5), ("cfg4", 19), ("cfg5a", 5)):
+        cfg = gen.config(name, reuse_interval=reuse)
+        desc = toma.desc_from_config(cfg)
+        tdt = toma.torch_dtype(desc)
+        x = torch.from_numpy(gen.features(cfg)).cuda().to(tdt)
+        y = torch.empty_like(x)
+        idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+        B, N, d = cfg.batch, cfg.n_tokens + cfg.n_extra, cfg.dim
+
+        def t_us(fn, reps=8):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            ts = []
+            for _ in range(reps):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                fn()
+                e1.record()
+                torch.cuda.synchronize()
+                ts.append(1e3 * e0.elapsed_time(e1))
+            return statistics.median(ts)
+
+        refresh = t_us(lambda: toma.toma_block(desc, 0, x, y, idx, w, ws, None))
+        reuse_us = t_us(lambda: toma.toma_block(desc, 1, x, y, idx, w, ws, None)) if reuse > 1 else None
+        full = t_us(lambda: toma.toma_attention(B, N, cfg.n_heads, cfg.head_dim, cfg.dtype, x, x, x, y, None))
+        mean = refresh if reuse == 1 else (refresh + (reuse - 1) * reuse_us) / reuse
+        out[name] = {"tokens": B * N, "reuse_interval": reuse, "refresh_us": refresh, "reuse_us": reuse_us,
+                     "block_mean_us": mean, "full_attention_us": full, "speedup_vs_full_attention": full / mean,
+                     "tokens_per_s": B * N / (mean * 1e-6),
+                     "full_attention_tflops": 4.0 * B * N * N * d / full / 1e6}
+        del x, y, idx, w, ws
+        torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -185,6 +229,7 @@ def main():
     ap.add_argument("--impl", default="toma", choices=["toma", "reference"])
     ap.add_argument("--workload", default="cfg3")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quick", action="store_true", help="skip the secondary workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "toma" else args.warmup
 
@@ -307,8 +352,12 @@ def main():
     att_flops = 4.0 * B * Lm * Lm * d
     att_tf = att_flops / (stage_ms["attention"] * 1e-3) / 1e12
     mrg_bytes = B * (cfg.n_tokens * d * esz + cfg.n_merged * d * esz + cfg.n_tiles * cfg.n_loc * cfg.d_loc * esz)
+    # traffic: dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this workload,
+    # from the ncu capture summarised in profiles/attention_tc_cfg3_cfg5a.md (only valid for the default workload)
+    traffic = 5289216 if args.workload == "cfg3" else None
     roofline = {"kernel": "attention over merged tokens", "bound": "tensor", "achieved": att_tf,
-                "peak": peaks["tf_burst"], "unit": "TFLOP/s", "frac": att_tf / peaks["tf_burst"], "traffic": None,
+                "peak": peaks["tf_burst"], "unit": "TFLOP/s", "frac": att_tf / peaks["tf_burst"], "traffic": traffic,
+                "algorithmic_flops_per_launch": att_flops,
                 "peak_source": peaks["source"] + " bf16 burst",
                 "merge_gbs": mrg_bytes / (stage_ms["merge"] * 1e-3) / 1e9,
                 "unmerge_gbs": mrg_bytes / (stage_ms["unmerge"] * 1e-3) / 1e9,
@@ -348,6 +397,8 @@ def main():
         "clocks": clocks,
         "paper_context": "paper reports -24%/-23% SDXL/Flux generation latency on RTX6000/V100/RTX8000 (other hardware)",
     }
+    if rank == 0 and world == 1 and not args.quick:
+        result["other_workloads"] = other_workloads(toma, torch, flush, peaks)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(cfg)
     if rank == 0:
