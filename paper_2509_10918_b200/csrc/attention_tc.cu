@@ -41,7 +41,7 @@ struct AttCfg {
   static constexpr int kKvSlab = kBN * 128;                // 64 key rows x 128 B
   static constexpr int kQBytes = kChunks * kQSlab;
   static constexpr int kKvBytes = kChunks * kKvSlab;       // one K or V tile
-  static constexpr int kOnesBytes = 2048;                  // [16][64] bf16 ones, K-major
+  static constexpr int kOnesBytes = kBN * 128;             // [64 keys][64] bf16 ones: the N chunk after V in the PV operand
   static constexpr int kSmemBytes = 1024 + kQBytes + 2 * kStages * kKvBytes + kOnesBytes + 256;
   static constexpr bool kSumMma = DH == 64;                // row sums on the tensor pipe, truncated P
   static constexpr int kTmemCols = 256;
@@ -284,21 +284,27 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   } else if (warp == 6) {
     // ------------------------------------------------------------------ MMA issuer for O += P V
     if (lane == 0) {
-      constexpr uint32_t idesc_o = idesc_f16(kFmtBF16, kFmtBF16, false, true, kBM, DH);
-      constexpr uint32_t idesc_l = idesc_f16(kFmtBF16, kFmtBF16, false, false, kBM, 16);
-      const uint64_t v_desc0 = smem_desc_sw128(smem_u32(sV), C::kKvSlab, 1024);
-      const uint64_t ones_desc = smem_desc_sw128(smem_u32(sOnes), 16, 1024);
-      const uint32_t t_o = tmem + C::kColO, t_l = tmem + C::kColL;
+      // With row sums on the tensor pipe the B operand is [V | ones]: N = DH + 16, the 16 extra
+      // columns come from a constant slab of ones placed one "leading byte offset" after V's slab,
+      // so one MMA per 16 keys updates O and the row sums (which sit right behind O in tensor memory).
+      constexpr uint32_t idesc_o = idesc_f16(kFmtBF16, kFmtBF16, false, true, kBM, C::kSumMma ? DH + 16 : DH);
+      uint64_t v_desc[4];
+#pragma unroll
+      for (int st = 0; st < 4; ++st) {
+        const int ss = st < C::kStages ? st : 0;
+        const uint32_t va = smem_u32(sV + ss * C::kKvBytes);
+        v_desc[st] = smem_desc_sw128(va, C::kSumMma ? smem_u32(sOnes) - va : (uint32_t)C::kKvSlab, 1024);
+      }
+      const uint32_t t_o = tmem + C::kColO;
       for (int j = 0; j < nblk; ++j) {
         const int s = j % C::kStages;
         if (!mbar_wait(&bar->p_full[j & 1], (j >> 1) & 1, dev_status, abort_flag)) break;  // implies K/V tile j has landed
         tc_fence_after();
-        const uint64_t vb = v_desc0 + (uint64_t)((s * C::kKvBytes) >> 4);
+        const uint64_t vb = s == 0 ? v_desc[0] : s == 1 ? v_desc[1] : s == 2 ? v_desc[2] : v_desc[3];
         const uint32_t t_p = tmem + C::kColS + (j & 1) * kBN;
 #pragma unroll
         for (int kk = 0; kk < kBN / 16; ++kk) {  // 16 keys per MMA: 8 packed columns of P, 16 rows of V
           mma_ts(t_o, t_p + kk * 8, vb + (uint64_t)((kk * 2048) >> 4), idesc_o, j > 0 || kk > 0);
-          if (C::kSumMma) mma_ts(t_l, t_p + kk * 8, ones_desc + (uint64_t)((kk * 32) >> 4), idesc_l, j > 0 || kk > 0);
         }
         mma_commit(&bar->v_empty[s]);  // frees the K/V slot and tells everyone that PV_j has landed
         if (j + 1 == nblk) mma_commit(&bar->o_done);  // single-phase barrier: the epilogue cannot mistake an older phase for it
