@@ -263,11 +263,13 @@ class BlockState:
 
 def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid_w: int,
                tile_h: int, tile_w: int, merge_ratio: float, tau: float, n_heads: int,
-               reuse_interval: int, n_extra: int = 0, round_fn=None):
+               reuse_interval: int, n_extra: int = 0, round_fn=None, weight_reuse_interval: int = 0):
     """One ToMA-wrapped attention call (Algorithm 3) on x [B, N + n_extra, d].
 
     Selection and weights are recomputed when step % reuse_interval == 0 and
-    reused otherwise (Sec. 4.3.2).  Merged tokens are ordered tile-major, pick
+    reused otherwise (Sec. 4.3.2).  With weight_reuse_interval > 0 the weights alone are also
+    recomputed when step % weight_reuse_interval == 0, from the current x at the cached
+    destinations (the paper's schedule: destinations every 10 steps, weights every 5).  Merged tokens are ordered tile-major, pick
     order inside a tile; the n_extra trailing tokens are not merged and join the
     attention after the merged image tokens.  The core module F is the attention
     core with Q = K = V = merged tokens.
@@ -283,15 +285,19 @@ def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid
     P, n_loc = ids.shape
     d_loc = dest_count(n_loc, merge_ratio)
     D = P * d_loc
-    if step % reuse_interval == 0 or state.idx is None:
+    refresh_sel = step % reuse_interval == 0 or state.idx is None
+    refresh_w = refresh_sel or (weight_reuse_interval > 0 and step % weight_reuse_interval == 0)
+    if refresh_sel:
         state.idx = np.empty((B, P, d_loc), dtype=np.int64)
+        for b in range(B):
+            for p in range(P):
+                state.idx[b, p], mg = select_tile(x[b, ids[p]], d_loc)
+                state.margins.append(mg)
+    if refresh_w:
         state.w = np.empty((B, P, d_loc, n_loc), dtype=np.float64)
         for b in range(B):
             for p in range(P):
-                xt = x[b, ids[p]]
-                state.idx[b, p], mg = select_tile(xt, d_loc)
-                state.margins.append(mg)
-                state.w[b, p] = merge_weights(xt, state.idx[b, p], tau)
+                state.w[b, p] = merge_weights(x[b, ids[p]], state.idx[b, p], tau)
     merged = np.empty((B, D + n_extra, d), dtype=np.float64)
     for b in range(B):
         for p in range(P):

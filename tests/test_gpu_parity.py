@@ -219,6 +219,25 @@ def test_block_sequence_parity(toma, name, over, _):
         assert_close(to_host64(out), want, cfg.dtype, f"block step {step}")
 
 
+def test_block_separate_weight_schedule_parity(toma):
+    """Destinations every 4 steps, weights every 2 (the paper refreshes weights more often than
+    destinations): indices stay put at step 2 while the weights follow the drifted features."""
+    cfg = gen.config("cfg3", batch=1, steps=5, reuse_interval=4)
+    desc = toma.desc_from_config(cfg, weight_reuse_interval=2)
+    idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    st = O.BlockState()
+    kw = dict(grid_h=cfg.grid_h, grid_w=cfg.grid_w, tile_h=cfg.tile_h, tile_w=cfg.tile_w, merge_ratio=cfg.merge_ratio,
+              tau=cfg.tau, n_heads=cfg.n_heads, reuse_interval=4, weight_reuse_interval=2)
+    for step, x_host in enumerate(gen.feature_sequence(cfg)):
+        x = to_dev(x_host, cfg.dtype)
+        out = torch.empty_like(x)
+        toma.toma_block(desc, step, x, out, idx, w, ws, None)
+        torch.cuda.synchronize()
+        want, _, _ = O.block_step(x_host, step, st, **kw)
+        assert np.array_equal(idx.cpu().numpy().astype(np.int64), st.idx)
+        assert_close(to_host64(out), want, cfg.dtype, f"block step {step}")
+
+
 def test_block_long_sequence_schedule_and_sampled_parity(toma):
     """The 28-step stress sequence: selection may only change on refresh steps, and sampled
     tiles of every refresh match the oracle exactly."""

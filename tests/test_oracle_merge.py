@@ -132,3 +132,20 @@ def test_block_step_passes_text_tokens_through():
     assert merged.shape == (1, D + 5, 32)
     assert np.array_equal(merged[0, D:], x[0, 256:].astype(np.float64))
     assert np.array_equal(out[0, 256:], att[0, D:])
+
+
+def test_block_step_separate_weight_schedule():
+    # destinations every 4 steps, weights every 2: at step 2 the indices are kept but the weights follow the new x
+    c = gen.config("cfg3", batch=1, grid_h=16, grid_w=16, tile_h=8, tile_w=8, dim=64, n_heads=2, head_dim=32, steps=4)
+    kw = dict(grid_h=16, grid_w=16, tile_h=8, tile_w=8, merge_ratio=0.5, tau=c.tau, n_heads=2, reuse_interval=4,
+              weight_reuse_interval=2)
+    st = O.BlockState()
+    xs = list(gen.feature_sequence(c))
+    O.block_step(xs[0], 0, st, **kw)
+    idx0, w0 = st.idx.copy(), st.w.copy()
+    O.block_step(xs[1], 1, st, **kw)
+    assert np.array_equal(st.idx, idx0) and np.array_equal(st.w, w0)
+    O.block_step(xs[2], 2, st, **kw)
+    assert np.array_equal(st.idx, idx0) and not np.array_equal(st.w, w0)
+    ids = O.tile_token_ids(16, 16, 8, 8)
+    assert np.allclose(st.w[0, 1], O.merge_weights(xs[2][0][ids[1]], idx0[0, 1], c.tau))
