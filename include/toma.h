@@ -124,8 +124,10 @@ TOMA_API toma_status toma_select_static(const toma_desc* desc, const void* x, in
 /* Merge weights (Sec. 4.2.1).  For each tile: logits between the D_loc selected
  * tokens and all N_loc tokens, softmax over the destination axis per source
  * token, then each destination row normalised to sum 1.
- *   w: opaque buffer of toma_weights_bytes(); holds A~^T as [batch][P][N_loc][D_loc]
- *      (fp16 in bf16 mode, fp32 in f32 mode).  Uses `ws` as scratch. */
+ *   w: opaque buffer of toma_weights_bytes(); holds A~^T per tile as [N_loc][D_loc].  In f32
+ *      mode one fp32 plane per tile; in bf16 mode two bf16 planes per tile, [2][N_loc][D_loc],
+ *      the weight rounded to bf16 and the bf16-rounded remainder, whose sum carries 16
+ *      significant bits.  Read it back as fp32 with toma_weights_export.  Uses `ws` as scratch. */
 TOMA_API toma_status toma_merge_weights(const toma_desc* desc, const void* x, const int32_t* idx, void* w, void* ws,
                                size_t ws_bytes, uint32_t* dev_status, void* stream);
 
@@ -133,11 +135,19 @@ TOMA_API toma_status toma_merge_weights(const toma_desc* desc, const void* x, co
 TOMA_API toma_status toma_merge(const toma_desc* desc, const void* w, const void* x, void* xm, uint32_t* dev_status,
                        void* stream);
 
+/* Scratch bytes toma_attention needs for this shape (0 when the shape's kernel needs none, or
+ * when an argument is invalid).  Host-only. */
+TOMA_API size_t toma_attention_workspace_bytes(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim,
+                                               int32_t dtype);
+
 /* Multi-head attention core softmax(Q K^T / sqrt(head_dim)) V (Eq. 1 with tau = 1), no mask.
- *   q, k, v, o: [batch][len][n_heads][head_dim]. */
+ *   q, k, v, o: [batch][len][n_heads][head_dim], device.
+ *   ws: device scratch of at least toma_attention_workspace_bytes(), 16-byte aligned, caller-owned,
+ *       no initialisation needed; may be NULL when that size is 0.  The call's kernels write it, so
+ *       calls that can overlap on the GPU need separate scratch.  TOMA_ERR_WORKSPACE otherwise. */
 TOMA_API toma_status toma_attention(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim, int32_t dtype,
-                           const void* q, const void* k, const void* v, void* o, uint32_t* dev_status,
-                           void* stream);
+                           const void* q, const void* k, const void* v, void* o, void* ws, size_t ws_bytes,
+                           uint32_t* dev_status, void* stream);
 
 /* Unmerge out = A~^T y per tile, written back in spatial order (Sec. 4.2.2, Algorithm 3 step 3).
  *   y [batch][D + n_extra][dim] in; out [batch][N + n_extra][dim]; extra tokens copied. */

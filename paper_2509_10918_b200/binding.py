@@ -20,7 +20,8 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_RATIO", "ERR_TA
                 "ERR_UNSUPPORTED", "ERR_CUDA", "ERR_TIMEOUT", "ERR_SCRATCH_LIMIT"]
 
 EXPORTS = ["toma_select_static", "toma_launch_counter", "toma_workspace_bytes", "toma_weights_bytes", "toma_dest_per_tile", "toma_validate", "toma_status_str",
-           "toma_select", "toma_merge_weights", "toma_merge", "toma_attention", "toma_unmerge", "toma_block",
+           "toma_select", "toma_merge_weights", "toma_merge", "toma_attention_workspace_bytes", "toma_attention",
+           "toma_unmerge", "toma_block",
            "toma_weights_export", "toma_weights_import"]
 
 
@@ -71,8 +72,10 @@ def _load() -> ctypes.CDLL:
     lib.toma_unmerge.restype = c_int32
     lib.toma_unmerge.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.toma_attention.restype = c_int32
+    lib.toma_attention_workspace_bytes.restype = c_size_t
+    lib.toma_attention_workspace_bytes.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32]
     lib.toma_attention.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
-                                   c_void_p, c_void_p, c_void_p]
+                                   c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
     lib.toma_block.restype = c_int32
     lib.toma_block.argtypes = [P, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p,
                                c_void_p]
@@ -175,10 +178,28 @@ def toma_unmerge(desc, w, y, out, dev_status=None):
            "toma_unmerge")
 
 
-def toma_attention(batch, length, n_heads, head_dim, dtype, q, k, v, o, dev_status=None):
-    code = {"bf16": TOMA_BF16, "f32": TOMA_F32, TOMA_BF16: TOMA_BF16, TOMA_F32: TOMA_F32}[dtype]
-    _check(lib.toma_attention(batch, length, n_heads, head_dim, code, _ptr(q), _ptr(k), _ptr(v), _ptr(o),
-                              _ptr(dev_status), _stream()), "toma_attention")
+def _dtype_code(dtype) -> int:
+    return {"bf16": TOMA_BF16, "f32": TOMA_F32, TOMA_BF16: TOMA_BF16, TOMA_F32: TOMA_F32}[dtype]
+
+
+def toma_attention_workspace_bytes(batch, length, n_heads, head_dim, dtype) -> int:
+    return int(lib.toma_attention_workspace_bytes(batch, length, n_heads, head_dim, _dtype_code(dtype)))
+
+
+_attention_ws = {}
+
+
+def toma_attention(batch, length, n_heads, head_dim, dtype, q, k, v, o, dev_status=None, ws=None):
+    """ws: scratch tensor of toma_attention_workspace_bytes(); when omitted, one buffer per device is
+    kept and grown on demand (callers that overlap attention calls on several streams pass their own)."""
+    code = _dtype_code(dtype)
+    need = toma_attention_workspace_bytes(batch, length, n_heads, head_dim, code)
+    if ws is None and need > 0:
+        ws = _attention_ws.get(q.device)
+        if ws is None or ws.numel() < need:
+            ws = _attention_ws[q.device] = torch.empty(need, dtype=torch.uint8, device=q.device)
+    _check(lib.toma_attention(batch, length, n_heads, head_dim, code, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(ws),
+                              ws.numel() if ws is not None else 0, _ptr(dev_status), _stream()), "toma_attention")
 
 
 def toma_block(desc, step, x, out, idx_state, w_state, ws, dev_status=None):

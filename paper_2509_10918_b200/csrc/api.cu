@@ -39,6 +39,12 @@ toma_status make_geom(const toma_desc* desc, Geom* g) {
   return TOMA_OK;
 }
 
+static bool attention_on_tc(int dh, bool f32) { return !f32 && (dh == 64 || dh == 128); }
+
+static size_t attention_ws_bytes(int B, int L, int heads, int dh, bool f32) {
+  return attention_on_tc(dh, f32) ? attention_tc_workspace_bytes(B, L, heads, dh) : 0;
+}
+
 WsLayout ws_layout(const Geom& g) {
   WsLayout l;
   const size_t tiles = (size_t)g.B * g.P;
@@ -50,6 +56,7 @@ WsLayout ws_layout(const Geom& g) {
   l.wts_off = off;    off = align_up(off + (weights_tc_supported(g) ? weights_tc_scratch_bytes(g) : 0), 256);
   l.xm_off = off;     off = align_up(off + (size_t)g.B * g.Lm * g.d * esz, 256);
   l.att_off = off;    off = align_up(off + (size_t)g.B * g.Lm * g.d * esz, 256);
+  l.att_ws_off = off; off = align_up(off + attention_ws_bytes(g.B, g.Lm, g.heads, g.dh, g.f32), 256);
   l.total = off;
   return l;
 }
@@ -88,10 +95,13 @@ static cudaError_t do_weights(const Geom& g, const void* x, const int32_t* idx, 
   return launch_weights_simt(g, x, idx, w, (float*)(ws + l.logits_off), s);
 }
 
-static cudaError_t do_merge(const Geom& g, const void* w, const void* x, void* xm, uint32_t* dev_status,
-                            cudaStream_t s) {
+// `zero`, `zero_bytes`: a region to clear on the side; *zeroed says whether the path taken did it.
+static cudaError_t do_merge(const Geom& g, const void* w, const void* x, void* xm, void* zero, size_t zero_bytes,
+                            bool* zeroed, uint32_t* dev_status, cudaStream_t s) {
+  if (zeroed) *zeroed = false;
   if (linear_tc_supported(g)) {
-    cudaError_t e = launch_merge_tc(g, w, x, xm, dev_status, s);
+    cudaError_t e = launch_merge_tc(g, w, x, xm, zero, zero_bytes, dev_status, s);
+    if (zeroed) *zeroed = e == cudaSuccess && zero_bytes > 0;
     return e != cudaSuccess ? e : launch_copy_extra(g, x, xm, true, s);
   }
   return launch_merge_simt(g, w, x, xm, s);
@@ -107,8 +117,10 @@ static cudaError_t do_unmerge(const Geom& g, const void* w, const void* y, void*
 }
 
 static cudaError_t do_attention(int B, int L, int heads, int dh, bool f32, const void* q, const void* k,
-                                const void* v, void* o, uint32_t* dev_status, cudaStream_t s) {
-  if (!f32 && (dh == 64 || dh == 128)) return launch_attention_tc(B, L, heads, dh, q, k, v, o, dev_status, s);
+                                const void* v, void* o, void* att_ws, bool tickets_clean, uint32_t* dev_status,
+                                cudaStream_t s) {
+  if (attention_on_tc(dh, f32))
+    return launch_attention_tc(B, L, heads, dh, q, k, v, o, att_ws, tickets_clean, dev_status, s);
   return launch_attention_simt(B, L, heads, dh, f32, q, k, v, o, s);
 }
 
@@ -187,7 +199,7 @@ toma_status toma_merge(const toma_desc* desc, const void* w, const void* x, void
   if (st != TOMA_OK) return st;
   if (!w || !x || !xm) return TOMA_ERR_NULL;
   if (misaligned(x) || misaligned(w) || misaligned(xm)) return TOMA_ERR_SHAPE;
-  return cuda_ok(do_merge(g, w, x, xm, dev_status, (cudaStream_t)stream));
+  return cuda_ok(do_merge(g, w, x, xm, nullptr, 0, nullptr, dev_status, (cudaStream_t)stream));
 }
 
 toma_status toma_unmerge(const toma_desc* desc, const void* w, const void* y, void* out, uint32_t* dev_status,
@@ -200,15 +212,22 @@ toma_status toma_unmerge(const toma_desc* desc, const void* w, const void* y, vo
   return cuda_ok(do_unmerge(g, w, y, out, dev_status, (cudaStream_t)stream));
 }
 
+size_t toma_attention_workspace_bytes(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim, int32_t dtype) {
+  if ((dtype != TOMA_BF16 && dtype != TOMA_F32) || batch < 1 || len < 1 || n_heads < 1 || head_dim < 1) return 0;
+  return attention_ws_bytes(batch, len, n_heads, head_dim, dtype == TOMA_F32);
+}
+
 toma_status toma_attention(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim, int32_t dtype,
-                           const void* q, const void* k, const void* v, void* o, uint32_t* dev_status,
-                           void* stream) {
+                           const void* q, const void* k, const void* v, void* o, void* ws, size_t ws_bytes,
+                           uint32_t* dev_status, void* stream) {
   if (dtype != TOMA_BF16 && dtype != TOMA_F32) return TOMA_ERR_DTYPE;
   if (batch < 1 || len < 1 || n_heads < 1 || head_dim < 1) return TOMA_ERR_SHAPE;
   if (!q || !k || !v || !o) return TOMA_ERR_NULL;
   if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(o)) return TOMA_ERR_SHAPE;
   if (!attention_supported_simt(head_dim)) return TOMA_ERR_UNSUPPORTED;
-  return cuda_ok(do_attention(batch, len, n_heads, head_dim, dtype == TOMA_F32, q, k, v, o, dev_status,
+  const size_t need = attention_ws_bytes(batch, len, n_heads, head_dim, dtype == TOMA_F32);
+  if (need > 0 && (!ws || misaligned(ws) || ws_bytes < need)) return TOMA_ERR_WORKSPACE;
+  return cuda_ok(do_attention(batch, len, n_heads, head_dim, dtype == TOMA_F32, q, k, v, o, ws, false, dev_status,
                               (cudaStream_t)stream));
 }
 
@@ -233,8 +252,11 @@ toma_status toma_block(const toma_desc* desc, int32_t step, const void* x, void*
   if (e == cudaSuccess && refresh_w) e = do_weights(g, x, idx_state, w_state, wsb, dev_status, s);
   void* xm = wsb + l.xm_off;
   void* att = wsb + l.att_off;
-  if (e == cudaSuccess) e = do_merge(g, w_state, x, xm, dev_status, s);
-  if (e == cudaSuccess) e = do_attention(g.B, g.Lm, g.heads, g.dh, g.f32, xm, xm, xm, att, dev_status, s);
+  // the merge kernel clears the attention kernel's tickets on the side (saves a memset between them)
+  bool tickets_clean = false;
+  const size_t ticket_bytes = attention_on_tc(g.dh, g.f32) ? attention_tc_ticket_bytes(g.B, g.Lm, g.heads) : 0;
+  if (e == cudaSuccess) e = do_merge(g, w_state, x, xm, wsb + l.att_ws_off, ticket_bytes, &tickets_clean, dev_status, s);
+  if (e == cudaSuccess) e = do_attention(g.B, g.Lm, g.heads, g.dh, g.f32, xm, xm, xm, att, wsb + l.att_ws_off, tickets_clean, dev_status, s);
   if (e == cudaSuccess) e = do_unmerge(g, w_state, att, out, dev_status, s);
   return cuda_ok(e);
 }

@@ -1,9 +1,18 @@
 // Attention core softmax(Q K^T / sqrt(dh)) V (Eq. 1 with tau = 1) on the sm_100a tensor
 // cores, bf16 in / bf16 out, fp32 softmax and accumulation.
 //
-// One CTA per (batch, head, 128 queries), keys in tiles of 64; two CTAs are resident per SM.
-// Warp 4 feeds K and V tiles through separate TMA rings, warp 5 issues tcgen05 MMAs, warps 0..3
-// (one thread per query row) run the online softmax straight out of tensor memory:
+// Work unit = (batch, head, 128 queries); one iteration = one 64-key tile of a unit.  The launch is
+// persistent, two CTAs per SM, and the units' iterations, laid end to end, are cut into one equal
+// contiguous span per CTA, so that every CTA runs the same number of key tiles whatever the unit
+// count (a launch of whole units leaves most SMs idle in its last wave: 320 units on 296 CTA slots
+// took as long as 592).  A span that covers only part of a unit's keys leaves the unnormalised
+// accumulator, the reference maximum and the row sum of its piece in global scratch; the warp that
+// arrives last at the (unit, warp) ticket adds the pieces up and writes the output rows.  Nobody
+// waits for another CTA.
+//
+// Inside a CTA warp 4 feeds K and V tiles through a TMA ring, warps 5 and 6 issue tcgen05 MMAs,
+// warp 7 publishes a partial first piece (memory fence and tickets, off everybody else's path),
+// warps 0..3 (one thread per query row) run the online softmax straight out of tensor memory:
 //   S_j = Q K_j^T          -> tensor memory, two 64-column buffers; S_{j+1} is issued before the
 //                             softmax of tile j has finished, so the softmax warps never wait for a
 //                             round trip through the MMA warp
@@ -20,6 +29,8 @@
 // The whole S row of a tile (64 fp32) is fetched with one tensor-memory round trip and kept in
 // registers for both the maximum and the exponentials.
 // Keys past the sequence end are zero-filled by TMA and masked out.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "tc.cuh"
 
@@ -49,12 +60,46 @@ struct AttCfg {
 };
 
 struct Barriers {
-  uint64_t q_full;
-  uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
-  uint64_t s_full[2], p_full[2], pv_done, o_done;
+  uint64_t q_full, q_empty;           // per piece: Q landed / every S MMA of the piece has read Q
+  uint64_t k_full[4], v_empty[4];     // per tile: K and V landed / PV MMAs of the tile done
+  uint64_t s_full[2], p_full[2];      // per tile: S ready for the softmax / P ready for the PV MMAs
+  uint64_t o_done, o_free;            // per piece: accumulator complete / epilogue has read it
+  uint64_t pub_ready, pub_done;       // first partial piece: written by the softmax warps / published, tickets drawn
+  uint32_t first_ticket[4];           // per softmax warp: ticket its first (partial) piece drew
   uint32_t tmem_base;
   int abort_flag;
 };
+
+// The iterations [0, T) are cut into G spans at multiples of `quantum`: with T / quantum = q * G + r,
+// the first r spans hold q + 1 quanta and the others q.
+// quantum = 1 balances the spans to within one key tile and splits units; quantum = nblk keeps
+// units whole (no scratch traffic), which wins when the unit count happens to fill the CTAs evenly.
+struct Spans {
+  int T, G, nblk, quantum, q, r;
+  __host__ __device__ int bound(int g) const { return (g * q + (g < r ? g : r)) * quantum; }
+  // the CTA whose span holds iteration `it` (quantum 1 only)
+  __host__ __device__ int owner(int it) const {
+    const int big = r * (q + 1);
+    return it < big ? it / (q + 1) : r + (it - big) / q;
+  }
+};
+
+// One piece = the part of a span inside one unit: key tiles [k0, k0 + cnt) of unit u.
+struct Piece {
+  int u, k0, cnt;
+};
+__device__ __forceinline__ Piece piece_at(int it, int it_end, int nblk) {
+  Piece p;
+  p.u = it / nblk;
+  p.k0 = it - p.u * nblk;
+  const int left = it_end - it;
+  p.cnt = left < nblk - p.k0 ? left : nblk - p.k0;
+  return p;
+}
+
+// Scratch of one piece: O as [DH / 4][128 rows] float4, then m[128], l[128].
+template <int DH>
+__host__ __device__ constexpr size_t piece_floats() { return (size_t)kBM * DH + 2 * kBM; }
 
 __device__ __forceinline__ float ex2_mufu(float x) {
   float y;
@@ -186,11 +231,231 @@ __device__ __forceinline__ bool softmax_tile(uint32_t sb, uint32_t ob, float sca
   return true;
 }
 
+// 32 accumulator columns of one row, scaled and rounded to bf16: 64 contiguous bytes.
+__device__ __forceinline__ void store_row32(__nv_bfloat16* dst, const uint32_t (&r)[32], float inv) {
+#pragma unroll
+  for (int e = 0; e < 32; e += 8) {
+    uint4 v;
+    v.x = pack_bf16_rn(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
+    v.y = pack_bf16_rn(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+    v.z = pack_bf16_rn(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+    v.w = pack_bf16_rn(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+    *reinterpret_cast<uint4*>(dst + e) = v;
+  }
+}
+
+// Where the output rows of unit u start for this thread's query row (nullptr past the sequence end).
 template <int DH>
-__global__ void __launch_bounds__(224, 2)
+__device__ __forceinline__ __nv_bfloat16* out_row(__nv_bfloat16* o, int u, int row, int L, int heads) {
+  const int nq = (L + kBM - 1) / kBM;
+  const int bh = u / nq, qi = (u - bh * nq) * kBM + row, b = bh / heads, h = bh - b * heads;
+  if (qi >= L) return nullptr;
+  return o + ((size_t)b * L + qi) * ((size_t)heads * DH) + (size_t)h * DH;
+}
+
+// Scratch slot of the piece of unit u that CTA g left: its first piece sits in slot 0, a later
+// partial piece (necessarily its last) in slot 1.
+template <int DH>
+__device__ __forceinline__ const float* slot_of(const float* pieces, const Spans& sp, int g, int u) {
+  const int first_unit = sp.bound(g) / sp.nblk;
+  return pieces + (size_t)(2 * g + (u > first_unit ? 1 : 0)) * piece_floats<DH>();
+}
+
+// Adds up the pieces of one query row of unit u, left by CTAs g_first..g_last:
+//   O = sum_i 2^(m_i - M) O_i / sum_i 2^(m_i - M) l_i,  M = max_i m_i  (m in the log2 domain).
+// Contributors are taken two at a time so that their loads are in flight together (the usual unit
+// has two).  Loads bypass L1: the pieces were written by other SMs during this launch.
+template <int DH>
+__device__ __noinline__ void combine_rows(const float* pieces, Spans sp, int u, int g_first, int g_last, int row,
+                                          __nv_bfloat16* dst) {
+  constexpr size_t kM = (size_t)kBM * DH, kL = (size_t)kBM * DH + kBM;
+  float M = -INFINITY;
+  for (int g = g_first; g <= g_last; g += 2) {
+    const float* sa = slot_of<DH>(pieces, sp, g, u);
+    const float* sb = g < g_last ? slot_of<DH>(pieces, sp, g + 1, u) : sa;
+    M = max3(M, __ldcg(sa + kM + row), __ldcg(sb + kM + row));
+  }
+#pragma unroll 1
+  for (int half = 0; half < DH / 64; ++half) {  // 64 accumulator columns at a time
+    float denom = 0.f;
+    float acc[64];
+#pragma unroll
+    for (int e = 0; e < 64; ++e) acc[e] = 0.f;
+    for (int g = g_first; g <= g_last; g += 2) {
+      const float* sa = slot_of<DH>(pieces, sp, g, u);
+      const float* sb = g < g_last ? slot_of<DH>(pieces, sp, g + 1, u) : sa;
+      const float ma = __ldcg(sa + kM + row), la = __ldcg(sa + kL + row);
+      const float mb = __ldcg(sb + kM + row), lb = __ldcg(sb + kL + row);
+      const float wa = ex2_mufu(ma - M), wb = g < g_last ? ex2_mufu(mb - M) : 0.f;
+      denom += wa * la + wb * lb;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        float4 va[8], vb[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          va[q] = __ldcg(reinterpret_cast<const float4*>(sa) + (size_t)(half * 16 + c * 8 + q) * kBM + row);
+          vb[q] = __ldcg(reinterpret_cast<const float4*>(sb) + (size_t)(half * 16 + c * 8 + q) * kBM + row);
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          float* a4 = &acc[c * 32 + 4 * q];
+          a4[0] = fmaf(wa, va[q].x, fmaf(wb, vb[q].x, a4[0]));
+          a4[1] = fmaf(wa, va[q].y, fmaf(wb, vb[q].y, a4[1]));
+          a4[2] = fmaf(wa, va[q].z, fmaf(wb, vb[q].z, a4[2]));
+          a4[3] = fmaf(wa, va[q].w, fmaf(wb, vb[q].w, a4[3]));
+        }
+      }
+    }
+    if (!dst) continue;
+    const float inv = 1.f / denom;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      uint32_t r[32];
+#pragma unroll
+      for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(acc[c * 32 + e]);
+      store_row32(dst + half * 64 + c * 32, r, inv);
+    }
+  }
+}
+
+__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// Publishes this warp's 32 rows of a piece and takes the (unit, warp) ticket.  Returns the number
+// of contributors that had taken it before.
+__device__ __forceinline__ uint32_t take_ticket(uint32_t* ticket, int lane) {
+  __threadfence();
+  __syncwarp();
+  uint32_t t = 0;
+  if (lane == 0) t = atomicAdd(ticket, 1u);
+  return __shfl_sync(0xffffffffu, t, 0);
+}
+
+// End of a piece, run by the softmax warps; waits for the piece's accumulator to be complete, then
+//   - a piece that covers all keys of its unit is normalised and written out;
+//   - the last piece of the CTA's span, when the unit's only other contributor has already
+//     published (it ran at the start of its own span, so it normally has), is added to that
+//     contributor's piece straight from tensor memory and written out: nothing of it goes through
+//     scratch, and the other piece is fetched while the last MMAs drain;
+//   - any other piece is left in scratch with its reference maximum and row sum and a (unit, warp)
+//     ticket is drawn; the warp that draws a unit's last ticket adds its pieces up.  A last piece
+//     does that here; a first piece, with more of the span to come, hands the fence and the
+//     tickets' round trips to the publisher thread and looks at the outcome in settle_first_piece.
+// `peek` is the ticket as read (with acquire) when the piece began.
+// Kept out of line so that its registers do not weigh on the softmax loop.  Returns false when the
+// wait ran out.
+template <int DH>
+__device__ __noinline__ bool finish_piece(uint32_t ob, Barriers* bar, Piece p, int pc, bool last_of_span, uint32_t peek,
+                                          int row, float m_used, float l, __nv_bfloat16* o, int L, int heads, Spans sp,
+                                          uint32_t* tickets, float* pieces, uint32_t* dev_status) {
+  using C = AttCfg<DH>;
+  constexpr size_t kM = (size_t)kBM * DH, kL = (size_t)kBM * DH + kBM;
+  const int warp = row >> 5, lane = row & 31;
+  const bool whole = p.cnt == sp.nblk;
+  uint32_t* ticket = tickets + (size_t)p.u * 4 + warp;
+  int g_first = 0, g_last = 0;
+  bool direct = false;
+  const float* other = nullptr;
+  float m_o = 0.f, l_o = 0.f;
+  float4 vo[16];
+  if (!whole) {
+    g_first = sp.owner(p.u * sp.nblk);
+    g_last = sp.owner((p.u + 1) * sp.nblk - 1);
+    if (last_of_span && g_last == g_first + 1 && peek == 1u) {
+      direct = true;
+      other = slot_of<DH>(pieces, sp, (int)blockIdx.x == g_first ? g_last : g_first, p.u);
+      m_o = __ldcg(other + kM + row);
+      l_o = __ldcg(other + kL + row);
+#pragma unroll
+      for (int q = 0; q < 16; ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)q * kBM + row);
+    }
+  }
+  if (!mbar_wait(&bar->o_done, pc & 1, dev_status, &bar->abort_flag)) return false;
+  tc_fence_after();
+  if (C::kSumMma) {
+    uint32_t rs[16];
+    tmem_ld16(ob + DH, rs);
+    tmem_wait_ld();
+    l = __uint_as_float(rs[0]);
+  }
+  __nv_bfloat16* dst = out_row<DH>(o, p.u, row, L, heads);
+  float* slot = pieces + (size_t)(2 * blockIdx.x + (pc > 0 ? 1 : 0)) * piece_floats<DH>();
+  float w_own = 1.f, w_o = 0.f, inv = 1.f / l;
+  if (direct) {
+    const float M = fmaxf(m_used, m_o);
+    w_own = ex2_mufu(m_used - M);
+    w_o = ex2_mufu(m_o - M);
+    inv = 1.f / (w_own * l + w_o * l_o);
+  }
+#pragma unroll
+  for (int c = 0; c < DH / 32; ++c) {
+    uint32_t r[32];
+    tmem_ld32(ob + c * 32, r);
+    tmem_wait_ld();
+    if (whole) {
+      if (dst) store_row32(dst + c * 32, r, inv);
+    } else if (direct) {
+      if (c > 0 && (c & 1) == 0) {  // next 64 columns of the other piece
+#pragma unroll
+        for (int q = 0; q < 16; ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)(c * 8 + q) * kBM + row);
+      }
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const float4 v = vo[(c & 1) * 8 + q];
+        r[4 * q] = __float_as_uint(fmaf(w_own, __uint_as_float(r[4 * q]), w_o * v.x));
+        r[4 * q + 1] = __float_as_uint(fmaf(w_own, __uint_as_float(r[4 * q + 1]), w_o * v.y));
+        r[4 * q + 2] = __float_as_uint(fmaf(w_own, __uint_as_float(r[4 * q + 2]), w_o * v.z));
+        r[4 * q + 3] = __float_as_uint(fmaf(w_own, __uint_as_float(r[4 * q + 3]), w_o * v.w));
+      }
+      if (dst) store_row32(dst + c * 32, r, inv);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 32; e += 4)
+        reinterpret_cast<float4*>(slot)[(size_t)(c * 8 + (e >> 2)) * kBM + row] =
+            make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+    }
+  }
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(&bar->o_free);  // the next piece's first PV product may overwrite the accumulator
+  if (whole || direct) return true;
+  slot[kM + row] = m_used;
+  slot[kL + row] = l;
+  if (!last_of_span) {  // the publisher thread fences, draws the tickets and leaves them for settle_first_piece
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&bar->pub_ready);
+  } else if (take_ticket(ticket, lane) == (uint32_t)(g_last - g_first)) {
+    __threadfence();
+    combine_rows<DH>(pieces, sp, p.u, g_first, g_last, row, dst);
+  }
+  return true;
+}
+
+// End of a CTA's span: if its first piece was partial and took the unit's last ticket (the other
+// contributors, which run that unit at the end of their spans, are normally later), add the
+// unit's pieces up now.
+template <int DH>
+__device__ __noinline__ void settle_first_piece(Barriers* bar, int it_begin, int it_end, int row, __nv_bfloat16* o, int L,
+                                                int heads, Spans sp, const float* pieces, uint32_t* dev_status) {
+  const int nblk = sp.nblk, u = it_begin / nblk;
+  const bool first_partial = it_begin > u * nblk || it_end < (u + 1) * nblk;
+  if (!first_partial || it_end <= (u + 1) * nblk) return;  // whole, or also the span's last piece: settled already
+  const int g_first = sp.owner(u * nblk), g_last = sp.owner((u + 1) * nblk - 1);
+  if (!mbar_wait(&bar->pub_done, 0, dev_status, &bar->abort_flag)) return;
+  if (bar->first_ticket[row >> 5] != (uint32_t)(g_last - g_first)) return;
+  __threadfence();
+  combine_rows<DH>(pieces, sp, u, g_first, g_last, row, out_row<DH>(o, u, row, L, heads));
+}
+
+template <int DH>
+__global__ void __launch_bounds__(256, 2)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, int L, int heads,
-                    float scale_log2, uint32_t* dev_status) {
+                    float scale_log2, Spans sp, uint32_t* __restrict__ tickets, float* __restrict__ pieces,
+                    uint32_t* dev_status) {
   using C = AttCfg<DH>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -201,23 +466,27 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   Barriers* bar = reinterpret_cast<Barriers*>(sOnes + C::kOnesBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int q0 = blockIdx.x * kBM, h = blockIdx.y, b = blockIdx.z;
-  const int nblk = (L + kBN - 1) / kBN;
+  const int nblk = sp.nblk;
+  const int nq = (L + kBM - 1) / kBM;  // units per (batch, head)
+  const int it_begin = sp.bound(blockIdx.x), it_end = sp.bound(blockIdx.x + 1);
+  // Every role walks the same pieces; `n` counts this CTA's tiles across pieces (ring slots, S
+  // buffers and their barrier phases follow n), `pc` counts pieces (phases of the per-piece barriers).
 
   if (threadIdx.x == 0) {
     mbar_init(&bar->q_full, 1);
+    mbar_init(&bar->q_empty, 1);
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&bar->k_full[s], 1);
-      mbar_init(&bar->k_empty[s], 1);
-      mbar_init(&bar->v_full[s], 1);
       mbar_init(&bar->v_empty[s], 1);
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bar->s_full[s], 1);
       mbar_init(&bar->p_full[s], 4);  // one arrival per softmax warp
     }
-    mbar_init(&bar->pv_done, 1);
     mbar_init(&bar->o_done, 1);
+    mbar_init(&bar->o_free, 4);
+    mbar_init(&bar->pub_ready, 4);
+    mbar_init(&bar->pub_done, 1);
     bar->abort_flag = 0;
     mbar_fence_init();
   }
@@ -238,17 +507,27 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       prefetch_tmap(&tm_q);
       prefetch_tmap(&tm_k);
       prefetch_tmap(&tm_v);
-      mbar_expect_tx(&bar->q_full, C::kQBytes);
-      for (int c = 0; c < C::kChunks; ++c) tma_load_3d(sQ + c * C::kQSlab, &tm_q, &bar->q_full, h * DH + c * 64, q0, b);
-      for (int j = 0; j < nblk; ++j) {
-        const int s = j % C::kStages;
-        const uint32_t par = ((j / C::kStages) - 1) & 1;
-        if (j >= C::kStages && !mbar_wait(&bar->v_empty[s], par, dev_status, abort_flag)) break;
-        mbar_expect_tx(&bar->k_full[s], 2 * C::kKvBytes);  // K and V of tile j arrive under one barrier
-        for (int c = 0; c < C::kChunks; ++c)
-          tma_load_3d(sK + s * C::kKvBytes + c * C::kKvSlab, &tm_k, &bar->k_full[s], h * DH + c * 64, j * kBN, b);
-        for (int c = 0; c < C::kChunks; ++c)
-          tma_load_3d(sV + s * C::kKvBytes + c * C::kKvSlab, &tm_v, &bar->k_full[s], h * DH + c * 64, j * kBN, b);
+      bool ok = true;
+      int n = 0, pc = 0;
+      for (int it = it_begin; ok && it < it_end; ++pc) {
+        const Piece p = piece_at(it, it_end, nblk);
+        it += p.cnt;
+        const int bh = p.u / nq, q0 = (p.u - bh * nq) * kBM, b = bh / heads, h = bh - b * heads;
+        // Q's buffer is free once the S MMAs of the previous piece have read it
+        if (pc > 0 && !mbar_wait(&bar->q_empty, (pc - 1) & 1, dev_status, abort_flag)) break;
+        mbar_expect_tx(&bar->q_full, C::kQBytes);
+        for (int c = 0; c < C::kChunks; ++c) tma_load_3d(sQ + c * C::kQSlab, &tm_q, &bar->q_full, h * DH + c * 64, q0, b);
+        for (int j = 0; j < p.cnt; ++j, ++n) {
+          const int s = n % C::kStages;
+          const uint32_t par = ((n / C::kStages) - 1) & 1;
+          if (n >= C::kStages && !mbar_wait(&bar->v_empty[s], par, dev_status, abort_flag)) { ok = false; break; }
+          const int key0 = (p.k0 + j) * kBN;
+          mbar_expect_tx(&bar->k_full[s], 2 * C::kKvBytes);  // K and V of a tile arrive under one barrier
+          for (int c = 0; c < C::kChunks; ++c)
+            tma_load_3d(sK + s * C::kKvBytes + c * C::kKvSlab, &tm_k, &bar->k_full[s], h * DH + c * 64, key0, b);
+          for (int c = 0; c < C::kChunks; ++c)
+            tma_load_3d(sV + s * C::kKvBytes + c * C::kKvSlab, &tm_v, &bar->k_full[s], h * DH + c * 64, key0, b);
+        }
       }
     }
   } else if (warp == 5) {
@@ -261,24 +540,34 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // field (no carry: all tiles live below 256 KB).
       const uint64_t q_desc = smem_desc_sw128(smem_u32(sQ), 16, 1024);
       const uint64_t k_desc0 = smem_desc_sw128(smem_u32(sK), 16, 1024);
-      bool ok = mbar_wait(&bar->q_full, 0, dev_status, abort_flag);
-      for (int j = 0; ok && j < nblk; ++j) {
-        const int s = j % C::kStages;
-        if (!mbar_wait(&bar->k_full[s], (j / C::kStages) & 1, dev_status, abort_flag)) break;
-        // S_j overwrites the buffer whose P_{j-2} the PV (and row-sum) MMAs of tile j-2 read as their
-        // A operand.  MMAs into different accumulators are not ordered among themselves, so that read
-        // has to be complete before the overwrite is issued.
-        if (j >= 2 && !mbar_wait(&bar->v_empty[(j - 2) % C::kStages], ((j - 2) / C::kStages) & 1, dev_status, abort_flag)) break;
-        tc_fence_after();
-        const uint64_t kb = k_desc0 + (uint64_t)((s * C::kKvBytes) >> 4);
-        const uint32_t t_s = tmem + C::kColS + (j & 1) * kBN;
+      bool ok = true;
+      int n = 0, pc = 0;
+      for (int it = it_begin; ok && it < it_end; ++pc) {
+        const Piece p = piece_at(it, it_end, nblk);
+        it += p.cnt;
+        if (!mbar_wait(&bar->q_full, pc & 1, dev_status, abort_flag)) break;
+        for (int j = 0; j < p.cnt; ++j, ++n) {
+          const int s = n % C::kStages;
+          if (!mbar_wait(&bar->k_full[s], (n / C::kStages) & 1, dev_status, abort_flag)) { ok = false; break; }
+          // S_n overwrites the buffer whose P_{n-2} the PV (and row-sum) MMAs of tile n-2 read as their
+          // A operand.  MMAs into different accumulators are not ordered among themselves, so that read
+          // has to be complete before the overwrite is issued.
+          if (n >= 2 && !mbar_wait(&bar->v_empty[(n - 2) % C::kStages], ((n - 2) / C::kStages) & 1, dev_status, abort_flag)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint64_t kb = k_desc0 + (uint64_t)((s * C::kKvBytes) >> 4);
+          const uint32_t t_s = tmem + C::kColS + (n & 1) * kBN;
 #pragma unroll
-        for (int kk = 0; kk < DH / 16; ++kk) {
-          const uint64_t qoff = (uint64_t)(((kk >> 2) * C::kQSlab + (kk & 3) * 32) >> 4);
-          const uint64_t koff = (uint64_t)(((kk >> 2) * C::kKvSlab + (kk & 3) * 32) >> 4);
-          mma_ss(t_s, q_desc + qoff, kb + koff, idesc_s, kk > 0);
+          for (int kk = 0; kk < DH / 16; ++kk) {
+            const uint64_t qoff = (uint64_t)(((kk >> 2) * C::kQSlab + (kk & 3) * 32) >> 4);
+            const uint64_t koff = (uint64_t)(((kk >> 2) * C::kKvSlab + (kk & 3) * 32) >> 4);
+            mma_ss(t_s, q_desc + qoff, kb + koff, idesc_s, kk > 0);
+          }
+          mma_commit(&bar->s_full[n & 1]);
         }
-        mma_commit(&bar->s_full[j & 1]);
+        if (ok) mma_commit(&bar->q_empty);
       }
     }
   } else if (warp == 6) {
@@ -296,18 +585,46 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         v_desc[st] = smem_desc_sw128(va, C::kSumMma ? smem_u32(sOnes) - va : (uint32_t)C::kKvSlab, 1024);
       }
       const uint32_t t_o = tmem + C::kColO;
-      for (int j = 0; j < nblk; ++j) {
-        const int s = j % C::kStages;
-        if (!mbar_wait(&bar->p_full[j & 1], (j >> 1) & 1, dev_status, abort_flag)) break;  // implies K/V tile j has landed
-        tc_fence_after();
-        const uint64_t vb = s == 0 ? v_desc[0] : s == 1 ? v_desc[1] : s == 2 ? v_desc[2] : v_desc[3];
-        const uint32_t t_p = tmem + C::kColS + (j & 1) * kBN;
+      bool ok = true;
+      int n = 0, pc = 0;
+      for (int it = it_begin; ok && it < it_end; ++pc) {
+        const Piece p = piece_at(it, it_end, nblk);
+        it += p.cnt;
+        for (int j = 0; j < p.cnt; ++j, ++n) {
+          const int s = n % C::kStages;
+          // P ready implies that the K/V tile has landed
+          if (!mbar_wait(&bar->p_full[n & 1], (n >> 1) & 1, dev_status, abort_flag)) { ok = false; break; }
+          // the first product of a piece overwrites the accumulator the previous epilogue reads
+          if (j == 0 && pc > 0 && !mbar_wait(&bar->o_free, (pc - 1) & 1, dev_status, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t vb = s == 0 ? v_desc[0] : s == 1 ? v_desc[1] : s == 2 ? v_desc[2] : v_desc[3];
+          const uint32_t t_p = tmem + C::kColS + (n & 1) * kBN;
 #pragma unroll
-        for (int kk = 0; kk < kBN / 16; ++kk) {  // 16 keys per MMA: 8 packed columns of P, 16 rows of V
-          mma_ts(t_o, t_p + kk * 8, vb + (uint64_t)((kk * 2048) >> 4), idesc_o, j > 0 || kk > 0);
+          for (int kk = 0; kk < kBN / 16; ++kk) {  // 16 keys per MMA: 8 packed columns of P, 16 rows of V
+            mma_ts(t_o, t_p + kk * 8, vb + (uint64_t)((kk * 2048) >> 4), idesc_o, j > 0 || kk > 0);
+          }
+          mma_commit(&bar->v_empty[s]);  // frees the K/V slot and tells everyone that this PV has landed
+          // One phase per piece: the next piece's products wait for o_free, which the epilogue gives
+          // only after it has seen this phase, so a waiter is never two phases behind.
+          if (j + 1 == p.cnt) mma_commit(&bar->o_done);
         }
-        mma_commit(&bar->v_empty[s]);  // frees the K/V slot and tells everyone that PV_j has landed
-        if (j + 1 == nblk) mma_commit(&bar->o_done);  // single-phase barrier: the epilogue cannot mistake an older phase for it
+      }
+    }
+  } else if (warp == 7) {
+    // ------------------------------------------------------------------ publisher
+    if (lane == 0) {
+      // When the span's first piece is partial and more pieces follow, make that piece
+      // visible to the other CTAs and draw its four tickets here, off the softmax warps' path.
+      const int u = it_begin / nblk;
+      const bool early = (it_begin > u * nblk || it_end < (u + 1) * nblk) && it_end > (u + 1) * nblk;
+      if (early && mbar_wait(&bar->pub_ready, 0, dev_status, abort_flag)) {
+        __threadfence();
+        uint32_t t[4];
+#pragma unroll
+        for (int w = 0; w < 4; ++w) t[w] = atomicAdd(&tickets[(size_t)u * 4 + w], 1u);
+#pragma unroll
+        for (int w = 0; w < 4; ++w) bar->first_ticket[w] = t[w];
+        mbar_arrive(&bar->pub_done);
       }
     }
   } else if (warp < 4) {
@@ -315,51 +632,34 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int row = warp * 32 + lane;  // query row inside the tile = tensor-memory lane
     const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
     const uint32_t ob = tmem + lane_addr + C::kColO;
-    float m_used = -INFINITY, l = 0.f;
     bool ok = true;
-    for (int j = 0; j < nblk; ++j) {
-      const uint32_t sb = tmem + lane_addr + C::kColS + (j & 1) * kBN;
-      if (!mbar_wait(&bar->s_full[j & 1], (j >> 1) & 1, dev_status, abort_flag)) { ok = false; break; }
-      tc_fence_after();
-      const int valid = L - j * kBN;  // keys of this tile inside the sequence (>= 64: all)
-      uint64_t* pvb = &bar->v_empty[(j + C::kStages - 1) % C::kStages];  // barrier PV_{j-1} commits to
-      const uint32_t pvp = (uint32_t)(((j - 1) / C::kStages) & 1);
-      if (valid >= kBN) ok = softmax_tile<DH, false>(sb, ob, scale_log2, kBN, j, m_used, l, pvb, pvp, dev_status, abort_flag);
-      else ok = softmax_tile<DH, true>(sb, ob, scale_log2, valid, j, m_used, l, pvb, pvp, dev_status, abort_flag);
+    int n = 0, pc = 0;
+    for (int it = it_begin; ok && it < it_end; ++pc) {
+      const Piece p = piece_at(it, it_end, nblk);
+      it += p.cnt;
+      float m_used = -INFINITY, l = 0.f;
+      // a partial last piece is normally the last contributor of its unit: look at the ticket now
+      // (acquire), so that the answer is there when the piece ends
+      uint32_t peek = 0;
+      if (it >= it_end && p.cnt < nblk) peek = ld_acquire_gpu(tickets + (size_t)p.u * 4 + warp);
+      for (int j = 0; j < p.cnt; ++j, ++n) {
+        const uint32_t sb = tmem + lane_addr + C::kColS + (n & 1) * kBN;
+        if (!mbar_wait(&bar->s_full[n & 1], (n >> 1) & 1, dev_status, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const int valid = L - (p.k0 + j) * kBN;  // keys of this tile inside the sequence (>= 64: all)
+        uint64_t* pvb = &bar->v_empty[(n + C::kStages - 1) % C::kStages];  // barrier the previous tile's PV commits to
+        const uint32_t pvp = (uint32_t)(((n - 1) / C::kStages) & 1);
+        if (valid >= kBN) ok = softmax_tile<DH, false>(sb, ob, scale_log2, kBN, j, m_used, l, pvb, pvp, dev_status, abort_flag);
+        else ok = softmax_tile<DH, true>(sb, ob, scale_log2, valid, j, m_used, l, pvb, pvp, dev_status, abort_flag);
+        if (!ok) break;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bar->p_full[n & 1]);
+      }
       if (!ok) break;
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bar->p_full[j & 1]);
+      ok = finish_piece<DH>(ob, bar, p, pc, it >= it_end, peek, row, m_used, l, o, L, heads, sp, tickets, pieces, dev_status);
     }
-    if (ok && mbar_wait(&bar->o_done, 0, dev_status, abort_flag)) {
-      tc_fence_after();
-      if (C::kSumMma) {
-        uint32_t rs[16];
-        tmem_ld16(ob + DH, rs);
-        tmem_wait_ld();
-        l = __uint_as_float(rs[0]);
-      }
-      const float inv = 1.f / l;
-      const int qi = q0 + row;
-      __nv_bfloat16* dst = o + ((size_t)b * L + (qi < L ? qi : 0)) * ((size_t)heads * DH) + (size_t)h * DH;
-#pragma unroll
-      for (int c = 0; c < DH / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(ob + c * 32, r);
-        tmem_wait_ld();
-        if (qi < L) {
-#pragma unroll
-          for (int e = 0; e < 32; e += 8) {
-            uint4 v;
-            v.x = pack_bf16_rn(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
-            v.y = pack_bf16_rn(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-            v.z = pack_bf16_rn(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-            v.w = pack_bf16_rn(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
-            *reinterpret_cast<uint4*>(dst + c * 32 + e) = v;
-          }
-        }
-      }
-    }
+    if (ok) settle_first_piece<DH>(bar, it_begin, it_end, row, o, L, heads, sp, pieces, dev_status);
   }
   tc_fence_before();
   __syncthreads();
@@ -369,9 +669,59 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   }
 }
 
+constexpr int kMaxCtas = 320;  // scratch is sized for this many persistent CTAs
+
+size_t ticket_bytes(int B, int L, int heads) {
+  const size_t units = (size_t)B * heads * ((L + kBM - 1) / kBM);
+  return (units * 4 * sizeof(uint32_t) + 255) & ~(size_t)255;
+}
+
+int max_ctas() {
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v < 1)
+      v = 148;
+    sms = v;
+  }
+  int G = 2 * sms < kMaxCtas ? 2 * sms : kMaxCtas;
+  if (const char* e = getenv("TOMA_ATTENTION_CTAS")) {  // tuning aid
+    const int v = atoi(e);
+    if (v >= 1 && v <= kMaxCtas) G = v;
+  }
+  return G;
+}
+
+// Key tiles a split costs a CTA, in units of one tile's time: writing, publishing and adding up the
+// partial results at the end of its span.
+constexpr int kSplitCostTiles = 5;
+
+// Whole units per CTA when that is at most kSplitCostTiles tiles slower than a perfectly even cut;
+// otherwise spans cut at single key tiles.
+Spans plan_spans(int units, int nblk) {
+  Spans sp;
+  sp.nblk = nblk;
+  sp.T = units * nblk;
+  const int gmax = max_ctas();
+  const int whole_tiles = ((units + gmax - 1) / gmax) * nblk;  // longest CTA with whole units
+  const int even_tiles = (sp.T + gmax - 1) / gmax;             // longest CTA with an even cut
+  int mode = whole_tiles <= even_tiles + kSplitCostTiles ? 0 : 1;
+  if (const char* e = getenv("TOMA_ATTENTION_SPLIT")) mode = atoi(e) != 0;  // tuning aid
+  if (mode == 0) {
+    sp.quantum = nblk;
+    sp.G = units < gmax ? units : gmax;
+  } else {
+    sp.quantum = 1;
+    sp.G = sp.T < gmax ? sp.T : gmax;
+  }
+  sp.q = sp.T / sp.quantum / sp.G;
+  sp.r = sp.T / sp.quantum - sp.q * sp.G;
+  return sp;
+}
+
 template <int DH>
-cudaError_t launch(int B, int L, int heads, const void* q, const void* k, const void* v, void* o, uint32_t* dev_status,
-                   cudaStream_t s) {
+cudaError_t launch(int B, int L, int heads, const void* q, const void* k, const void* v, void* o, void* ws,
+                   bool tickets_clean, uint32_t* dev_status, cudaStream_t s) {
   using C = AttCfg<DH>;
   CUtensorMap tq, tk, tv;
   const uint64_t dims[3] = {(uint64_t)heads * DH, (uint64_t)L, (uint64_t)B};
@@ -387,19 +737,35 @@ cudaError_t launch(int B, int L, int heads, const void* q, const void* k, const 
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  dim3 grid((L + kBM - 1) / kBM, heads, B);
+  const long long units = (long long)B * heads * ((L + kBM - 1) / kBM);
+  const int nblk = (L + kBN - 1) / kBN;
+  if (units * nblk > 0x7fffffffLL) return cudaErrorInvalidValue;  // iteration indices are 32-bit
+  const Spans sp = plan_spans((int)units, nblk);
+  const size_t tb = ticket_bytes(B, L, heads);
+  if (sp.quantum == 1 && !tickets_clean) {  // units are split: their tickets start at zero
+    cudaError_t e = cudaMemsetAsync(ws, 0, tb, s);
+    if (e != cudaSuccess) return e;
+  }
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  attention_tc_kernel<DH><<<grid, 224, C::kSmemBytes, s>>>(tq, tk, tv, (__nv_bfloat16*)o, L, heads, scale_log2, dev_status);
+  attention_tc_kernel<DH><<<sp.G, 256, C::kSmemBytes, s>>>(tq, tk, tv, (__nv_bfloat16*)o, L, heads, scale_log2, sp,
+                                                           (uint32_t*)ws, (float*)((char*)ws + tb), dev_status);
   count_launch();
   return cudaGetLastError();
 }
 
 }  // namespace
 
+size_t attention_tc_workspace_bytes(int B, int L, int heads, int dh) {
+  const size_t piece = (dh == 64 ? piece_floats<64>() : piece_floats<128>()) * sizeof(float);
+  return ticket_bytes(B, L, heads) + 2 * (size_t)kMaxCtas * piece;
+}
+
+size_t attention_tc_ticket_bytes(int B, int L, int heads) { return ticket_bytes(B, L, heads); }
+
 cudaError_t launch_attention_tc(int B, int L, int heads, int dh, const void* q, const void* k, const void* v, void* o,
-                                uint32_t* dev_status, cudaStream_t s) {
-  if (dh == 64) return launch<64>(B, L, heads, q, k, v, o, dev_status, s);
-  if (dh == 128) return launch<128>(B, L, heads, q, k, v, o, dev_status, s);
+                                void* ws, bool tickets_clean, uint32_t* dev_status, cudaStream_t s) {
+  if (dh == 64) return launch<64>(B, L, heads, q, k, v, o, ws, tickets_clean, dev_status, s);
+  if (dh == 128) return launch<128>(B, L, heads, q, k, v, o, ws, tickets_clean, dev_status, s);
   return cudaErrorInvalidValue;
 }
 

@@ -32,7 +32,7 @@ toma_status make_geom(const toma_desc* desc, Geom* g);
 
 // Workspace carve-up (all offsets 256-byte aligned).
 struct WsLayout {
-  size_t y_off, sq_off, logits_off, wts_off, xm_off, att_off, total;
+  size_t y_off, sq_off, logits_off, wts_off, xm_off, att_off, att_ws_off, total;
 };
 WsLayout ws_layout(const Geom& g);
 
@@ -57,12 +57,20 @@ size_t weights_tc_scratch_bytes(const Geom& g);
 cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, void* w, float* shares, void* scratch,
                               uint32_t* dev_status, cudaStream_t s);
 bool linear_tc_supported(const Geom& g);
-cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* xm, uint32_t* dev_status, cudaStream_t s);
+// `zero` / `zero_bytes` (multiple of 4, may be 0): a region the kernel clears on the side.
+cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* xm, void* zero, size_t zero_bytes,
+                            uint32_t* dev_status, cudaStream_t s);
 cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void* out, uint32_t* dev_status,
                               cudaStream_t s);
 cudaError_t launch_copy_extra(const Geom& g, const void* src, void* dst, bool merging, cudaStream_t s);
+// Scratch of the tensor-core attention (tickets and partial results of split work units).
+size_t attention_tc_workspace_bytes(int B, int L, int heads, int dh);
+// The scratch starts with the tickets (attention_tc_ticket_bytes()), which must be zero when the
+// kernel starts: the launcher clears them unless `tickets_clean` says an earlier kernel on the
+// stream already did.
+size_t attention_tc_ticket_bytes(int B, int L, int heads);
 cudaError_t launch_attention_tc(int B, int L, int heads, int dh, const void* q, const void* k, const void* v, void* o,
-                                uint32_t* dev_status, cudaStream_t s);
+                                void* ws, bool tickets_clean, uint32_t* dev_status, cudaStream_t s);
 cudaError_t launch_weights_export(const Geom& g, const void* w, float* dense, cudaStream_t s);
 cudaError_t launch_weights_import(const Geom& g, const float* dense, void* w, cudaStream_t s);
 

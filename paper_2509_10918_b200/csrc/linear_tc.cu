@@ -34,6 +34,8 @@ struct PipeBars {
 struct LinParams {
   int P, tiles_x, th, tw, W, Nloc, Dloc, d, n_all, Lm;
   int stages;  // pipeline depth
+  uint32_t* zero;  // merge only: words cleared on the side (the attention kernel's tickets)
+  int zero_words;
 };
 
 __device__ __forceinline__ uint32_t tmem_cols_for(int n) { return n > 128 ? 256u : n > 64 ? 128u : 64u; }
@@ -71,6 +73,11 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
 
   if (threadIdx.x == 0) pipe_init(bar, p.stages);
   if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
+  if (p.zero_words > 0) {
+    const int cta = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+    const int n_thr = gridDim.x * gridDim.y * gridDim.z * blockDim.x;
+    for (int i = cta * blockDim.x + threadIdx.x; i < p.zero_words; i += n_thr) p.zero[i] = 0u;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -235,6 +242,7 @@ LinParams make_params(const Geom& g) {
   LinParams p;
   p.P = g.P; p.tiles_x = g.tiles_x; p.th = g.th; p.tw = g.tw; p.W = g.W; p.Nloc = g.Nloc; p.Dloc = g.Dloc;
   p.d = g.d; p.n_all = (int)g.tokens_all(); p.Lm = g.Lm; p.stages = 2;
+  p.zero = nullptr; p.zero_words = 0;
   return p;
 }
 
@@ -264,8 +272,8 @@ bool linear_tc_supported(const Geom& g) {
   return true;
 }
 
-cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* xm, uint32_t* dev_status,
-                            cudaStream_t s) {
+cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* xm, void* zero, size_t zero_bytes,
+                            uint32_t* dev_status, cudaStream_t s) {
   CUtensorMap tx, tw;
   const uint64_t dims[4] = {(uint64_t)g.d, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.B};
   const uint64_t strides[3] = {(uint64_t)g.d * 2, (uint64_t)g.W * g.d * 2, (uint64_t)g.tokens_all() * g.d * 2};
@@ -274,6 +282,8 @@ cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* x
   LinParams p = make_params(g);
   const int slabs = ((g.Dloc < kMaxCols ? g.Dloc : kMaxCols) + 63) / 64;
   const int stage_bytes = (2 + 2 * slabs) * kSlab;
+  p.zero = (uint32_t*)zero;
+  p.zero_words = (int)(zero_bytes / 4);
   p.stages = 2;  // two stages keep a CTA below ~100 KB so that two or three CTAs share an SM and hide each other's latencies
   if (p.stages > g.Nloc / kKC) p.stages = g.Nloc / kKC;
   const int smem = 1024 + p.stages * stage_bytes + 256;

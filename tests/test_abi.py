@@ -73,8 +73,8 @@ def test_null_and_workspace_errors_are_returned_before_any_launch(toma):
     assert lib.toma_select(ctypes.byref(d), fake, fake, None, 0, None, None) == WS
     assert lib.toma_select(ctypes.byref(d), fake, fake, fake, 16, None, None) == WS
     assert lib.toma_merge(ctypes.byref(d), None, fake, fake, None, None) == NULL
-    assert lib.toma_attention(1, 0, 1, 64, 0, fake, fake, fake, fake, None, None) == 2
-    assert lib.toma_attention(1, 8, 1, 48, 0, fake, fake, fake, fake, None, None) == 7
+    assert lib.toma_attention(1, 0, 1, 64, 0, fake, fake, fake, fake, None, 0, None, None) == 2
+    assert lib.toma_attention(1, 8, 1, 48, 0, fake, fake, fake, fake, None, 0, None, None) == 7
 
 
 def test_binding_refuses_cpu_tensors(toma):
