@@ -263,8 +263,9 @@ __device__ __forceinline__ const float* slot_of(const float* pieces, const Spans
 
 // Adds up the pieces of one query row of unit u, left by CTAs g_first..g_last:
 //   O = sum_i 2^(m_i - M) O_i / sum_i 2^(m_i - M) l_i,  M = max_i m_i  (m in the log2 domain).
-// Contributors are taken two at a time so that their loads are in flight together (the usual unit
-// has two).  Loads bypass L1: the pieces were written by other SMs during this launch.
+// Contributors are taken two at a time so that their loads are in flight together, and summed in
+// ascending CTA order with one fused multiply-add each, starting from zero: finish_piece's direct
+// path follows the same order, so the result does not depend on which path a launch takes.  Loads bypass L1: the pieces were written by other SMs during this launch.
 template <int DH>
 __device__ __noinline__ void combine_rows(const float* pieces, Spans sp, int u, int g_first, int g_last, int row,
                                           __nv_bfloat16* dst) {
@@ -287,7 +288,7 @@ __device__ __noinline__ void combine_rows(const float* pieces, Spans sp, int u, 
       const float ma = __ldcg(sa + kM + row), la = __ldcg(sa + kL + row);
       const float mb = __ldcg(sb + kM + row), lb = __ldcg(sb + kL + row);
       const float wa = ex2_mufu(ma - M), wb = g < g_last ? ex2_mufu(mb - M) : 0.f;
-      denom += wa * la + wb * lb;
+      denom = fmaf(wb, lb, fmaf(wa, la, denom));
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         float4 va[8], vb[8];
@@ -299,10 +300,10 @@ __device__ __noinline__ void combine_rows(const float* pieces, Spans sp, int u, 
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
           float* a4 = &acc[c * 32 + 4 * q];
-          a4[0] = fmaf(wa, va[q].x, fmaf(wb, vb[q].x, a4[0]));
-          a4[1] = fmaf(wa, va[q].y, fmaf(wb, vb[q].y, a4[1]));
-          a4[2] = fmaf(wa, va[q].z, fmaf(wb, vb[q].z, a4[2]));
-          a4[3] = fmaf(wa, va[q].w, fmaf(wb, vb[q].w, a4[3]));
+          a4[0] = fmaf(wb, vb[q].x, fmaf(wa, va[q].x, a4[0]));
+          a4[1] = fmaf(wb, vb[q].y, fmaf(wa, va[q].y, a4[1]));
+          a4[2] = fmaf(wb, vb[q].z, fmaf(wa, va[q].z, a4[2]));
+          a4[3] = fmaf(wb, vb[q].w, fmaf(wa, va[q].w, a4[3]));
         }
       }
     }
@@ -357,7 +358,7 @@ __device__ __noinline__ bool finish_piece(uint32_t ob, Barriers* bar, Piece p, i
   const bool whole = p.cnt == sp.nblk;
   uint32_t* ticket = tickets + (size_t)p.u * 4 + warp;
   int g_first = 0, g_last = 0;
-  bool direct = false;
+  bool direct = false, own_first = false;  // own_first: this CTA is the lower of the two contributors
   const float* other = nullptr;
   float m_o = 0.f, l_o = 0.f;
   float4 vo[16];
@@ -366,6 +367,7 @@ __device__ __noinline__ bool finish_piece(uint32_t ob, Barriers* bar, Piece p, i
     g_last = sp.owner((p.u + 1) * sp.nblk - 1);
     if (last_of_span && g_last == g_first + 1 && peek == 1u) {
       direct = true;
+      own_first = (int)blockIdx.x == g_first;
       other = slot_of<DH>(pieces, sp, (int)blockIdx.x == g_first ? g_last : g_first, p.u);
       m_o = __ldcg(other + kM + row);
       l_o = __ldcg(other + kL + row);
@@ -388,7 +390,7 @@ __device__ __noinline__ bool finish_piece(uint32_t ob, Barriers* bar, Piece p, i
     const float M = fmaxf(m_used, m_o);
     w_own = ex2_mufu(m_used - M);
     w_o = ex2_mufu(m_o - M);
-    inv = 1.f / (w_own * l + w_o * l_o);
+    inv = 1.f / (own_first ? fmaf(w_o, l_o, w_own * l) : fmaf(w_own, l, w_o * l_o));
   }
 #pragma unroll
   for (int c = 0; c < DH / 32; ++c) {
@@ -405,10 +407,12 @@ __device__ __noinline__ bool finish_piece(uint32_t ob, Barriers* bar, Piece p, i
 #pragma unroll
       for (int q = 0; q < 8; ++q) {
         const float4 v = vo[(c & 1) * 8 + q];
-        r[4 * q] = __float_as_uint(fmaf(w_own, __uint_as_float(r[4 * q]), w_o * v.x));
-        r[4 * q + 1] = __float_as_uint(fmaf(w_own, __uint_as_float(r[4 * q + 1]), w_o * v.y));
-        r[4 * q + 2] = __float_as_uint(fmaf(w_own, __uint_as_float(r[4 * q + 2]), w_o * v.z));
-        r[4 * q + 3] = __float_as_uint(fmaf(w_own, __uint_as_float(r[4 * q + 3]), w_o * v.w));
+        const float vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float own = __uint_as_float(r[4 * q + e]);
+          r[4 * q + e] = __float_as_uint(own_first ? fmaf(w_o, vv[e], w_own * own) : fmaf(w_own, own, w_o * vv[e]));
+        }
       }
       if (dst) store_row32(dst + c * 32, r, inv);
     } else {
@@ -494,6 +498,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     for (int e = threadIdx.x; e < C::kOnesBytes / 4; e += blockDim.x) reinterpret_cast<uint32_t*>(sOnes)[e] = 0x3F803F80u;
     fence_proxy_async();
   }
+  dependency_wait();
+  if (threadIdx.x == 0) release_dependents();
   if (warp == 5) tmem_alloc(&bar->tmem_base, C::kTmemCols);
   tc_fence_before();
   __syncthreads();
@@ -747,8 +753,10 @@ cudaError_t launch(int B, int L, int heads, const void* q, const void* k, const 
     if (e != cudaSuccess) return e;
   }
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  attention_tc_kernel<DH><<<sp.G, 256, C::kSmemBytes, s>>>(tq, tk, tv, (__nv_bfloat16*)o, L, heads, scale_log2, sp,
-                                                           (uint32_t*)ws, (float*)((char*)ws + tb), dev_status);
+  cudaError_t e = launch_dependent(attention_tc_kernel<DH>, dim3(sp.G), dim3(256), (size_t)C::kSmemBytes, s, tq, tk, tv,
+                                   (__nv_bfloat16*)o, L, heads, scale_log2, sp, (uint32_t*)ws, (float*)((char*)ws + tb),
+                                   dev_status);
+  if (e != cudaSuccess) return e;
   count_launch();
   return cudaGetLastError();
 }

@@ -27,6 +27,7 @@ constexpr int kUnmergeTok = 128;  // tokens per unmerge CTA: small enough that t
 
 struct PipeBars {
   uint64_t full[4], empty[4], done;
+  uint64_t epi;  // the four epilogue warps have staged their part of the output tile
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -34,6 +35,7 @@ struct PipeBars {
 struct LinParams {
   int P, tiles_x, th, tw, W, Nloc, Dloc, d, n_all, Lm;
   int stages;  // pipeline depth
+  int out_rows;  // rows of one 64-channel slab of the staged output tile (= the output tensor map's box)
   uint32_t* zero;  // merge only: words cleared on the side (the attention kernel's tickets)
   int zero_words;
 };
@@ -46,8 +48,39 @@ __device__ __forceinline__ void pipe_init(PipeBars* bar, int stages) {
     mbar_init(&bar->empty[s], 1);
   }
   mbar_init(&bar->done, 1);
+  mbar_init(&bar->epi, 4);
   bar->abort_flag = 0;
   mbar_fence_init();
+}
+
+// Epilogue shared by both kernels.  Thread = channel `cl` (0..127) of the CTA's chunk, holding in
+// tensor memory one fp32 per output row.  The tile is staged in shared memory as two 64-channel
+// slabs of [rows][128 B], 128-byte swizzled, i.e. the layout of the output tensor map's box, and
+// leaves with one TMA store per slab (whole lines, asynchronous) issued by `store`.
+template <typename Store>
+__device__ __forceinline__ void stage_and_store(uint8_t* so, PipeBars* bar, uint32_t taddr, int cl, int n_rows, int slab_rows,
+                                                uint32_t* dev_status, Store store) {
+  uint8_t* mine = so + (cl >> 6) * slab_rows * 128 + (cl & 7) * 2;
+  const int chunk = (cl & 63) >> 3;
+  for (int i0 = 0; i0 < n_rows; i0 += 32) {
+    uint32_t r[32];
+    tmem_ld32(taddr + i0, r);
+    tmem_wait_ld();
+#pragma unroll
+    for (int e = 0; e < 32; ++e) {
+      const int row = i0 + e;
+      if (row < n_rows)
+        *reinterpret_cast<__nv_bfloat16*>(mine + row * 128 + ((chunk ^ (row & 7)) << 4)) = __float2bfloat16_rn(__uint_as_float(r[e]));
+    }
+  }
+  fence_proxy_async();  // the staged tile is read by the TMA engine
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) mbar_arrive(&bar->epi);
+  if (cl == 0 && mbar_wait(&bar->epi, 0, dev_status, &bar->abort_flag)) {
+    store();
+    tma_store_commit();
+    tma_store_wait_read();  // shared memory must outlive the engine's reads
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -55,7 +88,7 @@ __device__ __forceinline__ void pipe_init(PipeBars* bar, int stages) {
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(192, 1)
 merge_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
-                __nv_bfloat16* __restrict__ xm, const LinParams p, uint32_t* dev_status) {
+                const __grid_constant__ CUtensorMap tm_o, const LinParams p, uint32_t* dev_status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -72,6 +105,8 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
   const uint32_t ncols = tmem_cols_for(n_mma);
 
   if (threadIdx.x == 0) pipe_init(bar, p.stages);
+  dependency_wait();
+  if (threadIdx.x == 0) release_dependents();
   if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
   if (p.zero_words > 0) {
     const int cta = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
@@ -121,22 +156,14 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
       if (ok) mma_commit(&bar->done);
     }
   } else {
-    const int quarter = warp & 3;
-    const int ch = c0 + quarter * 32 + lane;
+    const int quarter = warp & 3, cl = quarter * 32 + lane;
     const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16);
-    if (mbar_wait(&bar->done, 0, dev_status, abort_flag)) {
+    if (mbar_wait(&bar->done, 0, dev_status, abort_flag)) {  // every load has been consumed: the stages are free
       tc_fence_after();
-      __nv_bfloat16* dst = xm + ((size_t)b * p.Lm + (size_t)tile * p.Dloc + i_base) * p.d + ch;
-      for (int i0 = 0; i0 < n_dest; i0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(taddr + i0, r);
-        tmem_wait_ld();
-        if (ch < p.d) {
-#pragma unroll
-          for (int e = 0; e < 32; ++e)
-            if (i0 + e < n_dest) dst[(size_t)(i0 + e) * p.d] = __float2bfloat16_rn(__uint_as_float(r[e]));
-        }
-      }
+      stage_and_store(smem, bar, taddr, cl, n_dest, p.out_rows, dev_status, [&] {
+        for (int c = 0; c < 2; ++c)
+          if (c0 + c * 64 < p.d) tma_store_4d(&tm_o, smem + c * p.out_rows * 128, c0 + c * 64, i_base, tile, b);
+      });
     }
   }
   tc_fence_before();
@@ -152,7 +179,7 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(192, 1)
 unmerge_tc_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_w,
-                  __nv_bfloat16* __restrict__ out, const LinParams p, int n_tok, uint32_t* dev_status) {
+                  const __grid_constant__ CUtensorMap tm_o, const LinParams p, int n_tok, uint32_t* dev_status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int w_plane = n_tok * 128;  // bytes of one [n_tok tokens][64 destinations] weight block
@@ -165,6 +192,8 @@ unmerge_tc_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constan
   const uint32_t ncols = tmem_cols_for(n_tok);
 
   if (threadIdx.x == 0) pipe_init(bar, p.stages);
+  dependency_wait();
+  if (threadIdx.x == 0) release_dependents();
   if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
   tc_fence_before();
   __syncthreads();
@@ -207,27 +236,17 @@ unmerge_tc_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constan
       if (ok) mma_commit(&bar->done);
     }
   } else {
-    const int quarter = warp & 3;
-    const int ch = c0 + quarter * 32 + lane;
+    const int quarter = warp & 3, cl = quarter * 32 + lane;
     const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16);
     if (mbar_wait(&bar->done, 0, dev_status, abort_flag)) {
       tc_fence_after();
-      __nv_bfloat16* base = out + (size_t)b * p.n_all * p.d + ch;
-      for (int l0 = 0; l0 < n_tok; l0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(taddr + l0, r);
-        tmem_wait_ld();
-        if (ch < p.d) {
-          // token of local slot l0 (one division per 32 slots), then walk the tile row by row
-          int lx = (t0 + l0) % p.tw;
-          size_t tok = (size_t)tile_token(tile, t0 + l0, p.tiles_x, p.th, p.tw, p.W);
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            base[tok * p.d] = __float2bfloat16_rn(__uint_as_float(r[e]));
-            if (++lx == p.tw) { lx = 0; tok += (size_t)(p.W - p.tw + 1); } else { ++tok; }
-          }
-        }
-      }
+      // rows of the staged tile = the CTA's token slots in tile order = the (x, y) box of the output map
+      const int ty = tile / p.tiles_x, tx = tile - ty * p.tiles_x;
+      stage_and_store(smem, bar, taddr, cl, n_tok, n_tok, dev_status, [&] {
+        for (int c = 0; c < 2; ++c)
+          if (c0 + c * 64 < p.d)
+            tma_store_4d(&tm_o, smem + c * n_tok * 128, c0 + c * 64, tx * p.tw, ty * p.th + t0 / p.tw, b);
+      });
     }
   }
   tc_fence_before();
@@ -242,7 +261,7 @@ LinParams make_params(const Geom& g) {
   LinParams p;
   p.P = g.P; p.tiles_x = g.tiles_x; p.th = g.th; p.tw = g.tw; p.W = g.W; p.Nloc = g.Nloc; p.Dloc = g.Dloc;
   p.d = g.d; p.n_all = (int)g.tokens_all(); p.Lm = g.Lm; p.stages = 2;
-  p.zero = nullptr; p.zero_words = 0;
+  p.zero = nullptr; p.zero_words = 0; p.out_rows = 0;
   return p;
 }
 
@@ -280,6 +299,13 @@ cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* x
   const uint32_t box[4] = {64, (uint32_t)g.tw, (uint32_t)(64 / g.tw), 1};
   if (!encode_tmap_16bit(&tx, x, 4, dims, strides, box) || !encode_w(g, w, &tw, 64)) return cudaErrorInvalidValue;
   LinParams p = make_params(g);
+  // merged rows as (channel, destination, tile, batch): a store that runs past a tile's D_loc rows is clipped
+  CUtensorMap to;
+  p.out_rows = g.Dloc < kMaxCols ? g.Dloc : kMaxCols;
+  const uint64_t odims[4] = {(uint64_t)g.d, (uint64_t)g.Dloc, (uint64_t)g.P, (uint64_t)g.B};
+  const uint64_t ostrides[3] = {(uint64_t)g.d * 2, (uint64_t)g.Dloc * g.d * 2, (uint64_t)g.Lm * g.d * 2};
+  const uint32_t obox[4] = {64, (uint32_t)p.out_rows, 1, 1};
+  if (!encode_tmap_16bit(&to, xm, 4, odims, ostrides, obox)) return cudaErrorInvalidValue;
   const int slabs = ((g.Dloc < kMaxCols ? g.Dloc : kMaxCols) + 63) / 64;
   const int stage_bytes = (2 + 2 * slabs) * kSlab;
   p.zero = (uint32_t*)zero;
@@ -291,9 +317,9 @@ cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* x
   cudaError_t e = raise_smem_limit((const void*)merge_tc_kernel, &attr);
   if (e != cudaSuccess) return e;
   dim3 grid(g.B * g.P, (g.d + 127) / 128, (g.Dloc + kMaxCols - 1) / kMaxCols);
-  merge_tc_kernel<<<grid, 192, smem, s>>>(tx, tw, (__nv_bfloat16*)xm, p, dev_status);
+  e = launch_dependent(merge_tc_kernel, grid, dim3(192), (size_t)smem, s, tx, tw, to, p, dev_status);
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void* out, uint32_t* dev_status,
@@ -306,6 +332,12 @@ cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void*
   if (!encode_tmap_16bit(&ty, y, 3, dims, strides, box) || !encode_w(g, w, &tw, (uint32_t)n_tok))
     return cudaErrorInvalidValue;
   LinParams p = make_params(g);
+  // output tokens as (channel, x, y, batch): a CTA's token block is n_tok / tile_w whole tile rows
+  CUtensorMap to;
+  const uint64_t odims[4] = {(uint64_t)g.d, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.B};
+  const uint64_t ostrides[3] = {(uint64_t)g.d * 2, (uint64_t)g.W * g.d * 2, (uint64_t)g.tokens_all() * g.d * 2};
+  const uint32_t obox[4] = {64, (uint32_t)g.tw, (uint32_t)(n_tok / g.tw), 1};
+  if (!encode_tmap_16bit(&to, out, 4, odims, ostrides, obox)) return cudaErrorInvalidValue;
   const int stage_bytes = 2 * kSlab + 2 * n_tok * 128;
   p.stages = 2;
   if (p.stages > (g.Dloc + kKC - 1) / kKC) p.stages = (g.Dloc + kKC - 1) / kKC;
@@ -314,9 +346,9 @@ cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void*
   cudaError_t e = raise_smem_limit((const void*)unmerge_tc_kernel, &attr);
   if (e != cudaSuccess) return e;
   dim3 grid(g.B * g.P, (g.d + 127) / 128, g.Nloc / n_tok);
-  unmerge_tc_kernel<<<grid, 192, smem, s>>>(ty, tw, (__nv_bfloat16*)out, p, n_tok, dev_status);
+  e = launch_dependent(unmerge_tc_kernel, grid, dim3(192), (size_t)smem, s, ty, tw, to, p, n_tok, dev_status);
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace toma

@@ -7,6 +7,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
 
 namespace toma {
 namespace tc {
@@ -173,6 +174,15 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with launch_dependent() may start while the previous kernel of the stream is
+// still running.  Until dependency_wait() returns (the previous kernel has completed and its
+// writes are visible) it must not touch global memory, and -- so that a waiting CTA cannot starve a
+// CTA of the previous kernel -- it must not hold tensor memory.  release_dependents() lets the
+// next kernel's CTAs be scheduled as this kernel's CTAs retire.
+__device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- descriptors
 // Shared-memory matrix descriptor, 128-byte swizzle, 16-bit elements.
 //   K-major operand  (rows = M or N, 64 K-elements = 128 B per row): SBO = bytes between 8-row groups.
@@ -210,6 +220,22 @@ __device__ __forceinline__ uint32_t sw128_offset(int row, int chunk) {
 // Encodes a bf16/fp16 tiled tensor map with 128-byte swizzle through the driver entry point
 // obtained from the runtime (the library does not link libcuda).  dims/strides innermost first;
 // strides[i] is the byte stride of dimension i+1.
+// Launch with programmatic stream serialisation: the kernel must call tc::dependency_wait().
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 bool encode_tmap_16bit(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
                        const uint32_t* box);
 

@@ -161,6 +161,35 @@ def test_attention_parity(toma, dtype, B, L, h, dh, n_rows):
         assert_close(got[b] if rows is None else got[b][rows], want, dtype, f"attention b={b}")
 
 
+@pytest.mark.parametrize("split,ctas,B,L,h,dh", [
+    ("1", "7", 1, 1000, 3, 64),     # spans run over several units: partial first piece, whole middle ones, partial last
+    ("1", "320", 1, 300, 3, 64),    # one key tile per CTA: five contributors per unit, all through scratch
+    ("1", "37", 2, 700, 2, 128),    # head_dim 128, ragged, units cut in two or three
+    ("1", "2", 1, 640, 1, 64),      # two CTAs share the middle unit
+    ("0", "5", 1, 1000, 3, 64),     # whole units, several per CTA
+    ("0", "320", 1, 300, 3, 128),   # whole units, fewer units than CTAs
+])
+def test_attention_span_plans(toma, monkeypatch, split, ctas, B, L, h, dh):
+    """The tensor-core kernel under forced work plans (the tuning knobs TOMA_ATTENTION_SPLIT and
+    TOMA_ATTENTION_CTAS): every way a unit's keys can be cut across CTAs gives the same result."""
+    monkeypatch.setenv("TOMA_ATTENTION_SPLIT", split)
+    monkeypatch.setenv("TOMA_ATTENTION_CTAS", ctas)
+    host = [gen.round_to_dtype(gen.normal(0, (78, L + dh, i), B * L * h * dh).reshape(B, L, h * dh).astype(np.float32),
+                               "bf16") for i in range(3)]
+    q, k, v = (to_dev(a, "bf16") for a in host)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    outs = []
+    for _ in range(2):  # twice: the second launch finds the scratch as the first left it
+        o = torch.full_like(q, float("nan"))
+        toma.toma_attention(B, L, h, dh, "bf16", q, k, v, o, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        outs.append(to_host64(o))
+    assert np.array_equal(outs[0], outs[1])
+    for b in range(B):
+        assert_close(outs[0][b], O.attention(host[0][b], host[1][b], host[2][b], h), "bf16", f"attention b={b}")
+
+
 @pytest.mark.parametrize("dh,L", [(64, 1536), (128, 1000)])
 def test_attention_growing_logits_exercise_the_rescale_path(toma, dh, L):
     """Keys grow along the sequence so that the row maximum rises by far more than the kernel's
