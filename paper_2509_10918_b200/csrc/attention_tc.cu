@@ -498,6 +498,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     for (int e = threadIdx.x; e < C::kOnesBytes / 4; e += blockDim.x) reinterpret_cast<uint32_t*>(sOnes)[e] = 0x3F803F80u;
     fence_proxy_async();
   }
+  if (threadIdx.x == 128) {  // descriptor fetches overlap the previous kernel's tail
+    prefetch_tmap(&tm_q);
+    prefetch_tmap(&tm_k);
+    prefetch_tmap(&tm_v);
+  }
   dependency_wait();
   if (threadIdx.x == 0) release_dependents();
   if (warp == 5) tmem_alloc(&bar->tmem_base, C::kTmemCols);
@@ -510,9 +515,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   if (warp == 4) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      prefetch_tmap(&tm_q);
-      prefetch_tmap(&tm_k);
-      prefetch_tmap(&tm_v);
       bool ok = true;
       int n = 0, pc = 0;
       for (int it = it_begin; ok && it < it_end; ++pc) {

@@ -104,7 +104,12 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
   const int nk = p.Nloc / kKC;
   const uint32_t ncols = tmem_cols_for(n_mma);
 
-  if (threadIdx.x == 0) pipe_init(bar, p.stages);
+  if (threadIdx.x == 0) {
+    pipe_init(bar, p.stages);
+    prefetch_tmap(&tm_x);
+    prefetch_tmap(&tm_w);
+    prefetch_tmap(&tm_o);
+  }
   dependency_wait();
   if (threadIdx.x == 0) release_dependents();
   if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
@@ -121,8 +126,6 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
 
   if (warp == 0) {
     if (lane == 0) {
-      prefetch_tmap(&tm_x);
-      prefetch_tmap(&tm_w);
       for (int k = 0; k < nk; ++k) {
         const int s = k % p.stages;
         if (k >= p.stages && !mbar_wait(&bar->empty[s], ((k / p.stages) - 1) & 1, dev_status, abort_flag)) break;
@@ -191,7 +194,12 @@ unmerge_tc_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constan
   const int nk = (p.Dloc + kKC - 1) / kKC;
   const uint32_t ncols = tmem_cols_for(n_tok);
 
-  if (threadIdx.x == 0) pipe_init(bar, p.stages);
+  if (threadIdx.x == 0) {
+    pipe_init(bar, p.stages);
+    prefetch_tmap(&tm_y);
+    prefetch_tmap(&tm_w);
+    prefetch_tmap(&tm_o);
+  }
   dependency_wait();
   if (threadIdx.x == 0) release_dependents();
   if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
@@ -203,8 +211,6 @@ unmerge_tc_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constan
 
   if (warp == 0) {
     if (lane == 0) {
-      prefetch_tmap(&tm_y);
-      prefetch_tmap(&tm_w);
       for (int k = 0; k < nk; ++k) {
         const int s = k % p.stages;
         if (k >= p.stages && !mbar_wait(&bar->empty[s], ((k / p.stages) - 1) & 1, dev_status, abort_flag)) break;
