@@ -66,6 +66,8 @@ struct Barriers {
   uint64_t o_done, o_free;            // per piece: accumulator complete / epilogue has read it
   uint64_t pub_ready, pub_done;       // first partial piece: written by the softmax warps / published, tickets drawn
   uint32_t first_ticket[4];           // per softmax warp: ticket its first (partial) piece drew
+  uint32_t others_done;               // set by the publisher when the span's last unit has all its other pieces in scratch
+  uint32_t poll_stop;                 // set by softmax warp 0 when the answer is no longer needed
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -325,6 +327,15 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p) {
   return v;
 }
 
+__device__ __forceinline__ void st_release_cta(uint32_t* smem_word, uint32_t v) {
+  asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(smem_u32(smem_word)), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_acquire_cta(const uint32_t* smem_word) {
+  uint32_t v;
+  asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(smem_word)) : "memory");
+  return v;
+}
+
 // Publishes this warp's 32 rows of a piece and takes the (unit, warp) ticket.  Returns the number
 // of contributors that had taken it before.
 __device__ __forceinline__ uint32_t take_ticket(uint32_t* ticket, int lane) {
@@ -335,8 +346,37 @@ __device__ __forceinline__ uint32_t take_ticket(uint32_t* ticket, int lane) {
   return __shfl_sync(0xffffffffu, t, 0);
 }
 
-// End of a piece, run by the softmax warps; waits for the piece's accumulator to be complete, then
-//   - a piece that covers all keys of its unit is normalised and written out;
+// End of a piece that covers all keys of its unit (the only kind when units are kept whole), run by
+// the softmax warps: wait for the accumulator, normalise, write the rows out.  Returns false when
+// the wait ran out.
+template <int DH>
+__device__ __forceinline__ bool finish_whole(uint32_t ob, Barriers* bar, int pos, int pc, int row, float l, __nv_bfloat16* o,
+                                             int L, int heads, uint32_t* dev_status) {
+  using C = AttCfg<DH>;
+  if (!mbar_wait(&bar->o_done, pc & 1, dev_status, &bar->abort_flag)) return false;
+  tc_fence_after();
+  if (C::kSumMma) {
+    uint32_t rs[16];
+    tmem_ld16(ob + DH, rs);
+    tmem_wait_ld();
+    l = __uint_as_float(rs[0]);
+  }
+  __nv_bfloat16* dst = out_row<DH>(o, pos, row, L, heads);
+  const float inv = 1.f / l;
+#pragma unroll
+  for (int c = 0; c < DH / 32; ++c) {
+    uint32_t r[32];
+    tmem_ld32(ob + c * 32, r);
+    tmem_wait_ld();
+    if (dst) store_row32(dst + c * 32, r, inv);
+  }
+  tc_fence_before();
+  __syncwarp();
+  if ((row & 31) == 0) mbar_arrive(&bar->o_free);  // the next piece's first PV product may overwrite the accumulator
+  return true;
+}
+
+// End of a piece that covers only part of its unit's keys, run by the softmax warps:
 //   - the last piece of the CTA's span, when the unit's only other contributor has already
 //     published (it ran at the start of its own span, so it normally has), is added to that
 //     contributor's piece straight from tensor memory and written out: nothing of it goes through
@@ -345,35 +385,32 @@ __device__ __forceinline__ uint32_t take_ticket(uint32_t* ticket, int lane) {
 //     ticket is drawn; the warp that draws a unit's last ticket adds its pieces up.  A last piece
 //     does that here; a first piece, with more of the span to come, hands the fence and the
 //     tickets' round trips to the publisher thread and looks at the outcome in settle_first_piece.
-// `peek` is the ticket as read (with acquire) when the piece began.
-// Kept out of line so that its registers do not weigh on the softmax loop.  Returns false when the
-// wait ran out.
+// Out of line (it runs at most twice per CTA and is register-hungry).  Returns false when the wait
+// ran out.
 template <int DH>
-__device__ __noinline__ bool finish_piece(uint32_t ob, Barriers* bar, Piece p, int pc, bool last_of_span, uint32_t peek,
-                                          int row, float m_used, float l, __nv_bfloat16* o, int L, int heads, Spans sp,
-                                          uint32_t* tickets, float* pieces, uint32_t* dev_status) {
+__device__ __noinline__ bool finish_partial(uint32_t ob, Barriers* bar, Piece p, int pc, bool last_of_span, int row,
+                                            float m_used, float l, __nv_bfloat16* o, int L, int heads, Spans sp,
+                                            uint32_t* tickets, float* pieces, uint32_t* dev_status) {
   using C = AttCfg<DH>;
   constexpr size_t kM = (size_t)kBM * DH, kL = (size_t)kBM * DH + kBM;
   const int warp = row >> 5, lane = row & 31;
-  const bool whole = p.cnt == sp.nblk;
   uint32_t* ticket = tickets + (size_t)p.u * 4 + warp;
-  int g_first = 0, g_last = 0;
-  bool direct = false, own_first = false;  // own_first: this CTA is the lower of the two contributors
+  const int g_first = sp.owner(p.u * sp.nblk), g_last = sp.owner((p.u + 1) * sp.nblk - 1);
+  bool own_first = false;  // this CTA is the lower of the two contributors
   const float* other = nullptr;
   float m_o = 0.f, l_o = 0.f;
   float4 vo[16];
-  if (!whole) {
-    g_first = sp.owner(p.u * sp.nblk);
-    g_last = sp.owner((p.u + 1) * sp.nblk - 1);
-    if (last_of_span && g_last == g_first + 1 && peek == 1u) {
-      direct = true;
-      own_first = (int)blockIdx.x == g_first;
-      other = slot_of<DH>(pieces, sp, (int)blockIdx.x == g_first ? g_last : g_first, p.u);
-      m_o = __ldcg(other + kM + row);
-      l_o = __ldcg(other + kL + row);
+  // the publisher warp watches the tickets of the span's last unit; its answer carries the
+  // acquire that orders the loads below after the other contributor's writes
+  const bool direct = last_of_span && g_last == g_first + 1 && ld_acquire_cta(&bar->others_done) == 1u;
+  if (last_of_span && row == 0) *(volatile uint32_t*)&bar->poll_stop = 1u;
+  if (direct) {
+    own_first = (int)blockIdx.x == g_first;
+    other = slot_of<DH>(pieces, sp, own_first ? g_last : g_first, p.u);
+    m_o = __ldcg(other + kM + row);
+    l_o = __ldcg(other + kL + row);
 #pragma unroll
-      for (int q = 0; q < 16; ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)q * kBM + row);
-    }
+    for (int q = 0; q < 16; ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)q * kBM + row);
   }
   if (!mbar_wait(&bar->o_done, pc & 1, dev_status, &bar->abort_flag)) return false;
   tc_fence_after();
@@ -385,7 +422,7 @@ __device__ __noinline__ bool finish_piece(uint32_t ob, Barriers* bar, Piece p, i
   }
   __nv_bfloat16* dst = out_row<DH>(o, p.u, row, L, heads);
   float* slot = pieces + (size_t)(2 * blockIdx.x + (pc > 0 ? 1 : 0)) * piece_floats<DH>();
-  float w_own = 1.f, w_o = 0.f, inv = 1.f / l;
+  float w_own = 1.f, w_o = 0.f, inv = 1.f;
   if (direct) {
     const float M = fmaxf(m_used, m_o);
     w_own = ex2_mufu(m_used - M);
@@ -397,9 +434,7 @@ __device__ __noinline__ bool finish_piece(uint32_t ob, Barriers* bar, Piece p, i
     uint32_t r[32];
     tmem_ld32(ob + c * 32, r);
     tmem_wait_ld();
-    if (whole) {
-      if (dst) store_row32(dst + c * 32, r, inv);
-    } else if (direct) {
+    if (direct) {
       if (c > 0 && (c & 1) == 0) {  // next 64 columns of the other piece
 #pragma unroll
         for (int q = 0; q < 16; ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)(c * 8 + q) * kBM + row);
@@ -425,7 +460,7 @@ __device__ __noinline__ bool finish_piece(uint32_t ob, Barriers* bar, Piece p, i
   tc_fence_before();
   __syncwarp();
   if (lane == 0) mbar_arrive(&bar->o_free);  // the next piece's first PV product may overwrite the accumulator
-  if (whole || direct) return true;
+  if (direct) return true;
   slot[kM + row] = m_used;
   slot[kL + row] = l;
   if (!last_of_span) {  // the publisher thread fences, draws the tickets and leaves them for settle_first_piece
@@ -452,6 +487,15 @@ __device__ __noinline__ void settle_first_piece(Barriers* bar, int it_begin, int
   if (bar->first_ticket[row >> 5] != (uint32_t)(g_last - g_first)) return;
   __threadfence();
   combine_rows<DH>(pieces, sp, u, g_first, g_last, row, out_row<DH>(o, u, row, L, heads));
+}
+
+// The ragged last key tile of a sequence: out of line, so that the hot loop holds one copy of the
+// softmax code.
+template <int DH>
+__device__ __noinline__ bool softmax_tile_ragged(uint32_t sb, uint32_t ob, float scale_log2, int valid, int j, float& m_used,
+                                                 float& l, uint64_t* pv_done, uint32_t pv_parity, uint32_t* dev_status,
+                                                 volatile int* abort_flag) {
+  return softmax_tile<DH, true>(sb, ob, scale_log2, valid, j, m_used, l, pv_done, pv_parity, dev_status, abort_flag);
 }
 
 template <int DH>
@@ -491,6 +535,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     mbar_init(&bar->o_free, 4);
     mbar_init(&bar->pub_ready, 4);
     mbar_init(&bar->pub_done, 1);
+    bar->others_done = 0;
+    bar->poll_stop = 0;
     bar->abort_flag = 0;
     mbar_fence_init();
   }
@@ -634,6 +680,24 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         for (int w = 0; w < 4; ++w) bar->first_ticket[w] = t[w];
         mbar_arrive(&bar->pub_done);
       }
+      // When the span ends inside a unit that one other CTA shares, that CTA ran its part at the
+      // start of its span and has normally published it long since.  Watch its four tickets (acquire)
+      // and leave the answer in shared memory for the softmax warps: they add the two pieces up
+      // straight from tensor memory if the answer is there when their last piece ends, and go
+      // through scratch and tickets otherwise.  Polling keeps the ticket out of their registers.
+      const int ul = (it_end - 1) / nblk;
+      if (it_end < (ul + 1) * nblk && sp.owner((ul + 1) * nblk - 1) == sp.owner(ul * nblk) + 1) {
+        const uint32_t* tk = tickets + (size_t)ul * 4;
+        for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+          if (*(volatile uint32_t*)&bar->poll_stop || *abort_flag) break;
+          if (ld_acquire_gpu(tk) == 1u && ld_acquire_gpu(tk + 1) == 1u && ld_acquire_gpu(tk + 2) == 1u &&
+              ld_acquire_gpu(tk + 3) == 1u) {
+            st_release_cta(&bar->others_done, 1u);
+            break;
+          }
+          __nanosleep(500);
+        }
+      }
     }
   } else if (warp < 4) {
     // ------------------------------------------------------------------ softmax / correction / epilogue
@@ -646,10 +710,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const Piece p = piece_at(it, it_end, nblk);
       it += p.cnt;
       float m_used = -INFINITY, l = 0.f;
-      // a partial last piece is normally the last contributor of its unit: look at the ticket now
-      // (acquire), so that the answer is there when the piece ends
-      uint32_t peek = 0;
-      if (it >= it_end && p.cnt < nblk) peek = ld_acquire_gpu(tickets + (size_t)p.u * 4 + warp);
       for (int j = 0; j < p.cnt; ++j, ++n) {
         const uint32_t sb = tmem + lane_addr + C::kColS + (n & 1) * kBN;
         if (!mbar_wait(&bar->s_full[n & 1], (n >> 1) & 1, dev_status, abort_flag)) { ok = false; break; }
@@ -658,14 +718,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         uint64_t* pvb = &bar->v_empty[(n + C::kStages - 1) % C::kStages];  // barrier the previous tile's PV commits to
         const uint32_t pvp = (uint32_t)(((n - 1) / C::kStages) & 1);
         if (valid >= kBN) ok = softmax_tile<DH, false>(sb, ob, scale_log2, kBN, j, m_used, l, pvb, pvp, dev_status, abort_flag);
-        else ok = softmax_tile<DH, true>(sb, ob, scale_log2, valid, j, m_used, l, pvb, pvp, dev_status, abort_flag);
+        else ok = softmax_tile_ragged<DH>(sb, ob, scale_log2, valid, j, m_used, l, pvb, pvp, dev_status, abort_flag);
         if (!ok) break;
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bar->p_full[n & 1]);
       }
       if (!ok) break;
-      ok = finish_piece<DH>(ob, bar, p, pc, it >= it_end, peek, row, m_used, l, o, L, heads, sp, tickets, pieces, dev_status);
+      if (p.cnt == nblk) ok = finish_whole<DH>(ob, bar, p.u, pc, row, l, o, L, heads, dev_status);
+      else ok = finish_partial<DH>(ob, bar, p, pc, it >= it_end, row, m_used, l, o, L, heads, sp, tickets, pieces, dev_status);
     }
     if (ok) settle_first_piece<DH>(bar, it_begin, it_end, row, o, L, heads, sp, pieces, dev_status);
   }
