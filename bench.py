@@ -364,12 +364,25 @@ def main():
                 "hbm_peak_gbs": peaks["hbm_gbs"]}
 
     # ---- end to end: pinned host input -> device -> block -> host output, every step ----------
-    x_dev = torch.empty_like(xs[0])
+    # One toma_block_host call per step (host pointers through the C ABI).  Copy-in, kernels and copy-out
+    # run on three streams chained by the call; two sets of staging buffers let step t+1's copy-in and
+    # step t-1's copy-out overlap step t's kernels.  The waits below order the reuse of a staging buffer.
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    x_stage = [torch.empty_like(xs[0]) for _ in range(2)]
+    out_stage = [torch.empty_like(xs[0]) for _ in range(2)]
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    ev_done = [torch.cuda.Event() for _ in range(2)]
+    ev_out = [torch.cuda.Event() for _ in range(2)]
+    for e in ev_in + ev_done + ev_out:
+        e.record()  # creates the handles; everything before the loop is complete by then
 
     def e2e_step(t):
-        x_dev.copy_(xs_host[t % cycle], non_blocking=True)
-        toma.toma_block(desc, t % cycle, x_dev, out, idx, w, ws, status)
-        out_host.copy_(out, non_blocking=True)
+        k = t % 2
+        s_in.wait_event(ev_done[k])                          # kernels of step t-2 have read x_stage[k]
+        torch.cuda.current_stream().wait_event(ev_out[k])    # copy-out of step t-2 has read out_stage[k]
+        toma.toma_block_host(desc, t % cycle, xs_host[t % cycle], out_host, x_stage[k], out_stage[k], idx, w, ws, status,
+                             s_in, s_out, ev_in[k], ev_done[k])
+        ev_out[k].record(s_out)
 
     for t in range(3):
         e2e_step(t)

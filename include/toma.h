@@ -161,6 +161,23 @@ TOMA_API toma_status toma_unmerge(const toma_desc* desc, const void* w, const vo
 TOMA_API toma_status toma_block(const toma_desc* desc, int32_t step, const void* x, void* out, int32_t* idx_state,
                        void* w_state, void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream);
 
+/* toma_block for callers whose tokens live in HOST memory (Algorithm 3 end to end, copies included):
+ * copy x_host -> x_dev, run toma_block(x_dev -> out_dev), copy out_dev -> out_host.
+ *   x_host, out_host: HOST buffers of batch*(N + n_extra)*dim elements, caller-owned.  Page-locked
+ *       memory makes the copies asynchronous; pageable memory works but the copies then block the host.
+ *   x_dev, out_dev: DEVICE staging buffers of the same size, caller-owned (the library never allocates).
+ *   stream: where the block's kernels run.  copy_in_stream / copy_out_stream: where the two copies
+ *       run; NULL means `stream` (everything in order on one stream).  With separate streams the call
+ *       chains copy-in -> kernels -> copy-out through the two caller-owned events (cudaEvent_t passed
+ *       as void*, required in that case), so that the copies of neighbouring steps overlap this step's
+ *       kernels.  The caller then orders what the call cannot see: a staging buffer may be handed to a
+ *       later call only after the earlier call's use of it has finished.
+ * Errors as toma_block; TOMA_ERR_NULL if separate streams are given without events. */
+TOMA_API toma_status toma_block_host(const toma_desc* desc, int32_t step, const void* x_host, void* out_host, void* x_dev,
+                                     void* out_dev, int32_t* idx_state, void* w_state, void* ws, size_t ws_bytes,
+                                     uint32_t* dev_status, void* stream, void* copy_in_stream, void* copy_out_stream,
+                                     void* copied_in_event, void* computed_event);
+
 /* Conversions between the opaque weight buffer and dense fp32 A~ [batch][P][D_loc][N_loc]
  * (device pointers).  For tests and for callers that bring their own weights (a
  * one-hot matrix makes merge a hard ToMeSD-style merge, Sec. 4.2). */

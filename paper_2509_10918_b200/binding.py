@@ -21,7 +21,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_RATIO", "ERR_TA
 
 EXPORTS = ["toma_select_static", "toma_launch_counter", "toma_workspace_bytes", "toma_weights_bytes", "toma_dest_per_tile", "toma_validate", "toma_status_str",
            "toma_select", "toma_merge_weights", "toma_merge", "toma_attention_workspace_bytes", "toma_attention",
-           "toma_unmerge", "toma_block",
+           "toma_unmerge", "toma_block", "toma_block_host",
            "toma_weights_export", "toma_weights_import"]
 
 
@@ -79,6 +79,9 @@ def _load() -> ctypes.CDLL:
     lib.toma_block.restype = c_int32
     lib.toma_block.argtypes = [P, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p,
                                c_void_p]
+    lib.toma_block_host.restype = c_int32
+    lib.toma_block_host.argtypes = [P, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                    c_size_t, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.toma_weights_export.restype = c_int32
     lib.toma_weights_export.argtypes = [P, c_void_p, c_void_p, c_void_p]
     lib.toma_weights_import.restype = c_int32
@@ -205,6 +208,24 @@ def toma_attention(batch, length, n_heads, head_dim, dtype, q, k, v, o, dev_stat
 def toma_block(desc, step, x, out, idx_state, w_state, ws, dev_status=None):
     _check(lib.toma_block(ctypes.byref(desc), step, _ptr(x), _ptr(out), _ptr(idx_state), _ptr(w_state), _ptr(ws),
                           ws.numel() * ws.element_size(), _ptr(dev_status), _stream()), "toma_block")
+
+
+def toma_block_host(desc, step, x_host, out_host, x_dev, out_dev, idx_state, w_state, ws, dev_status=None,
+                    copy_in_stream=None, copy_out_stream=None, copied_in_event=None, computed_event=None):
+    """x_host / out_host: CPU tensors (pinned for asynchronous copies); the streams are torch.cuda.Stream
+    objects and the events torch.cuda.Event objects that have been recorded at least once (so that
+    their handles exist), or None to run everything on the current stream."""
+    if x_host.is_cuda or out_host.is_cuda:
+        raise ValueError("toma_block_host takes host tensors for x_host / out_host")
+
+    def handle(obj, attr):
+        return None if obj is None else getattr(obj, attr)
+
+    _check(lib.toma_block_host(ctypes.byref(desc), step, x_host.data_ptr(), out_host.data_ptr(), _ptr(x_dev),
+                               _ptr(out_dev), _ptr(idx_state), _ptr(w_state), _ptr(ws), ws.numel() * ws.element_size(),
+                               _ptr(dev_status), _stream(), handle(copy_in_stream, "cuda_stream"),
+                               handle(copy_out_stream, "cuda_stream"), handle(copied_in_event, "cuda_event"),
+                               handle(computed_event, "cuda_event")), "toma_block_host")
 
 
 def toma_weights_export(desc, w, dense):

@@ -261,6 +261,33 @@ toma_status toma_block(const toma_desc* desc, int32_t step, const void* x, void*
   return cuda_ok(e);
 }
 
+toma_status toma_block_host(const toma_desc* desc, int32_t step, const void* x_host, void* out_host, void* x_dev,
+                            void* out_dev, int32_t* idx_state, void* w_state, void* ws, size_t ws_bytes,
+                            uint32_t* dev_status, void* stream, void* copy_in_stream, void* copy_out_stream,
+                            void* copied_in_event, void* computed_event) {
+  Geom g;
+  toma_status st = make_geom(desc, &g);
+  if (st != TOMA_OK) return st;
+  if (!x_host || !out_host || !x_dev || !out_dev) return TOMA_ERR_NULL;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaStream_t s_in = copy_in_stream ? (cudaStream_t)copy_in_stream : s;
+  cudaStream_t s_out = copy_out_stream ? (cudaStream_t)copy_out_stream : s;
+  if ((s_in != s && !copied_in_event) || (s_out != s && !computed_event)) return TOMA_ERR_NULL;
+  const size_t bytes = (size_t)g.B * (size_t)g.tokens_all() * g.d * (g.f32 ? 4 : 2);
+  if (cudaMemcpyAsync(x_dev, x_host, bytes, cudaMemcpyHostToDevice, s_in) != cudaSuccess) return TOMA_ERR_CUDA;
+  if (s_in != s) {
+    if (cudaEventRecord((cudaEvent_t)copied_in_event, s_in) != cudaSuccess) return TOMA_ERR_CUDA;
+    if (cudaStreamWaitEvent(s, (cudaEvent_t)copied_in_event, 0) != cudaSuccess) return TOMA_ERR_CUDA;
+  }
+  st = toma_block(desc, step, x_dev, out_dev, idx_state, w_state, ws, ws_bytes, dev_status, stream);
+  if (st != TOMA_OK) return st;
+  if (s_out != s) {
+    if (cudaEventRecord((cudaEvent_t)computed_event, s) != cudaSuccess) return TOMA_ERR_CUDA;
+    if (cudaStreamWaitEvent(s_out, (cudaEvent_t)computed_event, 0) != cudaSuccess) return TOMA_ERR_CUDA;
+  }
+  return cuda_ok(cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, s_out));
+}
+
 toma_status toma_weights_export(const toma_desc* desc, const void* w, float* dense, void* stream) {
   Geom g;
   toma_status st = make_geom(desc, &g);

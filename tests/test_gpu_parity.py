@@ -267,6 +267,33 @@ def test_block_separate_weight_schedule_parity(toma):
         assert_close(to_host64(out), want, cfg.dtype, f"block step {step}")
 
 
+@pytest.mark.parametrize("streams", [False, True])
+def test_block_host_matches_block(toma, streams):
+    """toma_block_host (host buffers through the C ABI, copies on the call's streams) returns what
+    toma_block returns on the same inputs, with one stream and with separate copy streams."""
+    cfg = gen.config("cfg2", batch=1, steps=4, reuse_interval=2)
+    desc = toma.desc_from_config(cfg)
+    idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    idx2, w2, ws2 = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    s_in = torch.cuda.Stream() if streams else None
+    s_out = torch.cuda.Stream() if streams else None
+    ev = [torch.cuda.Event() for _ in range(2)] if streams else [None, None]
+    for e in ev:
+        if e is not None:
+            e.record()
+    for step, x_host in enumerate(gen.feature_sequence(cfg)):
+        xh = torch.from_numpy(x_host).to(torch.bfloat16).pin_memory()
+        oh = torch.empty_like(xh).pin_memory()
+        x_dev, out_dev = torch.empty_like(xh, device="cuda"), torch.empty_like(xh, device="cuda")
+        toma.toma_block_host(desc, step, xh, oh, x_dev, out_dev, idx, w, ws, None, s_in, s_out, ev[0], ev[1])
+        x = xh.cuda()
+        want = torch.empty_like(x)
+        toma.toma_block(desc, step, x, want, idx2, w2, ws2, None)
+        torch.cuda.synchronize()
+        assert torch.equal(oh, want.cpu())
+        assert torch.equal(idx, idx2)
+
+
 def test_block_long_sequence_schedule_and_sampled_parity(toma):
     """The 28-step stress sequence: selection may only change on refresh steps, and sampled
     tiles of every refresh match the oracle exactly."""
