@@ -184,9 +184,13 @@ def other_workloads(toma, torch, flush, peaks):
     out = {}
     # cfg2 states no schedule: the paper's weight interval (5) is used.  cfg4 (Flux) does not reuse across
     # timesteps but shares one selection among the blocks of a kind within a step (19 joint blocks).
-    for name, reuse in (("cfg2", 5), ("cfg4", 19), ("cfg5a", 5)):
-        cfg = gen.config(name, reuse_interval=reuse)
-        desc = toma.desc_from_config(cfg)
+    # cfg3_stripes: the same tokens cut into stripes of 4 full rows (256 tokens per region, as a 16x16 tile) under
+    # the paper's own schedule, destinations every 10 steps and weights every 5.
+    for label, name, over, reuse, w_reuse in (("cfg2", "cfg2", {}, 5, 0), ("cfg4", "cfg4", {}, 19, 0),
+                                              ("cfg5a", "cfg5a", {}, 5, 0),
+                                              ("cfg3_stripes", "cfg3", dict(tile_h=4, tile_w=64), 10, 5)):
+        cfg = gen.config(name, reuse_interval=reuse, **over)
+        desc = toma.desc_from_config(cfg, weight_reuse_interval=w_reuse)
         tdt = toma.torch_dtype(desc)
         x = torch.from_numpy(gen.features(cfg)).cuda().to(tdt)
         y = torch.empty_like(x)
@@ -210,12 +214,16 @@ def other_workloads(toma, torch, flush, peaks):
 
         refresh = t_us(lambda: toma.toma_block(desc, 0, x, y, idx, w, ws, None))
         reuse_us = t_us(lambda: toma.toma_block(desc, 1, x, y, idx, w, ws, None)) if reuse > 1 else None
+        # steps that recompute the weights from the cached destinations
+        n_w = reuse // w_reuse - 1 if w_reuse else 0
+        weights_us = t_us(lambda: toma.toma_block(desc, w_reuse, x, y, idx, w, ws, None)) if n_w else None
         full = t_us(lambda: toma.toma_attention(B, N, cfg.n_heads, cfg.head_dim, cfg.dtype, x, x, x, y, None))
-        mean = refresh if reuse == 1 else (refresh + (reuse - 1) * reuse_us) / reuse
-        out[name] = {"tokens": B * N, "reuse_interval": reuse, "refresh_us": refresh, "reuse_us": reuse_us,
-                     "block_mean_us": mean, "full_attention_us": full, "speedup_vs_full_attention": full / mean,
-                     "tokens_per_s": B * N / (mean * 1e-6),
-                     "full_attention_tflops": 4.0 * B * N * N * d / full / 1e6}
+        mean = refresh if reuse == 1 else (refresh + n_w * (weights_us or 0.0) + (reuse - 1 - n_w) * reuse_us) / reuse
+        out[label] = {"tokens": B * N, "tile": [cfg.tile_h, cfg.tile_w], "reuse_interval": reuse,
+                      "weight_reuse_interval": w_reuse or reuse, "refresh_us": refresh, "weights_only_us": weights_us,
+                      "reuse_us": reuse_us, "block_mean_us": mean, "full_attention_us": full,
+                      "speedup_vs_full_attention": full / mean, "tokens_per_s": B * N / (mean * 1e-6),
+                      "full_attention_tflops": 4.0 * B * N * N * d / full / 1e6}
         del x, y, idx, w, ws
         torch.cuda.empty_cache()
     return out

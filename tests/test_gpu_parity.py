@@ -294,6 +294,28 @@ def test_block_host_matches_block(toma, streams):
         assert torch.equal(idx, idx2)
 
 
+def test_stripe_regions_full_size_parity(toma):
+    """Stripe regions (Sec. 4.3.1) at the benchmark size: 64x64 tokens cut into stripes of 4 full rows,
+    under the schedule the paper settles on (destinations every 10 steps, weights every 5)."""
+    cfg = gen.config("cfg3", batch=1, tile_h=4, tile_w=64, steps=7, reuse_interval=10)
+    desc = toma.desc_from_config(cfg, weight_reuse_interval=5)
+    idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    st = O.BlockState()
+    kw = dict(grid_h=cfg.grid_h, grid_w=cfg.grid_w, tile_h=4, tile_w=64, merge_ratio=cfg.merge_ratio, tau=cfg.tau,
+              n_heads=cfg.n_heads, reuse_interval=10, weight_reuse_interval=5)
+    for step, x_host in enumerate(gen.feature_sequence(cfg)):
+        x = to_dev(x_host, cfg.dtype)
+        out = torch.empty_like(x)
+        toma.toma_block(desc, step, x, out, idx, w, ws, None)
+        torch.cuda.synchronize()
+        if step in (0, 5, 6):  # refresh, weights-only refresh, reuse after it
+            want, _, _ = O.block_step(x_host, step, st, **kw)
+            assert np.array_equal(idx.cpu().numpy().astype(np.int64), st.idx)
+            assert_close(to_host64(out), want, cfg.dtype, f"stripe block step {step}")
+        else:  # keep the oracle's state in step without paying for its attention
+            assert step % 5 != 0
+
+
 def test_block_long_sequence_schedule_and_sampled_parity(toma):
     """The 28-step stress sequence: selection may only change on refresh steps, and sampled
     tiles of every refresh match the oracle exactly."""
