@@ -44,7 +44,11 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     mbar_init(&bar->done, 1);
     bar->abort_flag = 0;
     mbar_fence_init();
+    prefetch_tmap(&tm_a);
+    prefetch_tmap(&tm_b);
   }
+  dependency_wait();  // before tensor memory is held and before any global access
+  if (threadIdx.x == 0) release_dependents();
   if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
   tc_fence_before();
   __syncthreads();
@@ -54,8 +58,6 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
   if (warp == 0) {
     if (lane == 0) {
-      prefetch_tmap(&tm_a);
-      prefetch_tmap(&tm_b);
       for (int k = 0; k < nk; ++k) {
         const int s = k % kStages;
         if (k >= kStages && !mbar_wait(&bar->empty[s], ((k / kStages) - 1) & 1, dev_status, abort_flag)) break;
@@ -146,9 +148,9 @@ cudaError_t launch_gram_tc(const Geom& g, const __nv_bfloat16* y, int16_t* sq, u
     attr = true;
   }
   dim3 grid(g.B * g.P, (g.Nloc + 127) / 128, g.Nloc / n_cols);
-  gram_tc_kernel<<<grid, 192, smem, s>>>(ta, tb, sq, g.Nloc, g.d, n_cols, dev_status);
+  const cudaError_t le = launch_dependent(gram_tc_kernel, grid, dim3(192), (size_t)smem, s, ta, tb, sq, g.Nloc, g.d, n_cols, dev_status);
   count_launch();
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 }  // namespace toma

@@ -2,6 +2,7 @@
 // fixed-point Gram matrix per tile (plain FFMA version) and the greedy
 // facility-location argmax with exact incremental integer gains.
 #include "common.cuh"
+#include "tc.cuh"
 
 namespace toma {
 
@@ -14,6 +15,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) quantise_kernel(const T* __restrict__ x, __nv_bfloat16* __restrict__ y, int B,
                                                        int N, int n_all, int d, int W, int th, int tw, int tiles_x,
                                                        int P, int Nloc) {
+  tc::dependency_wait();  // launched with programmatic stream serialisation
+  if (threadIdx.x == 0) tc::release_dependents();
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (warp >= B * N) return;
@@ -40,14 +43,15 @@ __global__ void __launch_bounds__(256) quantise_kernel(const T* __restrict__ x, 
 cudaError_t launch_quantise(const Geom& g, const void* x, __nv_bfloat16* y, cudaStream_t s) {
   const long long warps = (long long)g.B * g.N;
   const int blocks = (int)((warps * 32 + 255) / 256);
+  cudaError_t e;
   if (g.f32)
-    quantise_kernel<float><<<blocks, 256, 0, s>>>((const float*)x, y, g.B, g.N, (int)g.tokens_all(), g.d, g.W, g.th,
+    e = launch_dependent(quantise_kernel<float>, dim3(blocks), dim3(256), 0, s, (const float*)x, y, g.B, g.N, (int)g.tokens_all(), g.d, g.W, g.th,
                                                   g.tw, g.tiles_x, g.P, g.Nloc);
   else
-    quantise_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>((const __nv_bfloat16*)x, y, g.B, g.N, (int)g.tokens_all(),
+    e = launch_dependent(quantise_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, s, (const __nv_bfloat16*)x, y, g.B, g.N, (int)g.tokens_all(),
                                                           g.d, g.W, g.th, g.tw, g.tiles_x, g.P, g.Nloc);
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------
@@ -152,6 +156,8 @@ __global__ void __launch_bounds__(1024) greedy_kernel(const int16_t* __restrict_
   const int16_t* Sg = sq + (size_t)blockIdx.x * Nloc * Nloc;
   const int16_t* S = Sg;
   if (threadIdx.x == 0) n_changed[0] = n_changed[1] = 0;
+  tc::dependency_wait();  // launched with programmatic stream serialisation
+  if (threadIdx.x == 0) tc::release_dependents();
   if (kSmemS) {
     const int n16 = Nloc * Nloc / 8;  // 16-byte packets
     const uint4* src = reinterpret_cast<const uint4*>(Sg);
@@ -235,19 +241,20 @@ cudaError_t launch_greedy(const Geom& g, const int16_t* sq, int32_t* idx, cudaSt
   const int threads = ((g.Nloc + 31) / 32) * 32;
   const size_t s_bytes = (size_t)g.Nloc * g.Nloc * 2;
   const bool smem_s = g.Nloc <= 256 && (g.Nloc * g.Nloc) % 8 == 0;
+  cudaError_t e;
   if (smem_s) {
     static bool attr = false;
     if (!attr) {
-      cudaError_t e = cudaFuncSetAttribute(greedy_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * 256 * 2);
+      e = cudaFuncSetAttribute(greedy_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * 256 * 2);
       if (e != cudaSuccess) return e;
       attr = true;
     }
-    greedy_kernel<true><<<g.B * g.P, threads, s_bytes, s>>>(sq, idx, g.Nloc, g.Dloc);
+    e = launch_dependent(greedy_kernel<true>, dim3(g.B * g.P), dim3(threads), s_bytes, s, sq, idx, g.Nloc, g.Dloc);
   } else {
-    greedy_kernel<false><<<g.B * g.P, threads, 0, s>>>(sq, idx, g.Nloc, g.Dloc);
+    e = launch_dependent(greedy_kernel<false>, dim3(g.B * g.P), dim3(threads), 0, s, sq, idx, g.Nloc, g.Dloc);
   }
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace toma

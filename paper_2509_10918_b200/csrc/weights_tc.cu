@@ -36,6 +36,8 @@ struct WParams {
 __global__ void __launch_bounds__(256)
 gather_dest_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ idx, __nv_bfloat16* __restrict__ dg,
                    WParams p, int rows_total) {
+  dependency_wait();  // launched with programmatic stream serialisation
+  if (threadIdx.x == 0) release_dependents();
   const int vec_per_row = p.d / 8;  // 16-byte packets
   const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= (long long)rows_total * vec_per_row) return;
@@ -85,7 +87,11 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
     mbar_init(&bar->done, 1);
     bar->abort_flag = 0;
     mbar_fence_init();
+    prefetch_tmap(&tm_x);
+    prefetch_tmap(&tm_d);
   }
+  dependency_wait();  // before tensor memory is held and before any global access
+  if (threadIdx.x == 0) release_dependents();
   if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
   tc_fence_before();
   __syncthreads();
@@ -95,8 +101,6 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
 
   if (warp == 0) {
     if (lane == 0) {
-      prefetch_tmap(&tm_x);
-      prefetch_tmap(&tm_d);
       for (int k = 0; k < nk; ++k) {
         const int s = k % p.stages;
         if (k >= p.stages && !mbar_wait(&bar->empty[s], ((k / p.stages) - 1) & 1, dev_status, abort_flag)) break;
@@ -204,6 +208,8 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
 __global__ void __launch_bounds__(256)
 weights_normalise_kernel(const float* __restrict__ shares, const float* __restrict__ zpart, __nv_bfloat16* __restrict__ w,
                          int Nloc, int Dloc, int mblocks, size_t total) {
+  dependency_wait();  // launched with programmatic stream serialisation
+  if (threadIdx.x == 0) release_dependents();
   const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= total) return;
   const size_t plane = (size_t)Nloc * Dloc;
@@ -249,8 +255,10 @@ cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, 
 
   const int rows_total = (int)(tiles * g.Dloc);
   const long long vecs = (long long)rows_total * (g.d / 8);
-  gather_dest_kernel<<<(unsigned)((vecs + 255) / 256), 256, 0, s>>>((const __nv_bfloat16*)x, idx, dg, p, rows_total);
+  cudaError_t le = launch_dependent(gather_dest_kernel, dim3((unsigned)((vecs + 255) / 256)), dim3(256), 0, s,
+                                    (const __nv_bfloat16*)x, idx, dg, p, rows_total);
   count_launch();
+  if (le != cudaSuccess) return le;
 
   CUtensorMap tx, td;
   const uint64_t xdims[4] = {(uint64_t)g.d, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.B};
@@ -274,13 +282,14 @@ cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, 
     attr = true;
   }
   dim3 grid((unsigned)tiles, mblocks);
-  weights_logits_kernel<<<grid, 192, smem, s>>>(tx, td, shares, zpart, p, dev_status);
+  le = launch_dependent(weights_logits_kernel, grid, dim3(192), (size_t)smem, s, tx, td, shares, zpart, p, dev_status);
   count_launch();
+  if (le != cudaSuccess) return le;
   const size_t total = tiles * g.Nloc * g.Dloc;
-  weights_normalise_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(shares, zpart, (__nv_bfloat16*)w, g.Nloc,
-                                                                           g.Dloc, mblocks, total);
+  le = launch_dependent(weights_normalise_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, s, (const float*)shares,
+                        (const float*)zpart, (__nv_bfloat16*)w, g.Nloc, g.Dloc, mblocks, total);
   count_launch();
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 }  // namespace toma
