@@ -207,21 +207,36 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
 
 __global__ void __launch_bounds__(256)
 weights_normalise_kernel(const float* __restrict__ shares, const float* __restrict__ zpart, __nv_bfloat16* __restrict__ w,
-                         int Nloc, int Dloc, int mblocks, size_t total) {
+                         int Nloc, int Dloc, int mblocks) {
+  // grid (blocks over the tile's [N_loc][D_loc] plane in groups of four destinations, tile)
+  __shared__ float zs[512];  // row sums of the tile's D_loc (<= 512) destinations
   dependency_wait();  // launched with programmatic stream serialisation
   if (threadIdx.x == 0) release_dependents();
-  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= total) return;
-  const size_t plane = (size_t)Nloc * Dloc;
-  const size_t batch = e / plane, r = e - batch * plane;
-  const int i = (int)(r % Dloc);
-  float z = 0.f;
-  for (int mb = 0; mb < mblocks; ++mb) z += zpart[(batch * mblocks + mb) * Dloc + i];
-  const float v = z > 0.f ? shares[e] / z : 0.f;
+  const size_t batch = blockIdx.y;
+  for (int i = threadIdx.x; i < Dloc; i += blockDim.x) {
+    float z = 0.f;
+    for (int mb = 0; mb < mblocks; ++mb) z += zpart[(batch * mblocks + mb) * Dloc + i];
+    zs[i] = z;
+  }
+  __syncthreads();
+  const int plane = Nloc * Dloc;
+  const float4* src = reinterpret_cast<const float4*>(shares + batch * plane);
   __nv_bfloat16* t = w + batch * 2 * plane;
-  const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-  t[r] = hi;
-  t[plane + r] = __float2bfloat16_rn(v - __bfloat162float(hi));
+  for (int q = blockIdx.x * blockDim.x + threadIdx.x; q < plane / 4; q += gridDim.x * blockDim.x) {
+    const int r = q * 4, i = r % Dloc;  // D_loc is a multiple of 4: the four stay in one row
+    const float4 a = src[q];
+    const float in[4] = {a.x, a.y, a.z, a.w};
+    __nv_bfloat16 hi[4], lo[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float z = zs[i + e];
+      const float v = z > 0.f ? in[e] / z : 0.f;
+      hi[e] = __float2bfloat16_rn(v);
+      lo[e] = __float2bfloat16_rn(v - __bfloat162float(hi[e]));
+    }
+    *reinterpret_cast<uint2*>(t + r) = *reinterpret_cast<const uint2*>(hi);
+    *reinterpret_cast<uint2*>(t + plane + r) = *reinterpret_cast<const uint2*>(lo);
+  }
 }
 
 }  // namespace
@@ -285,9 +300,10 @@ cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, 
   le = launch_dependent(weights_logits_kernel, grid, dim3(192), (size_t)smem, s, tx, td, shares, zpart, p, dev_status);
   count_launch();
   if (le != cudaSuccess) return le;
-  const size_t total = tiles * g.Nloc * g.Dloc;
-  le = launch_dependent(weights_normalise_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, s, (const float*)shares,
-                        (const float*)zpart, (__nv_bfloat16*)w, g.Nloc, g.Dloc, mblocks, total);
+  const int quads = g.Nloc * g.Dloc / 4;
+  const int nblocks = (quads + 1023) / 1024 > 0 ? (quads + 1023) / 1024 : 1;  // four quads per thread
+  le = launch_dependent(weights_normalise_kernel, dim3((unsigned)nblocks, (unsigned)tiles), dim3(256), 0, s,
+                        (const float*)shares, (const float*)zpart, (__nv_bfloat16*)w, g.Nloc, g.Dloc, mblocks);
   count_launch();
   return le != cudaSuccess ? le : cudaGetLastError();
 }
