@@ -362,7 +362,7 @@ def main():
     mrg_bytes = B * (cfg.n_tokens * d * esz + cfg.n_merged * d * esz + cfg.n_tiles * cfg.n_loc * cfg.d_loc * esz)
     # traffic: dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this workload,
     # from the ncu capture summarised in profiles/attention_tc_cfg3_cfg5a.md (only valid for the default workload)
-    traffic = 5289216 if args.workload == "cfg3" else None
+    traffic = 5331200 + 225024 if args.workload == "cfg3" else None
     roofline = {"kernel": "attention over merged tokens", "bound": "tensor", "achieved": att_tf,
                 "peak": peaks["tf_burst"], "unit": "TFLOP/s", "frac": att_tf / peaks["tf_burst"], "traffic": traffic,
                 "algorithmic_flops_per_launch": att_flops,
