@@ -56,7 +56,7 @@ struct AttCfg {
   static constexpr int kSmemBytes = 1024 + kQBytes + 2 * kStages * kKvBytes + kOnesBytes + 256;
   static constexpr bool kSumMma = DH == 64;                // row sums on the tensor pipe, truncated P
   static constexpr int kTmemCols = 256;
-  static constexpr int kColS = 0, kColO = 128, kColL = 128 + DH;  // S buffers at 0 and 64
+  static constexpr int kColS = 0, kColO = 128;  // S buffers at columns 0 and 64; O (and, behind it, the row sums) at 128
 };
 
 struct Barriers {

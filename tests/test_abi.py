@@ -75,6 +75,16 @@ def test_null_and_workspace_errors_are_returned_before_any_launch(toma):
     assert lib.toma_merge(ctypes.byref(d), None, fake, fake, None, None) == NULL
     assert lib.toma_attention(1, 0, 1, 64, 0, fake, fake, fake, fake, None, 0, None, None) == 2
     assert lib.toma_attention(1, 8, 1, 48, 0, fake, fake, fake, fake, None, 0, None, None) == 7
+    # the tensor-core attention needs scratch: missing or short scratch is refused before any launch
+    need = lib.toma_attention_workspace_bytes(2, 2048, 10, 64, 0)
+    assert need > 0 and lib.toma_attention_workspace_bytes(2, 2048, 10, 64, 1) == 0  # fp32 path needs none
+    assert lib.toma_attention(2, 2048, 10, 64, 0, fake, fake, fake, fake, None, 0, None, None) == WS
+    assert lib.toma_attention(2, 2048, 10, 64, 0, fake, fake, fake, fake, fake, need - 1, None, None) == WS
+    assert lib.toma_block_host(ctypes.byref(d), 0, None, fake, fake, fake, fake, fake, fake, 1 << 40, None, None, None,
+                               None, None, None) == NULL
+    # separate copy streams without the events that chain them
+    assert lib.toma_block_host(ctypes.byref(d), 0, fake, fake, fake, fake, fake, fake, fake, 1 << 40, None, None, fake,
+                               None, None, None) == NULL
 
 
 def test_binding_refuses_cpu_tensors(toma):
