@@ -294,6 +294,35 @@ def test_block_host_matches_block(toma, streams):
         assert torch.equal(idx, idx2)
 
 
+def test_block_replays_from_a_cuda_graph(toma):
+    """A reuse step and a refresh step captured into CUDA graphs (the calls never allocate or synchronise,
+    and their dependent launches are capturable) replay to the same bits as direct calls."""
+    cfg = gen.config("cfg3", batch=1, steps=3, reuse_interval=2)
+    desc = toma.desc_from_config(cfg)
+    xs = [to_dev(x, cfg.dtype) for x in gen.feature_sequence(cfg)]
+    idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    idx2, w2, ws2 = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    x_in, out = torch.empty_like(xs[0]), torch.empty_like(xs[0])
+    x_in.copy_(xs[0])
+    toma.toma_block(desc, 0, x_in, out, idx, w, ws, None)  # first call outside capture (one-time attribute setup)
+    toma.toma_block(desc, 1, x_in, out, idx, w, ws, None)
+    torch.cuda.synchronize()
+    graphs = {}
+    for step in (0, 1):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            toma.toma_block(desc, step, x_in, out, idx, w, ws, None)
+        graphs[step] = g
+    for t, x in enumerate(xs):
+        x_in.copy_(x)
+        graphs[t % 2].replay()
+        want = torch.empty_like(x)
+        toma.toma_block(desc, t, x, want, idx2, w2, ws2, None)
+        torch.cuda.synchronize()
+        assert torch.equal(out, want), f"graph replay differs at step {t}"
+        assert torch.equal(idx, idx2)
+
+
 def test_stripe_regions_full_size_parity(toma):
     """Stripe regions (Sec. 4.3.1) at the benchmark size: 64x64 tokens cut into stripes of 4 full rows,
     under the schedule the paper settles on (destinations every 10 steps, weights every 5)."""
