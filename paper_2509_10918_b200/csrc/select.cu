@@ -146,16 +146,32 @@ __device__ __forceinline__ ArgMax block_argmax(ArgMax v, ArgMax* red, int nwarps
   return warp_argmax(lane < nwarps ? red[lane] : ArgMax{INT_MIN, INT_MAX});
 }
 
+// Argmax for tiles of at most 256 tokens (8 warps): gain (< 2^23) and index packed into one positive
+// int, gain in the high bits and 255 - index below, so that the largest key is the largest gain with
+// the lowest index; -1 never wins.  One warp reduction, one barrier, then every thread takes the
+// maximum of the eight warp keys itself (two 16-byte shared loads instead of two more reductions).
+__device__ __forceinline__ int block_argmax_packed(int gain, int i, bool candidate, int* keys /*[8], 16-byte aligned*/) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int key = __reduce_max_sync(0xffffffffu, candidate ? (gain << 8) | (255 - i) : -1);
+  if (lane == 0) keys[warp] = key;
+  __syncthreads();
+  const int4 a = reinterpret_cast<const int4*>(keys)[0], b = reinterpret_cast<const int4*>(keys)[1];
+  const int best = max(max(max(a.x, a.y), max(a.z, a.w)), max(max(b.x, b.y), max(b.z, b.w)));
+  return 255 - (best & 255);
+}
+
 template <bool kSmemS>
 __global__ void __launch_bounds__(1024) greedy_kernel(const int16_t* __restrict__ sq, int32_t* __restrict__ idx,
                                                       int Nloc, int Dloc) {
   extern __shared__ __align__(16) uint8_t greedy_smem[];
   __shared__ int2 changed[2][kMaxNloc];  // (column j, new << 16 | old & 0xffff) of columns whose cached maximum improved
   __shared__ ArgMax red[2][32];
+  __shared__ __align__(16) int keys[2][8];  // warp keys of block_argmax_packed (unused slots stay -1)
   __shared__ int n_changed[2];
   const int16_t* Sg = sq + (size_t)blockIdx.x * Nloc * Nloc;
   const int16_t* S = Sg;
   if (threadIdx.x == 0) n_changed[0] = n_changed[1] = 0;
+  if (threadIdx.x < 16) keys[threadIdx.x >> 3][threadIdx.x & 7] = -1;
   tc::dependency_wait();  // launched with programmatic stream serialisation
   if (threadIdx.x == 0) tc::release_dependents();
   if (kSmemS) {
@@ -193,7 +209,8 @@ __global__ void __launch_bounds__(1024) greedy_kernel(const int16_t* __restrict_
 
   for (int r = 1; r < Dloc; ++r) {
     const int pb = r & 1;
-    pick = block_argmax(ArgMax{(live && !selected) ? gain : kNever, i}, red[pb], nwarps);
+    if (kSmemS) pick.i = block_argmax_packed(gain, i, live && !selected, keys[pb]);  // N_loc <= 256
+    else pick = block_argmax(ArgMax{(live && !selected) ? gain : kNever, i}, red[pb], nwarps);
     if (i == pick.i) {
       selected = true;
       out[r] = pick.i;
