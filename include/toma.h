@@ -140,6 +140,19 @@ TOMA_API toma_status toma_merge(const toma_desc* desc, const void* w, const void
 TOMA_API size_t toma_attention_workspace_bytes(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim,
                                                int32_t dtype);
 
+/* Host-only diagnostic: how toma_attention would cut this shape's work across its persistent CTAs.
+ * A work unit is (batch, head, 128 queries); an iteration is one 64-key tile of a unit; CTA g runs the
+ * iterations bounds[g] .. bounds[g+1]-1 of the units laid end to end.
+ *   info[0] = number of CTAs G, info[1] = 1 if units are split between CTAs (cut at single key
+ *   tiles) or 0 if every CTA gets whole units, info[2] = work units, info[3] = key tiles per unit.
+ *   bounds (NULL or >= min(G+1, capacity) entries), owner_first / owner_last (NULL or >= min(G, capacity)
+ *   entries; filled only when units are split): the CTA the kernel's own arithmetic assigns to the
+ *   first and to the last iteration of span g (both equal g).
+ * Returns G, or 0 when the shape does not run on the tensor-core kernel (fp32, head_dim not 64/128). */
+TOMA_API int32_t toma_attention_plan(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim, int32_t dtype,
+                                     int32_t info[4], int32_t* bounds, int32_t* owner_first, int32_t* owner_last,
+                                     int32_t capacity);
+
 /* Multi-head attention core softmax(Q K^T / sqrt(head_dim)) V (Eq. 1 with tau = 1), no mask.
  *   q, k, v, o: [batch][len][n_heads][head_dim], device.
  *   ws: device scratch of at least toma_attention_workspace_bytes(), 16-byte aligned, caller-owned,

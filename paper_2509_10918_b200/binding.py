@@ -20,7 +20,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_RATIO", "ERR_TA
                 "ERR_UNSUPPORTED", "ERR_CUDA", "ERR_TIMEOUT", "ERR_SCRATCH_LIMIT"]
 
 EXPORTS = ["toma_select_static", "toma_launch_counter", "toma_workspace_bytes", "toma_weights_bytes", "toma_dest_per_tile", "toma_validate", "toma_status_str",
-           "toma_select", "toma_merge_weights", "toma_merge", "toma_attention_workspace_bytes", "toma_attention",
+           "toma_select", "toma_merge_weights", "toma_merge", "toma_attention_workspace_bytes", "toma_attention_plan", "toma_attention",
            "toma_unmerge", "toma_block", "toma_block_host",
            "toma_weights_export", "toma_weights_import"]
 
@@ -74,6 +74,8 @@ def _load() -> ctypes.CDLL:
     lib.toma_attention.restype = c_int32
     lib.toma_attention_workspace_bytes.restype = c_size_t
     lib.toma_attention_workspace_bytes.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32]
+    lib.toma_attention_plan.restype = c_int32
+    lib.toma_attention_plan.argtypes = [c_int32] * 5 + [c_void_p] * 4 + [c_int32]
     lib.toma_attention.argtypes = [c_int32, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
                                    c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
     lib.toma_block.restype = c_int32
@@ -187,6 +189,19 @@ def _dtype_code(dtype) -> int:
 
 def toma_attention_workspace_bytes(batch, length, n_heads, head_dim, dtype) -> int:
     return int(lib.toma_attention_workspace_bytes(batch, length, n_heads, head_dim, _dtype_code(dtype)))
+
+
+def toma_attention_plan(batch, length, n_heads, head_dim, dtype):
+    """Work plan of toma_attention for this shape: dict with the CTA count, whether units are split, the
+    span bounds and (when split) the owners the kernel's arithmetic gives each span's first and last iteration."""
+    cap = 1024
+    info = (c_int32 * 4)()
+    bounds, first, last = (c_int32 * cap)(), (c_int32 * cap)(), (c_int32 * cap)()
+    g = lib.toma_attention_plan(batch, length, n_heads, head_dim, _dtype_code(dtype), info, bounds, first, last, cap)
+    if g == 0:
+        return None
+    return {"ctas": g, "split": bool(info[1]), "units": info[2], "tiles_per_unit": info[3], "bounds": list(bounds[:g + 1]),
+            "owner_first": list(first[:g]) if info[1] else None, "owner_last": list(last[:g]) if info[1] else None}
 
 
 _attention_ws = {}

@@ -217,6 +217,12 @@ size_t toma_attention_workspace_bytes(int32_t batch, int32_t len, int32_t n_head
   return attention_ws_bytes(batch, len, n_heads, head_dim, dtype == TOMA_F32);
 }
 
+int32_t toma_attention_plan(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim, int32_t dtype, int32_t info[4],
+                            int32_t* bounds, int32_t* owner_first, int32_t* owner_last, int32_t capacity) {
+  if (!info || batch < 1 || len < 1 || n_heads < 1 || !attention_on_tc(head_dim, dtype == TOMA_F32)) return 0;
+  return attention_tc_plan(batch, len, n_heads, info, bounds, owner_first, owner_last, capacity);
+}
+
 toma_status toma_attention(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim, int32_t dtype,
                            const void* q, const void* k, const void* v, void* o, void* ws, size_t ws_bytes,
                            uint32_t* dev_status, void* stream) {

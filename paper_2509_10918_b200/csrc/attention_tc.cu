@@ -833,6 +833,25 @@ size_t attention_tc_workspace_bytes(int B, int L, int heads, int dh) {
 
 size_t attention_tc_ticket_bytes(int B, int L, int heads) { return ticket_bytes(B, L, heads); }
 
+int attention_tc_plan(int B, int L, int heads, int info[4], int* bounds, int* owner_first, int* owner_last, int capacity) {
+  const long long units = (long long)B * heads * ((L + kBM - 1) / kBM);
+  const int nblk = (L + kBN - 1) / kBN;
+  if (units * nblk > 0x7fffffffLL) return 0;
+  const Spans sp = plan_spans((int)units, nblk);
+  info[0] = sp.G;
+  info[1] = sp.quantum == 1 ? 1 : 0;
+  info[2] = (int)units;
+  info[3] = nblk;
+  for (int g = 0; g <= sp.G && g < capacity; ++g) {
+    if (bounds) bounds[g] = sp.bound(g);
+    if (g < sp.G && sp.quantum == 1) {
+      if (owner_first) owner_first[g] = sp.owner(sp.bound(g));
+      if (owner_last) owner_last[g] = sp.owner(sp.bound(g + 1) - 1);
+    }
+  }
+  return sp.G;
+}
+
 cudaError_t launch_attention_tc(int B, int L, int heads, int dh, const void* q, const void* k, const void* v, void* o,
                                 void* ws, bool tickets_clean, uint32_t* dev_status, cudaStream_t s) {
   if (dh == 64) return launch<64>(B, L, heads, q, k, v, o, ws, tickets_clean, dev_status, s);

@@ -69,6 +69,8 @@ size_t attention_tc_workspace_bytes(int B, int L, int heads, int dh);
 // kernel starts: the launcher clears them unless `tickets_clean` says an earlier kernel on the
 // stream already did.
 size_t attention_tc_ticket_bytes(int B, int L, int heads);
+// The work plan of a launch (see toma_attention_plan); returns the CTA count, 0 if the shape is too large.
+int attention_tc_plan(int B, int L, int heads, int info[4], int* bounds, int* owner_first, int* owner_last, int capacity);
 cudaError_t launch_attention_tc(int B, int L, int heads, int dh, const void* q, const void* k, const void* v, void* o,
                                 void* ws, bool tickets_clean, uint32_t* dev_status, cudaStream_t s);
 cudaError_t launch_weights_export(const Geom& g, const void* w, float* dense, cudaStream_t s);
