@@ -11,6 +11,23 @@ namespace toma {
 // written tile-major: row (b*P + p)*N_loc + l.  fp64 arithmetic so that the CPU
 // definition can be matched bit for bit.
 // ---------------------------------------------------------------------------
+// Eight consecutive elements as floats (16-byte aligned source).
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
+  const uint4 raw = *reinterpret_cast<const uint4*>(p);
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float2 f = __bfloat1622float2(h[e]);
+    v[2 * e] = f.x;
+    v[2 * e + 1] = f.y;
+  }
+}
+__device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
+  const float4 a = reinterpret_cast<const float4*>(p)[0], b = reinterpret_cast<const float4*>(p)[1];
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+  v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) quantise_kernel(const T* __restrict__ x, __nv_bfloat16* __restrict__ y, int B,
                                                        int N, int n_all, int d, int W, int th, int tw, int tiles_x,
@@ -26,17 +43,24 @@ __global__ void __launch_bounds__(256) quantise_kernel(const T* __restrict__ x, 
   const int l = (yy % th) * tw + xx % tw;
   const T* row = x + ((size_t)b * n_all + n) * d;
   __nv_bfloat16* out = y + ((size_t)(b * P + p) * Nloc + l) * d;
+  // eight channels (16 or 32 contiguous bytes) per lane and trip; dim is a multiple of 8
   double ss = 0.0;
-  for (int c = lane; c < d; c += 32) {
-    const double v = (double)to_f32(row[c]);
-    ss += v * v;
+  for (int c = lane * 8; c < d; c += 256) {
+    float v[8];
+    load8(row + c, v);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) ss += (double)v[e] * (double)v[e];
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
   const double scale = kCosScaleTimesOne / fmax(sqrt(ss), 1e-30);
-  for (int c = lane; c < d; c += 32) {
-    const double k = rint((double)to_f32(row[c]) * scale);
-    out[c] = __float2bfloat16_rn((float)k * (1.0f / 4096.0f));
+  for (int c = lane * 8; c < d; c += 256) {  // second read of the row: an L1/L2 hit
+    float v[8];
+    load8(row + c, v);
+    __align__(16) __nv_bfloat16 q[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) q[e] = __float2bfloat16_rn((float)rint((double)v[e] * scale) * (1.0f / 4096.0f));
+    *reinterpret_cast<uint4*>(out + c) = *reinterpret_cast<const uint4*>(q);
   }
 }
 
