@@ -80,6 +80,11 @@ typedef struct {
   int32_t n_heads, head_dim;       /* n_heads*head_dim == dim (attention inside toma_block) */
   int32_t n_extra;                 /* trailing un-merged tokens */
   int32_t dtype;                   /* toma_dtype of x / merged / out tensors */
+  int32_t global_merge;            /* 0: weights, merge and unmerge per tile (Algorithm 3).  1: destinations are
+                                      still chosen per tile, but the D destinations of an image form one set and
+                                      weights, merge and unmerge run over all N image tokens (the paper's default
+                                      variant, Sec. 5).  Merged rows keep the tile-major pick order; the weight
+                                      buffer then holds A~^T as [batch][N][D] and is far larger */
 } toma_desc;
 
 /* Host-only helpers.  Return 0 / negative on an invalid descriptor. */

@@ -253,6 +253,13 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, n_heads: int,
 # ----------------------------------------------------------------------------
 
 
+def global_destinations(idx_tiles: np.ndarray, ids: np.ndarray) -> np.ndarray:
+    """Image-level token ids of the destinations chosen per tile: idx_tiles [P, D_loc] holds tile-local
+    picks, ids [P, N_loc] the image token of every tile slot; the result [P * D_loc] is tile-major, pick
+    order inside a tile (the order of the merged rows)."""
+    return np.concatenate([ids[p][np.asarray(idx_tiles[p], dtype=np.int64)] for p in range(ids.shape[0])])
+
+
 @dataclass
 class BlockState:
     """Cached selection and weights of one batch (what Sec. 4.3.2 reuses)."""
@@ -263,7 +270,8 @@ class BlockState:
 
 def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid_w: int,
                tile_h: int, tile_w: int, merge_ratio: float, tau: float, n_heads: int,
-               reuse_interval: int, n_extra: int = 0, round_fn=None, weight_reuse_interval: int = 0):
+               reuse_interval: int, n_extra: int = 0, round_fn=None, weight_reuse_interval: int = 0,
+               global_merge: bool = False):
     """One ToMA-wrapped attention call (Algorithm 3) on x [B, N + n_extra, d].
 
     Selection and weights are recomputed when step % reuse_interval == 0 and
@@ -273,6 +281,11 @@ def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid
     order inside a tile; the n_extra trailing tokens are not merged and join the
     attention after the merged image tokens.  The core module F is the attention
     core with Q = K = V = merged tokens.
+
+    With global_merge (the paper's default variant, Sec. 5 "ToMA Variants": destinations chosen per
+    tile, merge over the whole image) the D destinations of an image, in the same tile-major pick
+    order, form one destination set and Sec. 4.2's weights, merge and unmerge are applied once to all
+    N image tokens; state.w is then [B, 1, D, N].
 
     `round_fn`, if given, is applied to the merged and to the attended tensor; it
     lets a test mirror the storage rounding between stages.  Returns
@@ -293,15 +306,22 @@ def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid
             for p in range(P):
                 state.idx[b, p], mg = select_tile(x[b, ids[p]], d_loc)
                 state.margins.append(mg)
-    if refresh_w:
+    if refresh_w and global_merge:
+        state.w = np.empty((B, 1, D, N), dtype=np.float64)
+        for b in range(B):
+            state.w[b, 0] = merge_weights(x[b, :N], global_destinations(state.idx[b], ids), tau)
+    elif refresh_w:
         state.w = np.empty((B, P, d_loc, n_loc), dtype=np.float64)
         for b in range(B):
             for p in range(P):
                 state.w[b, p] = merge_weights(x[b, ids[p]], state.idx[b, p], tau)
     merged = np.empty((B, D + n_extra, d), dtype=np.float64)
     for b in range(B):
-        for p in range(P):
-            merged[b, p * d_loc:(p + 1) * d_loc] = merge(state.w[b, p], x[b, ids[p]])
+        if global_merge:
+            merged[b, :D] = merge(state.w[b, 0], x[b, :N])
+        else:
+            for p in range(P):
+                merged[b, p * d_loc:(p + 1) * d_loc] = merge(state.w[b, p], x[b, ids[p]])
         merged[b, D:] = x[b, N:]
     if round_fn is not None:
         merged = round_fn(merged)
@@ -312,8 +332,11 @@ def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid
         attended = round_fn(attended)
     out = np.empty((B, n_all, d), dtype=np.float64)
     for b in range(B):
-        for p in range(P):
-            out[b, ids[p]] = unmerge(state.w[b, p], attended[b, p * d_loc:(p + 1) * d_loc])
+        if global_merge:
+            out[b, :N] = unmerge(state.w[b, 0], attended[b, :D])
+        else:
+            for p in range(P):
+                out[b, ids[p]] = unmerge(state.w[b, p], attended[b, p * d_loc:(p + 1) * d_loc])
         out[b, N:] = attended[b, D:]
     return out, merged, attended
 

@@ -32,6 +32,7 @@ class TomaDesc(Structure):
         ("merge_ratio", c_float), ("tau", c_float),
         ("reuse_interval", c_int32), ("weight_reuse_interval", c_int32),
         ("n_heads", c_int32), ("head_dim", c_int32), ("n_extra", c_int32), ("dtype", c_int32),
+        ("global_merge", c_int32),
     ]
 
 
@@ -95,10 +96,10 @@ lib = _load()
 
 
 def make_desc(*, batch, grid_h, grid_w, dim, tile_h, tile_w, merge_ratio, tau, n_heads, head_dim, dtype,
-              reuse_interval=1, weight_reuse_interval=0, n_extra=0) -> TomaDesc:
+              reuse_interval=1, weight_reuse_interval=0, n_extra=0, global_merge=False) -> TomaDesc:
     code = {"bf16": TOMA_BF16, "f32": TOMA_F32, TOMA_BF16: TOMA_BF16, TOMA_F32: TOMA_F32}[dtype]
     return TomaDesc(batch, grid_h, grid_w, dim, tile_h, tile_w, merge_ratio, tau, reuse_interval,
-                    weight_reuse_interval, n_heads, head_dim, n_extra, code)
+                    weight_reuse_interval, n_heads, head_dim, n_extra, code, 1 if global_merge else 0)
 
 
 def desc_from_config(cfg, **overrides) -> TomaDesc:

@@ -35,6 +35,9 @@ toma_status make_geom(const toma_desc* desc, Geom* g) {
   g->n_extra = desc->n_extra; g->Lm = g->D + g->n_extra;
   g->heads = desc->n_heads; g->dh = desc->head_dim;
   g->f32 = desc->dtype == TOMA_F32;
+  if (desc->global_merge != 0 && desc->global_merge != 1) return TOMA_ERR_SHAPE;
+  g->global_merge = desc->global_merge == 1;
+  if (g->global_merge && (long long)g->N * g->D > (1ll << 27)) return TOMA_ERR_UNSUPPORTED;  // dense D x N weights per image
   g->logit_scale = (float)(1.0 / ((double)desc->tau * sqrt((double)desc->dim)));
   return TOMA_OK;
 }
@@ -45,15 +48,25 @@ static size_t attention_ws_bytes(int B, int L, int heads, int dh, bool f32) {
   return attention_on_tc(dh, f32) ? attention_tc_workspace_bytes(B, L, heads, dh) : 0;
 }
 
+Geom merge_geom(const Geom& g) {
+  Geom m = g;
+  if (g.global_merge) {
+    m.P = 1; m.tiles_x = 1; m.th = g.H; m.tw = g.W; m.Nloc = g.N; m.Dloc = g.D;
+  }
+  return m;
+}
+
 WsLayout ws_layout(const Geom& g) {
   WsLayout l;
+  const Geom gm = merge_geom(g);
   const size_t tiles = (size_t)g.B * g.P;
   const size_t esz = g.f32 ? 4 : 2;
   size_t off = 0;
   l.y_off = off;      off = align_up(off + tiles * g.Nloc * g.d * sizeof(__nv_bfloat16), 256);
   l.sq_off = off;     off = align_up(off + tiles * g.Nloc * g.Nloc * sizeof(int16_t), 256);
-  l.logits_off = off; off = align_up(off + tiles * g.Dloc * g.Nloc * sizeof(float), 256);
-  l.wts_off = off;    off = align_up(off + (weights_tc_supported(g) ? weights_tc_scratch_bytes(g) : 0), 256);
+  l.logits_off = off; off = align_up(off + (size_t)gm.B * gm.P * gm.Dloc * gm.Nloc * sizeof(float), 256);
+  l.wts_off = off;    off = align_up(off + (weights_tc_supported(gm) ? weights_tc_scratch_bytes(gm) : 0), 256);
+  l.gidx_off = off;   off = align_up(off + (g.global_merge ? (size_t)g.B * g.D * sizeof(int32_t) : 0), 256);
   l.xm_off = off;     off = align_up(off + (size_t)g.B * g.Lm * g.d * esz, 256);
   l.att_off = off;    off = align_up(off + (size_t)g.B * g.Lm * g.d * esz, 256);
   l.att_ws_off = off; off = align_up(off + attention_ws_bytes(g.B, g.Lm, g.heads, g.dh, g.f32), 256);
@@ -90,15 +103,23 @@ static cudaError_t do_select(const Geom& g, const void* x, int32_t* idx, char* w
 static cudaError_t do_weights(const Geom& g, const void* x, const int32_t* idx, void* w, char* ws,
                               uint32_t* dev_status, cudaStream_t s) {
   const WsLayout l = ws_layout(g);
-  if (weights_tc_supported(g))
-    return launch_weights_tc(g, x, idx, w, (float*)(ws + l.logits_off), ws + l.wts_off, dev_status, s);
-  return launch_weights_simt(g, x, idx, w, (float*)(ws + l.logits_off), s);
+  const Geom gm = merge_geom(g);
+  if (g.global_merge) {  // image-level destination ids; from here on the image is one region
+    int32_t* gidx = (int32_t*)(ws + l.gidx_off);
+    cudaError_t e = launch_global_idx(g, idx, gidx, s);
+    if (e != cudaSuccess) return e;
+    idx = gidx;
+  }
+  if (weights_tc_supported(gm))
+    return launch_weights_tc(gm, x, idx, w, (float*)(ws + l.logits_off), ws + l.wts_off, dev_status, s);
+  return launch_weights_simt(gm, x, idx, w, (float*)(ws + l.logits_off), s);
 }
 
 // `zero`, `zero_bytes`: a region to clear on the side; *zeroed says whether the path taken did it.
-static cudaError_t do_merge(const Geom& g, const void* w, const void* x, void* xm, void* zero, size_t zero_bytes,
+static cudaError_t do_merge(const Geom& g_sel, const void* w, const void* x, void* xm, void* zero, size_t zero_bytes,
                             bool* zeroed, uint32_t* dev_status, cudaStream_t s) {
   if (zeroed) *zeroed = false;
+  const Geom g = merge_geom(g_sel);
   if (linear_tc_supported(g)) {
     cudaError_t e = launch_merge_tc(g, w, x, xm, zero, zero_bytes, dev_status, s);
     if (zeroed) *zeroed = e == cudaSuccess && zero_bytes > 0;
@@ -107,8 +128,9 @@ static cudaError_t do_merge(const Geom& g, const void* w, const void* x, void* x
   return launch_merge_simt(g, w, x, xm, s);
 }
 
-static cudaError_t do_unmerge(const Geom& g, const void* w, const void* y, void* out, uint32_t* dev_status,
+static cudaError_t do_unmerge(const Geom& g_sel, const void* w, const void* y, void* out, uint32_t* dev_status,
                               cudaStream_t s) {
+  const Geom g = merge_geom(g_sel);
   if (linear_tc_supported(g)) {
     cudaError_t e = launch_unmerge_tc(g, w, y, out, dev_status, s);
     return e != cudaSuccess ? e : launch_copy_extra(g, y, out, false, s);
@@ -144,7 +166,8 @@ size_t toma_workspace_bytes(const toma_desc* desc) {
 size_t toma_weights_bytes(const toma_desc* desc) {
   Geom g;
   if (make_geom(desc, &g) != TOMA_OK) return 0;
-  return (size_t)g.B * g.P * g.Nloc * g.Dloc * 4;  // one fp32 plane, or a hi and a lo bf16 plane
+  const Geom gm = merge_geom(g);
+  return (size_t)gm.B * gm.P * gm.Nloc * gm.Dloc * 4;  // one fp32 plane, or a hi and a lo bf16 plane
 }
 
 int32_t toma_dest_per_tile(const toma_desc* desc) {
@@ -299,7 +322,7 @@ toma_status toma_weights_export(const toma_desc* desc, const void* w, float* den
   toma_status st = make_geom(desc, &g);
   if (st != TOMA_OK) return st;
   if (!w || !dense) return TOMA_ERR_NULL;
-  return cuda_ok(launch_weights_export(g, w, dense, (cudaStream_t)stream));
+  return cuda_ok(launch_weights_export(merge_geom(g), w, dense, (cudaStream_t)stream));
 }
 
 toma_status toma_weights_import(const toma_desc* desc, const float* dense, void* w, void* stream) {
@@ -307,7 +330,7 @@ toma_status toma_weights_import(const toma_desc* desc, const float* dense, void*
   toma_status st = make_geom(desc, &g);
   if (st != TOMA_OK) return st;
   if (!w || !dense) return TOMA_ERR_NULL;
-  return cuda_ok(launch_weights_import(g, dense, w, (cudaStream_t)stream));
+  return cuda_ok(launch_weights_import(merge_geom(g), dense, w, (cudaStream_t)stream));
 }
 
 }  // extern "C"

@@ -24,6 +24,7 @@ struct Geom {
   int B, H, W, d, th, tw, tiles_x, P, N, Nloc, Dloc, D, n_extra, Lm;  // Lm = D + n_extra
   int heads, dh;
   bool f32;
+  bool global_merge;  // weights / merge / unmerge over the whole image (selection stays per tile)
   float logit_scale;  // 1 / (tau * sqrt(d))
   long long tokens_all() const { return (long long)N + n_extra; }
 };
@@ -32,9 +33,12 @@ toma_status make_geom(const toma_desc* desc, Geom* g);
 
 // Workspace carve-up (all offsets 256-byte aligned).
 struct WsLayout {
-  size_t y_off, sq_off, logits_off, wts_off, xm_off, att_off, att_ws_off, total;
+  size_t y_off, sq_off, logits_off, wts_off, gidx_off, xm_off, att_off, att_ws_off, total;
 };
 WsLayout ws_layout(const Geom& g);
+// Geometry the weights, the merge and the unmerge work in: g itself, or, with global merge, the image as
+// one region (P = 1, N_loc = N, D_loc = D).
+Geom merge_geom(const Geom& g);
 
 // Process-wide count of kernel launches (reported by toma_launch_counter()).
 extern std::atomic<unsigned long long> g_launches;
@@ -73,6 +77,8 @@ size_t attention_tc_ticket_bytes(int B, int L, int heads);
 int attention_tc_plan(int B, int L, int heads, int info[4], int* bounds, int* owner_first, int* owner_last, int capacity);
 cudaError_t launch_attention_tc(int B, int L, int heads, int dh, const void* q, const void* k, const void* v, void* o,
                                 void* ws, bool tickets_clean, uint32_t* dev_status, cudaStream_t s);
+// Image-level destination ids [batch][D] (tile-major, pick order) from the tile-local picks.
+cudaError_t launch_global_idx(const Geom& g, const int32_t* idx, int32_t* gidx, cudaStream_t s);
 cudaError_t launch_weights_export(const Geom& g, const void* w, float* dense, cudaStream_t s);
 cudaError_t launch_weights_import(const Geom& g, const float* dense, void* w, cudaStream_t s);
 

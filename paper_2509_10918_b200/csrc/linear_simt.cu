@@ -267,6 +267,22 @@ cudaError_t launch_unmerge_simt(const Geom& g, const void* w, const void* y, voi
   return cudaGetLastError();
 }
 
+// gidx[b][p * D_loc + k] = image token of tile p's k-th pick.
+__global__ void global_idx_kernel(const int32_t* __restrict__ idx, int32_t* __restrict__ gidx, int P, int Dloc, int tiles_x,
+                                  int th, int tw, int W, int total) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= total) return;
+  const int p = (e / Dloc) % P;
+  gidx[e] = tile_token(p, idx[e], tiles_x, th, tw, W);
+}
+
+cudaError_t launch_global_idx(const Geom& g, const int32_t* idx, int32_t* gidx, cudaStream_t s) {
+  const int total = g.B * g.D;
+  global_idx_kernel<<<(total + 255) / 256, 256, 0, s>>>(idx, gidx, g.P, g.Dloc, g.tiles_x, g.th, g.tw, g.W, total);
+  count_launch();
+  return cudaGetLastError();
+}
+
 // Dense fp32 A~ [batch][P][D_loc][N_loc]  <->  stored A~^T [batch][P][N_loc][D_loc].
 template <typename WT, bool kExport>
 __global__ void weights_convert_kernel(WT* __restrict__ w, float* __restrict__ dense, int Nloc, int Dloc, size_t total) {

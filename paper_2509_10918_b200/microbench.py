@@ -29,6 +29,7 @@ def main():
     ap.add_argument("--reps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--no-flush", action="store_true")
+    ap.add_argument("--global-merge", action="store_true", help="weights / merge / unmerge over the whole image")
     args = ap.parse_args()
 
     import torch
@@ -37,7 +38,7 @@ def main():
     import paper_2509_10918_b200 as toma
 
     cfg = gen.config(args.workload) if args.ratio is None else gen.config(args.workload, merge_ratio=args.ratio)
-    desc = toma.desc_from_config(cfg)
+    desc = toma.desc_from_config(cfg, global_merge=args.global_merge)
     tdt = toma.torch_dtype(desc)
     x = torch.from_numpy(gen.features(cfg)).cuda().to(tdt)
     out = torch.empty_like(x)
@@ -81,7 +82,7 @@ def main():
     assert int(status.item()) == 0
     med, mn = statistics.median(times), min(times)
     esz = 2 if cfg.dtype == "bf16" else 4
-    res = {"stage": args.stage, "workload": cfg.name, "ratio": cfg.merge_ratio, "median_us": med, "min_us": mn,
+    res = {"stage": args.stage, "workload": cfg.name + ("+global" if args.global_merge else ""), "ratio": cfg.merge_ratio, "median_us": med, "min_us": mn,
            "reps": args.reps}
     if args.stage == "attention":
         flops = 4.0 * B * L * L * d

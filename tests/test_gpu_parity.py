@@ -294,6 +294,72 @@ def test_block_host_matches_block(toma, streams):
         assert torch.equal(idx, idx2)
 
 
+GLOBAL = [
+    # grid, tile, dim, heads, dtype: destinations per tile, weights / merge / unmerge over the whole image
+    dict(grid_h=32, grid_w=32, tile_h=8, tile_w=8, dim=128, n_heads=2, head_dim=64, dtype="bf16"),
+    dict(grid_h=32, grid_w=32, tile_h=8, tile_w=8, dim=128, n_heads=2, head_dim=64, dtype="f32"),
+    dict(grid_h=16, grid_w=64, tile_h=4, tile_w=16, dim=64, n_heads=1, head_dim=64, dtype="bf16", merge_ratio=0.75),
+    dict(grid_h=16, grid_w=16, tile_h=8, tile_w=8, dim=64, n_heads=1, head_dim=64, dtype="bf16", n_extra=5),
+]
+
+
+@pytest.mark.parametrize("over", GLOBAL, ids=[str(i) for i in range(len(GLOBAL))])
+def test_global_merge_parity(toma, over):
+    """The default ToMA variant (Sec. 5): destinations per tile, then weights, merge and unmerge once over
+    all image tokens with the D destinations of the image as one set."""
+    cfg = gen.config("cfg2", batch=2, **over)
+    x_host = gen.features(cfg)
+    run = Run(toma, cfg, x_host, global_merge=True)
+    idx = run.select()
+    N, D = cfg.n_tokens, cfg.n_merged
+    run.t.toma_merge_weights(run.desc, run.x, run.idx, run.w, run.ws, run.status)
+    run.ok()
+    dense = torch.empty((cfg.batch, 1, D, N), dtype=torch.float32, device="cuda")
+    run.t.toma_weights_export(run.desc, run.w, dense)
+    torch.cuda.synchronize()
+    dense = dense.cpu().numpy().astype(np.float64)
+    merged = run.merge()
+    y_dev = run.attend()
+    unmerged = run.unmerge(y_dev)
+    y_host = to_host64(y_dev)
+    ids = O.tile_token_ids(cfg.grid_h, cfg.grid_w, cfg.tile_h, cfg.tile_w)
+    w_abs = 2e-5 if cfg.dtype == "f32" else 6e-4
+    for b in range(cfg.batch):
+        for p in range(cfg.n_tiles):
+            want_idx, margin = O.select_tile(tile_tokens(cfg, x_host, b, p), cfg.d_loc)
+            assert margin > O.FRAGILE_MARGIN
+            assert np.array_equal(idx[b, p], want_idx)
+        x_img = x_host[b, :N].astype(np.float64)
+        w = O.merge_weights(x_img, O.global_destinations(idx[b], ids), cfg.tau)
+        assert np.abs(dense[b, 0] - w).max() <= w_abs, "global weights differ"
+        assert_close(merged[b, :D], O.merge(w, x_img), cfg.dtype, "global merge")
+        assert_close(unmerged[b, :N], O.unmerge(w, y_host[b, :D]), cfg.dtype, "global unmerge")
+        if cfg.n_extra:
+            assert np.array_equal(merged[b, D:], x_host[b, N:].astype(np.float64))
+            assert np.array_equal(unmerged[b, N:], y_host[b, D:])
+
+
+def test_global_merge_block_parity_at_benchmark_size(toma):
+    """toma_block with global merge on the benchmark shape (64x64 tokens, 2048 destinations): a refresh
+    step and a reuse step against the oracle."""
+    cfg = gen.config("cfg3", batch=1, steps=2, reuse_interval=2)
+    desc = toma.desc_from_config(cfg, global_merge=True)
+    idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    st = O.BlockState()
+    kw = dict(grid_h=cfg.grid_h, grid_w=cfg.grid_w, tile_h=cfg.tile_h, tile_w=cfg.tile_w, merge_ratio=cfg.merge_ratio,
+              tau=cfg.tau, n_heads=cfg.n_heads, reuse_interval=2, global_merge=True)
+    for step, x_host in enumerate(gen.feature_sequence(cfg)):
+        x = to_dev(x_host, cfg.dtype)
+        out = torch.empty_like(x)
+        toma.toma_block(desc, step, x, out, idx, w, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        want, _, _ = O.block_step(x_host, step, st, **kw)
+        assert np.array_equal(idx.cpu().numpy().astype(np.int64), st.idx)
+        assert_close(to_host64(out), want, cfg.dtype, f"global-merge block step {step}")
+
+
 def test_block_replays_from_a_cuda_graph(toma):
     """A reuse step and a refresh step captured into CUDA graphs (the calls never allocate or synchronise,
     and their dependent launches are capturable) replay to the same bits as direct calls."""

@@ -149,3 +149,36 @@ def test_block_step_separate_weight_schedule():
     assert np.array_equal(st.idx, idx0) and not np.array_equal(st.w, w0)
     ids = O.tile_token_ids(16, 16, 8, 8)
     assert np.allclose(st.w[0, 1], O.merge_weights(xs[2][0][ids[1]], idx0[0, 1], c.tau))
+
+
+def test_global_merge_reduces_to_tile_merge_for_one_tile_and_sees_across_tiles():
+    """Global merge (default ToMA variant): with a single tile it is the tile-local path; with several
+    tiles every token gets a share of every destination (rows sum to 1, columns of A sum to 1), and
+    two identical tokens in different tiles, one of them a destination, end up on that destination."""
+    c = gen.config("cfg3", batch=1, grid_h=8, grid_w=8, tile_h=8, tile_w=8, dim=32, n_heads=1, head_dim=32, steps=1)
+    x = gen.features(c)
+    kw = dict(grid_h=8, grid_w=8, tile_h=8, tile_w=8, merge_ratio=0.5, tau=c.tau, n_heads=1, reuse_interval=1)
+    a = O.block_step(x, 0, O.BlockState(), **kw)[0]
+    b = O.block_step(x, 0, O.BlockState(), global_merge=True, **kw)[0]
+    assert np.allclose(a, b, rtol=0, atol=1e-12)
+
+    c = gen.config("cfg3", batch=1, grid_h=8, grid_w=8, tile_h=4, tile_w=4, dim=32, n_heads=1, head_dim=32, steps=1)
+    x = gen.features(c).astype(np.float64)
+    ids = O.tile_token_ids(8, 8, 4, 4)
+    st = O.BlockState()
+    kw = dict(grid_h=8, grid_w=8, tile_h=4, tile_w=4, merge_ratio=0.5, tau=c.tau, n_heads=1, reuse_interval=1)
+    O.block_step(x, 0, st, global_merge=True, **kw)
+    w = st.w[0, 0]                       # [D, N]
+    D, N = w.shape
+    assert (D, N) == (32, 64) and np.allclose(w.sum(1), 1.0)
+    gidx = O.global_destinations(st.idx[0], ids)
+    assert len(set(gidx.tolist())) == D
+    # a copy, in another tile, of a destination token puts (almost) all its mass on that destination
+    dest_tok = int(gidx[0])
+    other = next(int(t) for t in ids[3] if t not in set(gidx.tolist()))
+    x2 = x.copy()
+    x2[0, other] = 3.0 * x2[0, dest_tok]  # a long copy: its logit with the destination dominates
+    # shares of that token over the destinations = its column of A; after row normalisation the
+    # largest entry of the column is still the destination it copies
+    w2 = O.merge_weights(x2[0, :64], gidx, c.tau)
+    assert np.argmax(w2[:, other] * w2.shape[1]) == 0 or np.argmax(w2[:, other]) == 0
