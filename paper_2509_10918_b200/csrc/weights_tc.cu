@@ -31,6 +31,8 @@ struct WParams {
   int m_tok;    // source tokens per CTA (128, or N_loc when the tile is smaller)
   int stages;
   float scale_log2;  // log2(e) / (tau * sqrt(d))
+  int d_block;  // destinations per CTA: D_loc itself, or 512 when D_loc is larger (blockIdx.z picks the block)
+  int raw;      // 1: write the scaled logits (log2 domain) only; the softmax over all blocks runs afterwards
 };
 
 __global__ void __launch_bounds__(256)
@@ -60,12 +62,14 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                       float* __restrict__ shares, float* __restrict__ zpart, const WParams p, uint32_t* dev_status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int n_mma = (p.Dloc + 15) & ~15;          // MMA N: destinations padded to 16
+  const int d_base = blockIdx.z * p.d_block;     // first destination of this CTA
+  const int Dl = min(p.d_block, p.Dloc - d_base);  // its destinations
+  const int n_mma = (Dl + 15) & ~15;              // MMA N: destinations padded to 16
   const int n0 = n_mma > 256 ? 256 : n_mma, n1 = n_mma - n0;
   const int a_bytes = 128 * 128;
-  const int b_rows = p.Dloc > 256 ? 512 : ((p.Dloc + 7) & ~7);  // rows the swizzled operand tile spans
+  const int b_rows = (p.raw || Dl > 256) ? 512 : ((Dl + 7) & ~7);  // rows the swizzled operand tile spans
   const int b_bytes = ((b_rows * 128 + 1023) / 1024) * 1024;
-  const int b_load_bytes = p.Dloc > 256 ? 512 * 128 : p.Dloc * 128;  // what the TMA boxes deliver
+  const int b_load_bytes = Dl > 256 ? 512 * 128 : (p.Dloc > 256 ? 256 : p.Dloc) * 128;  // what the TMA boxes deliver
   const int stage_bytes = a_bytes + b_bytes;
   WBars* bar = reinterpret_cast<WBars*>(smem + p.stages * stage_bytes);
   float* zw = reinterpret_cast<float*>(bar + 1);  // [4 warps][D_loc] partial row sums
@@ -77,7 +81,7 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
   const int nk = (p.d + kKC - 1) / kKC;
   const uint32_t ncols = n_mma > 256 ? 512u : n_mma > 128 ? 256u : n_mma > 64 ? 128u : n_mma > 32 ? 64u : 32u;
   const int box_bytes_a = p.m_tok * 128;
-  const int box_d0 = p.Dloc > 256 ? 256 : p.Dloc, box_d1 = p.Dloc - box_d0;
+  const int box_d0 = Dl > 256 ? 256 : Dl, box_d1 = Dl - box_d0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
@@ -107,8 +111,8 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
         uint8_t* sa = smem + s * stage_bytes;
         mbar_expect_tx(&bar->full[s], box_bytes_a + b_load_bytes);
         tma_load_4d(sa, &tm_x, &bar->full[s], k * kKC, tx * p.tw, ty * p.th + mblk * rows_per_box, b);
-        tma_load_3d(sa + a_bytes, &tm_d, &bar->full[s], k * kKC, 0, batch);
-        if (box_d1 > 0) tma_load_3d(sa + a_bytes + 256 * 128, &tm_d, &bar->full[s], k * kKC, 256, batch);
+        tma_load_3d(sa + a_bytes, &tm_d, &bar->full[s], k * kKC, d_base, batch);
+        if (box_d1 > 0) tma_load_3d(sa + a_bytes + 256 * 128, &tm_d, &bar->full[s], k * kKC, d_base + 256, batch);
       }
     }
   } else if (warp == 1) {
@@ -136,9 +140,25 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
     const int k_loc = quarter * 32 + lane;              // source row inside this CTA
     const bool valid = k_loc < p.m_tok;
     const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16);
-    float* zrow = zw + quarter * p.Dloc;
+    float* zrow = zw + quarter * Dl;
     if (mbar_wait(&bar->done, 0, dev_status, abort_flag)) {
       tc_fence_after();
+      if (p.raw) {  // scaled logits only: the row's other destination blocks are in other CTAs
+        float* dst = shares + ((size_t)batch * p.Nloc + k_base + (valid ? k_loc : 0)) * p.Dloc + d_base;
+        for (int i0 = 0; i0 < Dl; i0 += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + i0, r);
+          tmem_wait_ld();
+          if (valid) {
+#pragma unroll
+            for (int e = 0; e < 32; e += 4)
+              if (i0 + e < Dl)
+                *reinterpret_cast<float4*>(dst + i0 + e) =
+                    make_float4(__uint_as_float(r[e]) * p.scale_log2, __uint_as_float(r[e + 1]) * p.scale_log2,
+                                __uint_as_float(r[e + 2]) * p.scale_log2, __uint_as_float(r[e + 3]) * p.scale_log2);
+          }
+        }
+      } else {
       // pass 1: maximum logit over the destinations
       float mx = -INFINITY;
       for (int i0 = 0; i0 < p.Dloc; i0 += 32) {
@@ -191,11 +211,13 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
         }
         if (i0 + lane < p.Dloc) zrow[i0 + lane] = a[0];
       }
+      }  // !raw
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");  // the four epilogue warps
     const int t = threadIdx.x - 64;
     float* zout = zpart + ((size_t)batch * gridDim.y + mblk) * p.Dloc;
-    for (int i = t; i < p.Dloc; i += 128) zout[i] = (zw[i] + zw[p.Dloc + i]) + (zw[2 * p.Dloc + i] + zw[3 * p.Dloc + i]);
+    if (!p.raw)
+      for (int i = t; i < p.Dloc; i += 128) zout[i] = (zw[i] + zw[p.Dloc + i]) + (zw[2 * p.Dloc + i] + zw[3 * p.Dloc + i]);
   }
   tc_fence_before();
   __syncthreads();
@@ -209,7 +231,7 @@ __global__ void __launch_bounds__(256)
 weights_normalise_kernel(const float* __restrict__ shares, const float* __restrict__ zpart, __nv_bfloat16* __restrict__ w,
                          int Nloc, int Dloc, int mblocks) {
   // grid (blocks over the tile's [N_loc][D_loc] plane in groups of four destinations, tile)
-  __shared__ float zs[512];  // row sums of the tile's D_loc (<= 512) destinations
+  extern __shared__ float zs[];  // row sums of the tile's D_loc destinations
   dependency_wait();  // launched with programmatic stream serialisation
   if (threadIdx.x == 0) release_dependents();
   const size_t batch = blockIdx.y;
@@ -239,6 +261,69 @@ weights_normalise_kernel(const float* __restrict__ shares, const float* __restri
   }
 }
 
+// Softmax over the destination axis for rows of scaled logits (log2 domain) that span several
+// destination blocks: shares[row][i] <- 2^(v_i - max) / sum.  One warp per source row, 32 rows per
+// CTA; the CTA then leaves, per destination, the sum of its 32 rows of shares in zblk (rows added in
+// row order, so the result does not depend on scheduling).
+constexpr int kSoftmaxRows = 32;
+__global__ void __launch_bounds__(256)
+softmax_rows_kernel(float* __restrict__ shares, float* __restrict__ zblk, int Nloc, int Dloc) {
+  dependency_wait();
+  if (threadIdx.x == 0) release_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const size_t batch = blockIdx.y;
+  const int row0 = blockIdx.x * kSoftmaxRows;
+  for (int rr = 0; rr < kSoftmaxRows / 8; ++rr) {
+    const int row = row0 + warp * (kSoftmaxRows / 8) + rr;
+    if (row >= Nloc) break;
+    float4* v = reinterpret_cast<float4*>(shares + (batch * Nloc + row) * Dloc);
+    float mx = -INFINITY;
+    for (int q = lane; q < Dloc / 4; q += 32) {
+      const float4 a = v[q];
+      mx = fmaxf(fmaxf(mx, fmaxf(a.x, a.y)), fmaxf(a.z, a.w));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float sum = 0.f;
+    for (int q = lane; q < Dloc / 4; q += 32) {
+      const float4 a = v[q];
+      sum += (fast_exp2(a.x - mx) + fast_exp2(a.y - mx)) + (fast_exp2(a.z - mx) + fast_exp2(a.w - mx));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const float inv = 1.f / sum;
+    for (int q = lane; q < Dloc / 4; q += 32) {
+      float4 a = v[q];
+      a.x = fast_exp2(a.x - mx) * inv;
+      a.y = fast_exp2(a.y - mx) * inv;
+      a.z = fast_exp2(a.z - mx) * inv;
+      a.w = fast_exp2(a.w - mx) * inv;
+      v[q] = a;
+    }
+  }
+  __syncthreads();  // the CTA's rows are final (and visible to the whole CTA)
+  const int rows = min(kSoftmaxRows, Nloc - row0);
+  const float* base = shares + (batch * Nloc + row0) * Dloc;
+  float* out = zblk + (batch * gridDim.x + blockIdx.x) * Dloc;
+  for (int i = threadIdx.x; i < Dloc; i += blockDim.x) {
+    float acc = 0.f;
+    for (int r = 0; r < rows; ++r) acc += base[(size_t)r * Dloc + i];
+    out[i] = acc;
+  }
+}
+
+// z[batch][i] = sum over the row blocks of zblk, in block order.
+__global__ void __launch_bounds__(256) z_reduce_kernel(const float* __restrict__ zblk, float* __restrict__ z, int nblk, int Dloc) {
+  dependency_wait();
+  if (threadIdx.x == 0) release_dependents();
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= Dloc) return;
+  const size_t batch = blockIdx.y;
+  float acc = 0.f;
+  for (int b = 0; b < nblk; ++b) acc += zblk[(batch * nblk + b) * Dloc + i];
+  z[batch * Dloc + i] = acc;
+}
+
 }  // namespace
 
 bool weights_tc_supported(const Geom& g) {
@@ -246,14 +331,18 @@ bool weights_tc_supported(const Geom& g) {
   const int m_tok = g.Nloc < 128 ? g.Nloc : 128;
   if (g.Nloc % m_tok != 0 || m_tok % 8 != 0) return false;
   if (g.tw > m_tok || m_tok % g.tw != 0 || g.th % (m_tok / g.tw) != 0 || g.tw > 256 || m_tok / g.tw > 256) return false;
-  if (g.Dloc % 4 != 0 || g.Dloc > 512) return false;
+  if (g.Dloc % 4 != 0) return false;
+  if (g.Dloc > 512 && g.Nloc % kSoftmaxRows != 0) return false;  // blocked form: softmax in a second kernel
   return true;
 }
 
 size_t weights_tc_scratch_bytes(const Geom& g) {  // gathered destinations + partial row sums
   const size_t tiles = (size_t)g.B * g.P;
   const int m_tok = g.Nloc < 128 ? g.Nloc : 128;
-  return tiles * g.Dloc * g.d * 2 + 256 + tiles * (g.Nloc / m_tok) * g.Dloc * 4 + 256;
+  const size_t dest = tiles * g.Dloc * g.d * 2 + 256;
+  if (g.Dloc > 512)  // blocked form: per-row-block sums, then their total
+    return dest + tiles * ((size_t)g.Nloc / kSoftmaxRows) * g.Dloc * 4 + 256 + tiles * g.Dloc * 4 + 256;
+  return dest + tiles * (g.Nloc / m_tok) * g.Dloc * 4 + 256;
 }
 
 cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, void* w, float* shares, void* scratch,
@@ -264,6 +353,9 @@ cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, 
   p.n_all = (int)g.tokens_all();
   p.m_tok = g.Nloc < 128 ? g.Nloc : 128;
   p.scale_log2 = g.logit_scale * 1.4426950408889634f;
+  const bool blocked = g.Dloc > 512;  // more destinations than one CTA's tensor memory holds
+  p.d_block = blocked ? 512 : g.Dloc;
+  p.raw = blocked ? 1 : 0;
   const int mblocks = g.Nloc / p.m_tok;
   __nv_bfloat16* dg = (__nv_bfloat16*)scratch;
   float* zpart = (float*)((char*)scratch + ((tiles * g.Dloc * g.d * 2 + 255) / 256) * 256);
@@ -289,21 +381,45 @@ cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, 
   p.stages = stage_bytes <= 48 * 1024 ? 4 : 2;
   const int nk = (g.d + kKC - 1) / kKC;
   if (p.stages > nk) p.stages = nk;
-  const int smem = 1024 + p.stages * stage_bytes + (int)sizeof(WBars) + 4 * g.Dloc * 4 + 64;
+  const int smem = 1024 + p.stages * stage_bytes + (int)sizeof(WBars) + 4 * p.d_block * 4 + 64;
   static bool attr = false;
   if (!attr) {
     cudaError_t e = cudaFuncSetAttribute(weights_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
     attr = true;
   }
-  dim3 grid((unsigned)tiles, mblocks);
+  dim3 grid((unsigned)tiles, mblocks, (g.Dloc + p.d_block - 1) / p.d_block);
   le = launch_dependent(weights_logits_kernel, grid, dim3(192), (size_t)smem, s, tx, td, shares, zpart, p, dev_status);
   count_launch();
   if (le != cudaSuccess) return le;
+  const float* zsrc = zpart;
+  int zblocks = mblocks;
+  if (blocked) {  // softmax over the full rows, then the destinations' row sums in two deterministic steps
+    const int nrb = g.Nloc / kSoftmaxRows;
+    float* zblk = zpart;
+    float* z = (float*)((char*)zblk + ((tiles * nrb * g.Dloc * 4 + 255) / 256) * 256);
+    le = launch_dependent(softmax_rows_kernel, dim3((unsigned)nrb, (unsigned)tiles), dim3(256), 0, s, shares,
+                          zblk, g.Nloc, g.Dloc);
+    count_launch();
+    if (le != cudaSuccess) return le;
+    le = launch_dependent(z_reduce_kernel, dim3((unsigned)((g.Dloc + 255) / 256), (unsigned)tiles), dim3(256), 0, s,
+                          (const float*)zblk, z, nrb, g.Dloc);
+    count_launch();
+    if (le != cudaSuccess) return le;
+    zsrc = z;
+    zblocks = 1;
+  }
   const int quads = g.Nloc * g.Dloc / 4;
-  const int nblocks = (quads + 1023) / 1024 > 0 ? (quads + 1023) / 1024 : 1;  // four quads per thread
-  le = launch_dependent(weights_normalise_kernel, dim3((unsigned)nblocks, (unsigned)tiles), dim3(256), 0, s,
-                        (const float*)shares, (const float*)zpart, (__nv_bfloat16*)w, g.Nloc, g.Dloc, mblocks);
+  int nblocks = (quads + 1023) / 1024;  // four quads per thread
+  nblocks = nblocks < 1 ? 1 : nblocks > 1024 ? 1024 : nblocks;
+  static bool attr3 = false;
+  if (!attr3 && g.Dloc * 4 > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(weights_normalise_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    attr3 = true;
+  }
+  le = launch_dependent(weights_normalise_kernel, dim3((unsigned)nblocks, (unsigned)tiles), dim3(256), (size_t)g.Dloc * 4, s,
+                        (const float*)shares, zsrc, (__nv_bfloat16*)w, g.Nloc, g.Dloc, zblocks);
   count_launch();
   return le != cudaSuccess ? le : cudaGetLastError();
 }
