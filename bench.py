@@ -185,12 +185,15 @@ def other_workloads(toma, torch, flush, peaks):
     # cfg2 states no schedule: the paper's weight interval (5) is used.  cfg4 (Flux) does not reuse across
     # timesteps but shares one selection among the blocks of a kind within a step (19 joint blocks).
     # cfg3_stripes: the same tokens cut into stripes of 4 full rows (256 tokens per region, as a 16x16 tile) under
-    # the paper's own schedule, destinations every 10 steps and weights every 5.
+    # the paper's own schedule, destinations every 10 steps and weights every 5.  cfg3_global_merge: the paper's
+    # default variant (destinations per 16x16 tile, one dense 2048 x 4096 weight matrix per image), same schedule.
     for label, name, over, reuse, w_reuse in (("cfg2", "cfg2", {}, 5, 0), ("cfg4", "cfg4", {}, 19, 0),
                                               ("cfg5a", "cfg5a", {}, 5, 0),
-                                              ("cfg3_stripes", "cfg3", dict(tile_h=4, tile_w=64), 10, 5)):
+                                              ("cfg3_stripes", "cfg3", dict(tile_h=4, tile_w=64), 10, 5),
+                                              ("cfg3_global_merge", "cfg3", dict(global_merge=True), 10, 5)):
+        global_merge = over.pop("global_merge", False) if isinstance(over, dict) else False
         cfg = gen.config(name, reuse_interval=reuse, **over)
-        desc = toma.desc_from_config(cfg, weight_reuse_interval=w_reuse)
+        desc = toma.desc_from_config(cfg, weight_reuse_interval=w_reuse, global_merge=global_merge)
         tdt = toma.torch_dtype(desc)
         x = torch.from_numpy(gen.features(cfg)).cuda().to(tdt)
         y = torch.empty_like(x)
@@ -219,7 +222,8 @@ def other_workloads(toma, torch, flush, peaks):
         weights_us = t_us(lambda: toma.toma_block(desc, w_reuse, x, y, idx, w, ws, None)) if n_w else None
         full = t_us(lambda: toma.toma_attention(B, N, cfg.n_heads, cfg.head_dim, cfg.dtype, x, x, x, y, None))
         mean = refresh if reuse == 1 else (refresh + n_w * (weights_us or 0.0) + (reuse - 1 - n_w) * reuse_us) / reuse
-        out[label] = {"tokens": B * N, "tile": [cfg.tile_h, cfg.tile_w], "reuse_interval": reuse,
+        out[label] = {"tokens": B * N, "tile": [cfg.tile_h, cfg.tile_w], "global_merge": bool(global_merge),
+                      "reuse_interval": reuse,
                       "weight_reuse_interval": w_reuse or reuse, "refresh_us": refresh, "weights_only_us": weights_us,
                       "reuse_us": reuse_us, "block_mean_us": mean, "full_attention_us": full,
                       "speedup_vs_full_attention": full / mean, "tokens_per_s": B * N / (mean * 1e-6),
