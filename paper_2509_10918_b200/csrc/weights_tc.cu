@@ -231,14 +231,14 @@ __global__ void __launch_bounds__(256)
 weights_normalise_kernel(const float* __restrict__ shares, const float* __restrict__ zpart, __nv_bfloat16* __restrict__ w,
                          int Nloc, int Dloc, int mblocks) {
   // grid (blocks over the tile's [N_loc][D_loc] plane in groups of four destinations, tile)
-  extern __shared__ float zs[];  // row sums of the tile's D_loc destinations
+  extern __shared__ float zs[];  // reciprocal row sums of the tile's D_loc destinations
   dependency_wait();  // launched with programmatic stream serialisation
   if (threadIdx.x == 0) release_dependents();
   const size_t batch = blockIdx.y;
   for (int i = threadIdx.x; i < Dloc; i += blockDim.x) {
     float z = 0.f;
     for (int mb = 0; mb < mblocks; ++mb) z += zpart[(batch * mblocks + mb) * Dloc + i];
-    zs[i] = z;
+    zs[i] = z > 0.f ? 1.f / z : 0.f;  // a row sum that underflowed to 0 gives a zero row
   }
   __syncthreads();
   const int plane = Nloc * Dloc;
@@ -251,8 +251,7 @@ weights_normalise_kernel(const float* __restrict__ shares, const float* __restri
     __nv_bfloat16 hi[4], lo[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      const float z = zs[i + e];
-      const float v = z > 0.f ? in[e] / z : 0.f;
+      const float v = in[e] * zs[i + e];
       hi[e] = __float2bfloat16_rn(v);
       lo[e] = __float2bfloat16_rn(v - __bfloat162float(hi[e]));
     }
