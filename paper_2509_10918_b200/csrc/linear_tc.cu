@@ -35,6 +35,7 @@ struct PipeBars {
 struct LinParams {
   int P, tiles_x, th, tw, W, Nloc, Dloc, d, n_all, Lm;
   int stages;  // pipeline depth
+  int dest_block;  // merge: destinations (MMA N before padding) per CTA, at most kMaxCols
   int out_rows;  // rows of one 64-channel slab of the staged output tile (= the output tensor map's box)
   uint32_t* zero;  // merge only: words cleared on the side (the attention kernel's tickets)
   int zero_words;
@@ -86,14 +87,17 @@ __device__ __forceinline__ void stage_and_store(uint8_t* so, PipeBars* bar, uint
 // ------------------------------------------------------------------------------------------------
 // merge: grid (tile, channel chunk, destination block); K loop over the tile's tokens.
 // ------------------------------------------------------------------------------------------------
+// kBlocked: the destinations of a region are split into blocks of p.dest_block (global merge); otherwise a
+// region's destinations (<= kMaxCols) belong to one CTA and the block size is a compile-time constant.
+template <bool kBlocked>
 __global__ void __launch_bounds__(192, 1)
 merge_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                 const __grid_constant__ CUtensorMap tm_o, const LinParams p, uint32_t* dev_status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int batch = blockIdx.x, c0 = blockIdx.y * 128, i_base = blockIdx.z * kMaxCols;
-  const int n_dest = min(kMaxCols, p.Dloc - i_base);  // destinations this CTA produces
+  const int batch = blockIdx.x, c0 = blockIdx.y * 128, i_base = blockIdx.z * (kBlocked ? p.dest_block : kMaxCols);
+  const int n_dest = min(kBlocked ? p.dest_block : kMaxCols, p.Dloc - i_base);  // destinations this CTA produces
   const int slabs = (n_dest + 63) / 64;               // 64-destination slabs per weight plane
   const int n_mma = slabs * 64;                       // MMA N (zero padded by TMA)
   const int stage_bytes = (2 + 2 * slabs) * kSlab;
@@ -267,7 +271,7 @@ LinParams make_params(const Geom& g) {
   LinParams p;
   p.P = g.P; p.tiles_x = g.tiles_x; p.th = g.th; p.tw = g.tw; p.W = g.W; p.Nloc = g.Nloc; p.Dloc = g.Dloc;
   p.d = g.d; p.n_all = (int)g.tokens_all(); p.Lm = g.Lm; p.stages = 2;
-  p.zero = nullptr; p.zero_words = 0; p.out_rows = 0;
+  p.zero = nullptr; p.zero_words = 0; p.out_rows = 0; p.dest_block = 0;
   return p;
 }
 
@@ -307,23 +311,49 @@ cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* x
   LinParams p = make_params(g);
   // merged rows as (channel, destination, tile, batch): a store that runs past a tile's D_loc rows is clipped
   CUtensorMap to;
-  p.out_rows = g.Dloc < kMaxCols ? g.Dloc : kMaxCols;
+  // Destinations per CTA.  A tile's destinations normally fit one CTA (<= 256).  When they do not (global
+  // merge) the launch is bound by how many bytes the SMs keep in flight, so the block size is the
+  // one that gives every SM a CTA with the deepest pipeline its shared memory holds: the largest multiple
+  // of 16 whose CTA count does not exceed the SM count (a few CTAs more would double the run time).
+  p.dest_block = g.Dloc < kMaxCols ? g.Dloc : kMaxCols;
+  if (g.Dloc > kMaxCols) {
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int per_block = g.B * g.P * ((g.d + 127) / 128);  // CTAs per destination block
+    for (int nb = (g.Dloc + kMaxCols - 1) / kMaxCols; nb * per_block <= sms; ++nb) {
+      const int cand = (((g.Dloc + nb - 1) / nb) + 15) & ~15;
+      if (cand >= 64) p.dest_block = cand;
+    }
+  }
+  p.out_rows = p.dest_block;
   const uint64_t odims[4] = {(uint64_t)g.d, (uint64_t)g.Dloc, (uint64_t)g.P, (uint64_t)g.B};
   const uint64_t ostrides[3] = {(uint64_t)g.d * 2, (uint64_t)g.Dloc * g.d * 2, (uint64_t)g.Lm * g.d * 2};
   const uint32_t obox[4] = {64, (uint32_t)p.out_rows, 1, 1};
   if (!encode_tmap_16bit(&to, xm, 4, odims, ostrides, obox)) return cudaErrorInvalidValue;
-  const int slabs = ((g.Dloc < kMaxCols ? g.Dloc : kMaxCols) + 63) / 64;
+  const int slabs = (p.dest_block + 63) / 64;
   const int stage_bytes = (2 + 2 * slabs) * kSlab;
   p.zero = (uint32_t*)zero;
   p.zero_words = (int)(zero_bytes / 4);
   p.stages = 2;  // two stages keep a CTA below ~100 KB so that two or three CTAs share an SM and hide each other's latencies
+  if (g.Dloc > kMaxCols) {  // one CTA per SM anyway: as deep as shared memory allows
+    p.stages = (198 * 1024) / stage_bytes;
+    p.stages = p.stages > 4 ? 4 : p.stages < 2 ? 2 : p.stages;
+  }
   if (p.stages > g.Nloc / kKC) p.stages = g.Nloc / kKC;
   const int smem = 1024 + p.stages * stage_bytes + 256;
-  static bool attr = false;
-  cudaError_t e = raise_smem_limit((const void*)merge_tc_kernel, &attr);
-  if (e != cudaSuccess) return e;
-  dim3 grid(g.B * g.P, (g.d + 127) / 128, (g.Dloc + kMaxCols - 1) / kMaxCols);
-  e = launch_dependent(merge_tc_kernel, grid, dim3(192), (size_t)smem, s, tx, tw, to, p, dev_status);
+  dim3 grid(g.B * g.P, (g.d + 127) / 128, (g.Dloc + p.dest_block - 1) / p.dest_block);
+  cudaError_t e;
+  if (g.Dloc > kMaxCols) {
+    static bool attr_b = false;
+    e = raise_smem_limit((const void*)merge_tc_kernel<true>, &attr_b);
+    if (e != cudaSuccess) return e;
+    e = launch_dependent(merge_tc_kernel<true>, grid, dim3(192), (size_t)smem, s, tx, tw, to, p, dev_status);
+  } else {
+    static bool attr = false;
+    e = raise_smem_limit((const void*)merge_tc_kernel<false>, &attr);
+    if (e != cudaSuccess) return e;
+    e = launch_dependent(merge_tc_kernel<false>, grid, dim3(192), (size_t)smem, s, tx, tw, to, p, dev_status);
+  }
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }
