@@ -267,6 +267,122 @@ unmerge_tc_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constan
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// unmerge for regions with many destinations (global merge), tokens on M:
+//   Y [tok x ch] = A~^T [tok x D] * X' [D x ch]
+// one CTA = (128 tokens, block of up to 320 channels).  The stored weights are the K-major A operand
+// as they are, the attended rows an MN-major B operand (two MMAs along N: at most 192 + 128 channels).
+// Against channels on M (128 x 128 tiles) a k-step moves 72 KB for 10.5 MFLOP instead of 48 KB for
+// 4.2 MFLOP, the weights are read twice instead of five times, and the 128 CTAs of the 64x64-token
+// case fit the SMs in one wave with a three-stage pipeline; each thread then owns a token row and
+// writes its channels as one contiguous run.
+// ------------------------------------------------------------------------------------------------
+constexpr int kRowsChBlock = 320;  // channels per CTA (five 64-channel slabs)
+
+__global__ void __launch_bounds__(192, 1)
+unmerge_rows_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_w,
+                    __nv_bfloat16* __restrict__ out, const LinParams p, uint32_t* dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int blocks_per_tile = p.Nloc / 128;
+  const int batch = blockIdx.x / blocks_per_tile, t0 = (blockIdx.x - batch * blocks_per_tile) * 128;
+  const int b = batch / p.P, tile = batch - b * p.P;
+  const int c0 = blockIdx.y * kRowsChBlock;
+  const int n_ch = min(kRowsChBlock, p.d - c0);   // channels of this CTA (multiple of 8)
+  const int slabs = (n_ch + 63) / 64;             // 64-channel slabs of the B operand
+  const int n_a = min(slabs, 3) * 64;             // MMA N of the first accumulator (<= 192)
+  const int n_b = (slabs - min(slabs, 3)) * 64;   // and of the second (0, 64 or 128)
+  const int w_plane = 128 * 128;                  // [128 tokens][64 destinations] of one plane
+  const int stage_bytes = 2 * w_plane + slabs * kSlab;
+  PipeBars* bar = reinterpret_cast<PipeBars*>(smem + p.stages * stage_bytes);
+  const int nk = (p.Dloc + kKC - 1) / kKC;
+  constexpr uint32_t ncols = 512;
+
+  if (threadIdx.x == 0) {
+    pipe_init(bar, p.stages);
+    prefetch_tmap(&tm_y);
+    prefetch_tmap(&tm_w);
+  }
+  dependency_wait();
+  if (threadIdx.x == 0) release_dependents();
+  if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bar->tmem_base;
+  volatile int* abort_flag = &bar->abort_flag;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % p.stages;
+        if (k >= p.stages && !mbar_wait(&bar->empty[s], ((k / p.stages) - 1) & 1, dev_status, abort_flag)) break;
+        uint8_t* sw = smem + s * stage_bytes;
+        uint8_t* sy = sw + 2 * w_plane;
+        mbar_expect_tx(&bar->full[s], stage_bytes);
+        for (int pl = 0; pl < 2; ++pl) tma_load_3d(sw + pl * w_plane, &tm_w, &bar->full[s], k * kKC, t0, 2 * batch + pl);
+        for (int c = 0; c < slabs; ++c)
+          tma_load_3d(sy + c * kSlab, &tm_y, &bar->full[s], c0 + c * 64, tile * p.Dloc + k * kKC, b);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc_a = idesc_f16(kFmtBF16, kFmtBF16, false, true, 128, n_a);
+      const uint32_t idesc_b = idesc_f16(kFmtBF16, kFmtBF16, false, true, 128, n_b > 0 ? n_b : 64);
+      bool ok = true;
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % p.stages;
+        if (!mbar_wait(&bar->full[s], (k / p.stages) & 1, dev_status, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t wa = smem_u32(smem + s * stage_bytes), ya = wa + 2 * w_plane;
+        const int ksteps = min(kKC, p.Dloc - k * kKC + 15) / 16;  // 16 destinations per MMA
+        for (int kk = 0; kk < ksteps; ++kk) {
+          const uint64_t yd_a = smem_desc_sw128(ya + kk * 2048, kSlab, 1024);
+          const uint64_t yd_b = smem_desc_sw128(ya + 3 * kSlab + kk * 2048, kSlab, 1024);
+          for (int pl = 0; pl < 2; ++pl) {
+            const uint64_t wd = smem_desc_sw128(wa + pl * w_plane + kk * 32, 16, 1024);
+            const bool acc = k > 0 || kk > 0 || pl > 0;
+            mma_ss(tmem, wd, yd_a, idesc_a, acc);
+            if (n_b > 0) mma_ss(tmem + 192, wd, yd_b, idesc_b, acc);
+          }
+        }
+        mma_commit(&bar->empty[s]);
+      }
+      if (ok) mma_commit(&bar->done);
+    }
+  } else {
+    const int quarter = warp & 3, row = quarter * 32 + lane;  // token slot t0 + row = tensor-memory lane
+    const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16);
+    if (mbar_wait(&bar->done, 0, dev_status, abort_flag)) {
+      tc_fence_after();
+      const size_t tok = (size_t)tile_token(tile, t0 + row, p.tiles_x, p.th, p.tw, p.W);
+      __nv_bfloat16* dst = out + ((size_t)b * p.n_all + tok) * p.d + c0;
+      for (int c = 0; c < n_ch; c += 32) {  // accumulator column = channel (the second accumulator starts at 192)
+        uint32_t r[32];
+        tmem_ld32(taddr + c, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; e += 8) {
+          if (c + e < n_ch) {
+            __align__(16) __nv_bfloat162 q[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              q[u] = __floats2bfloat162_rn(__uint_as_float(r[e + 2 * u]), __uint_as_float(r[e + 2 * u + 1]));
+            *reinterpret_cast<uint4*>(dst + c + e) = *reinterpret_cast<const uint4*>(q);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, ncols);
+  }
+}
+
 LinParams make_params(const Geom& g) {
   LinParams p;
   p.P = g.P; p.tiles_x = g.tiles_x; p.th = g.th; p.tw = g.tw; p.W = g.W; p.Nloc = g.Nloc; p.Dloc = g.Dloc;
@@ -368,6 +484,27 @@ cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void*
   if (!encode_tmap_16bit(&ty, y, 3, dims, strides, box) || !encode_w(g, w, &tw, (uint32_t)n_tok))
     return cudaErrorInvalidValue;
   LinParams p = make_params(g);
+  if (g.Dloc > kMaxCols && g.Nloc % 128 == 0) {  // many destinations per region: tokens on M
+    CUtensorMap tw128;
+    if (!encode_w(g, w, &tw128, 128)) return cudaErrorInvalidValue;
+    const int slabs = ((g.d < kRowsChBlock ? g.d : kRowsChBlock) + 63) / 64;
+    const int stage_bytes = 2 * 128 * 128 + slabs * kSlab;
+    p.stages = (224 * 1024) / stage_bytes;
+    p.stages = p.stages > 4 ? 4 : p.stages < 2 ? 2 : p.stages;
+    if (p.stages > (g.Dloc + kKC - 1) / kKC) p.stages = (g.Dloc + kKC - 1) / kKC;
+    const int smem = 1024 + p.stages * stage_bytes + 256;
+    static bool attr_r = false;
+    if (!attr_r) {
+      cudaError_t e = cudaFuncSetAttribute(unmerge_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      if (e != cudaSuccess) return e;
+      attr_r = true;
+    }
+    dim3 grid(g.B * g.P * (g.Nloc / 128), (g.d + kRowsChBlock - 1) / kRowsChBlock);
+    cudaError_t e = launch_dependent(unmerge_rows_kernel, grid, dim3(192), (size_t)smem, s, ty, tw128, (__nv_bfloat16*)out, p,
+                                     dev_status);
+    count_launch();
+    return e != cudaSuccess ? e : cudaGetLastError();
+  }
   // output tokens as (channel, x, y, batch): a CTA's token block is n_tok / tile_w whole tile rows
   CUtensorMap to;
   const uint64_t odims[4] = {(uint64_t)g.d, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.B};

@@ -300,6 +300,8 @@ GLOBAL = [
     dict(grid_h=32, grid_w=32, tile_h=8, tile_w=8, dim=128, n_heads=2, head_dim=64, dtype="f32"),
     dict(grid_h=16, grid_w=64, tile_h=4, tile_w=16, dim=64, n_heads=1, head_dim=64, dtype="bf16", merge_ratio=0.75),
     dict(grid_h=16, grid_w=16, tile_h=8, tile_w=8, dim=64, n_heads=1, head_dim=64, dtype="bf16", n_extra=5),
+    # 384 channels: a full 320-channel block and a 64-channel one in the tokens-on-M unmerge; 768 destinations
+    dict(grid_h=32, grid_w=32, tile_h=16, tile_w=16, dim=384, n_heads=6, head_dim=64, dtype="bf16", merge_ratio=0.25),
 ]
 
 
