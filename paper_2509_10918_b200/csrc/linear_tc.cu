@@ -484,7 +484,14 @@ cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void*
   if (!encode_tmap_16bit(&ty, y, 3, dims, strides, box) || !encode_w(g, w, &tw, (uint32_t)n_tok))
     return cudaErrorInvalidValue;
   LinParams p = make_params(g);
-  if (g.Dloc > kMaxCols && g.Nloc % 128 == 0) {  // many destinations per region: tokens on M
+  // Tokens on M when a region has many destinations, and also when that form fits the SMs in one wave while
+  // the channels-on-M grid would spill into a second one (64x64 tokens: 128 CTAs against 320 on 296 slots).
+  int sms = 148, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int rows_ctas = g.B * g.P * (g.Nloc / 128) * ((g.d + kRowsChBlock - 1) / kRowsChBlock);
+  const int classic_ctas = g.B * g.P * ((g.d + 127) / 128) * (g.Nloc / n_tok);
+  const bool one_wave = rows_ctas <= sms && classic_ctas > 2 * sms;
+  if ((g.Dloc > kMaxCols || one_wave) && g.Nloc % 128 == 0) {
     CUtensorMap tw128;
     if (!encode_w(g, w, &tw128, 128)) return cudaErrorInvalidValue;
     const int slabs = ((g.d < kRowsChBlock ? g.d : kRowsChBlock) + 63) / 64;
