@@ -359,7 +359,7 @@ def main():
         if t >= 3:
             for i, name in enumerate(stages):
                 stages[name].append(ev[i].elapsed_time(ev[i + 1]))
-    stage_ms = {k: statistics.mean(v) for k, v in stages.items()}
+    stage_ms = {k: statistics.median(v) for k, v in stages.items()}
     esz = 2 if cfg.dtype == "bf16" else 4
     att_flops = 4.0 * B * Lm * Lm * d
     att_tf = att_flops / (stage_ms["attention"] * 1e-3) / 1e12
