@@ -172,6 +172,13 @@ TOMA_API toma_status toma_attention(int32_t batch, int32_t len, int32_t n_heads,
 TOMA_API toma_status toma_unmerge(const toma_desc* desc, const void* w, const void* y, void* out, uint32_t* dev_status,
                          void* stream);
 
+/* Dense projection c = a w: the linear maps of the wrapped module (the Q/K/V and output projections of
+ * attention, whose cost App. C counts as the 4 d^2 N term that shrinks with the merged length).
+ *   a [m][k], w [k][n], c [m][n]: device, row-major, dense, 16-byte aligned; bf16 needs n and k
+ *   multiples of 8.  bf16 runs on the tensor cores with fp32 accumulation, fp32 on FFMA. */
+TOMA_API toma_status toma_linear(int32_t m, int32_t n, int32_t k, int32_t dtype, const void* a, const void* w, void* c,
+                                 uint32_t* dev_status, void* stream);
+
 /* One ToMA-wrapped attention call (Algorithm 3) with pattern reuse (Sec. 4.3.2):
  * refresh idx_state / w_state when the schedule says so, then merge, attention
  * with Q = K = V = merged tokens, unmerge.  idx_state [batch][P][D_loc] and

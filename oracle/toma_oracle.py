@@ -224,6 +224,12 @@ def unmerge(w: np.ndarray, y_tile: np.ndarray) -> np.ndarray:
 # ----------------------------------------------------------------------------
 
 
+def linear(a: np.ndarray, w: np.ndarray) -> np.ndarray:
+    """Projection c = a w (the Q/K/V and output maps of the wrapped attention module; App. C's 4 d^2 N
+    term): a [m, k], w [k, n] -> [m, n], fp64."""
+    return np.asarray(a, dtype=np.float64) @ np.asarray(w, dtype=np.float64)
+
+
 def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, n_heads: int,
               query_rows: Optional[np.ndarray] = None) -> np.ndarray:
     """Multi-head softmax(Q K^T / sqrt(dh)) V for one batch item.

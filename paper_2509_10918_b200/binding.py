@@ -21,7 +21,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_RATIO", "ERR_TA
 
 EXPORTS = ["toma_select_static", "toma_launch_counter", "toma_workspace_bytes", "toma_weights_bytes", "toma_dest_per_tile", "toma_validate", "toma_status_str",
            "toma_select", "toma_merge_weights", "toma_merge", "toma_attention_workspace_bytes", "toma_attention_plan", "toma_attention",
-           "toma_unmerge", "toma_block", "toma_block_host",
+           "toma_unmerge", "toma_block", "toma_block_host", "toma_linear",
            "toma_weights_export", "toma_weights_import"]
 
 
@@ -82,6 +82,8 @@ def _load() -> ctypes.CDLL:
     lib.toma_block.restype = c_int32
     lib.toma_block.argtypes = [P, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p,
                                c_void_p]
+    lib.toma_linear.restype = c_int32
+    lib.toma_linear.argtypes = [c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.toma_block_host.restype = c_int32
     lib.toma_block_host.argtypes = [P, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                     c_size_t, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
@@ -224,6 +226,14 @@ def toma_attention(batch, length, n_heads, head_dim, dtype, q, k, v, o, dev_stat
 def toma_block(desc, step, x, out, idx_state, w_state, ws, dev_status=None):
     _check(lib.toma_block(ctypes.byref(desc), step, _ptr(x), _ptr(out), _ptr(idx_state), _ptr(w_state), _ptr(ws),
                           ws.numel() * ws.element_size(), _ptr(dev_status), _stream()), "toma_block")
+
+
+def toma_linear(a, w, c, dev_status=None):
+    """c = a @ w for 2-D tensors a [m, k], w [k, n], c [m, n] of the same dtype (bf16 or fp32)."""
+    m, k = a.shape
+    n = w.shape[1]
+    code = TOMA_F32 if a.dtype == torch.float32 else TOMA_BF16
+    _check(lib.toma_linear(m, n, k, code, _ptr(a), _ptr(w), _ptr(c), _ptr(dev_status), _stream()), "toma_linear")
 
 
 def toma_block_host(desc, step, x_host, out_host, x_dev, out_dev, idx_state, w_state, ws, dev_status=None,

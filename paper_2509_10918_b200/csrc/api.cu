@@ -260,6 +260,29 @@ toma_status toma_attention(int32_t batch, int32_t len, int32_t n_heads, int32_t 
                               (cudaStream_t)stream));
 }
 
+// c[i] = a w[i] for n_mats weight / output pairs
+static cudaError_t do_linear(int M, int N, int K, bool f32, const void* a, const void* const* w, void* const* c, int n_mats,
+                             uint32_t* dev_status, cudaStream_t s) {
+  if (!f32 && linear_tc_shape_ok(M, N, K)) return launch_linear_tc(M, N, K, a, w, c, n_mats, dev_status, s);
+  for (int i = 0; i < n_mats; ++i) {
+    cudaError_t e = launch_linear_simt(M, N, K, f32, a, w[i], c[i], s);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+toma_status toma_linear(int32_t m, int32_t n, int32_t k, int32_t dtype, const void* a, const void* w, void* c,
+                        uint32_t* dev_status, void* stream) {
+  if (dtype != TOMA_BF16 && dtype != TOMA_F32) return TOMA_ERR_DTYPE;
+  if (m < 1 || n < 1 || k < 1) return TOMA_ERR_SHAPE;
+  if (!a || !w || !c) return TOMA_ERR_NULL;
+  if (misaligned(a) || misaligned(w) || misaligned(c)) return TOMA_ERR_SHAPE;
+  if (dtype == TOMA_BF16 && (n % 8 || k % 8)) return TOMA_ERR_SHAPE;  // 16-byte rows
+  const void* ws[1] = {w};
+  void* cs[1] = {c};
+  return cuda_ok(do_linear(m, n, k, dtype == TOMA_F32, a, ws, cs, 1, dev_status, (cudaStream_t)stream));
+}
+
 toma_status toma_block(const toma_desc* desc, int32_t step, const void* x, void* out, int32_t* idx_state,
                        void* w_state, void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream) {
   Geom g;

@@ -79,6 +79,12 @@ cudaError_t launch_attention_tc(int B, int L, int heads, int dh, const void* q, 
                                 void* ws, bool tickets_clean, uint32_t* dev_status, cudaStream_t s);
 // Image-level destination ids [batch][D] (tile-major, pick order) from the tile-local picks.
 cudaError_t launch_global_idx(const Geom& g, const int32_t* idx, int32_t* gidx, cudaStream_t s);
+// Projection c = a w (a [M][K], w [K][N], c [M][N], row-major): tensor-core form for bf16 (up to three
+// weight / output pairs sharing a), FFMA form otherwise.
+bool linear_tc_shape_ok(int M, int N, int K);
+cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* const* w, void* const* c, int n_mats,
+                             uint32_t* dev_status, cudaStream_t s);
+cudaError_t launch_linear_simt(int M, int N, int K, bool f32, const void* a, const void* w, void* c, cudaStream_t s);
 cudaError_t launch_weights_export(const Geom& g, const void* w, float* dense, cudaStream_t s);
 cudaError_t launch_weights_import(const Geom& g, const float* dense, void* w, cudaStream_t s);
 

@@ -1,0 +1,178 @@
+// Dense projection C[m][n] = sum_k A[m][k] W[k][n] on the sm_100a tensor cores (bf16 in, fp32
+// accumulation in tensor memory, bf16 out): the QKV and output projections of the attention module
+// that ToMA wraps (Algorithm 3's core module F; App. C counts them as the 4 d^2 N term).
+//
+// Rows of A (tokens) sit on the MMA M dimension, 128 per CTA; a CTA covers up to 320 output columns
+// (two MMAs along N, at most 192 + 128).  A is the K-major operand exactly as stored ([m][k] row-major),
+// W the MN-major one exactly as stored ([k][n] row-major), so neither is transposed or copied.
+// blockIdx.z selects one of up to three weight / output pairs that share A (Q, K and V in one
+// launch).  Warp 0 feeds a TMA ring, warp 1 issues the MMAs, warps 2..5 write each token row's
+// columns as one contiguous run.
+#include "common.cuh"
+#include "tc.cuh"
+
+namespace toma {
+
+using namespace tc;
+
+namespace {
+
+constexpr int kKC = 64;                  // contraction elements per stage
+constexpr int kSlab = kKC * 128;         // [64 k][64 n] slab of W, 128-byte rows
+constexpr int kABytes = 128 * 128;       // [128 m][64 k] slab of A
+constexpr int kColBlock = 320;           // output columns per CTA
+
+struct GemmBars {
+  uint64_t full[4], empty[4], done;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct GemmOut {
+  __nv_bfloat16* c[3];
+};
+
+__global__ void __launch_bounds__(192, 1)
+linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w0,
+                   const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2, GemmOut out, int M,
+                   int N, int K, int stages, uint32_t* dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * 128, n0 = blockIdx.y * kColBlock;
+  const CUtensorMap* tm_w = blockIdx.z == 0 ? &tm_w0 : blockIdx.z == 1 ? &tm_w1 : &tm_w2;
+  __nv_bfloat16* c = out.c[blockIdx.z];
+  const int n_cols = min(kColBlock, N - n0);     // columns of this CTA (multiple of 8)
+  const int slabs = (n_cols + 63) / 64;
+  const int n_a = min(slabs, 3) * 64, n_b = (slabs - min(slabs, 3)) * 64;
+  const int stage_bytes = kABytes + slabs * kSlab;
+  GemmBars* bar = reinterpret_cast<GemmBars*>(smem + stages * stage_bytes);
+  const int nk = (K + kKC - 1) / kKC;
+  constexpr uint32_t ncols = 512;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(&bar->full[s], 1);
+      mbar_init(&bar->empty[s], 1);
+    }
+    mbar_init(&bar->done, 1);
+    bar->abort_flag = 0;
+    mbar_fence_init();
+    prefetch_tmap(&tm_a);
+    prefetch_tmap(tm_w);
+  }
+  dependency_wait();
+  if (threadIdx.x == 0) release_dependents();
+  if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bar->tmem_base;
+  volatile int* abort_flag = &bar->abort_flag;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % stages;
+        if (k >= stages && !mbar_wait(&bar->empty[s], ((k / stages) - 1) & 1, dev_status, abort_flag)) break;
+        uint8_t* sa = smem + s * stage_bytes;
+        mbar_expect_tx(&bar->full[s], stage_bytes);
+        tma_load_2d(sa, &tm_a, &bar->full[s], k * kKC, m0);
+        for (int j = 0; j < slabs; ++j) tma_load_2d(sa + kABytes + j * kSlab, tm_w, &bar->full[s], n0 + j * 64, k * kKC);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc_a = idesc_f16(kFmtBF16, kFmtBF16, false, true, 128, n_a);
+      const uint32_t idesc_b = idesc_f16(kFmtBF16, kFmtBF16, false, true, 128, n_b > 0 ? n_b : 64);
+      bool ok = true;
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % stages;
+        if (!mbar_wait(&bar->full[s], (k / stages) & 1, dev_status, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t aa = smem_u32(smem + s * stage_bytes), wa = aa + kABytes;
+        const int ksteps = min(kKC, K - k * kKC + 15) / 16;  // 16 contraction elements per MMA (zero filled past K)
+        for (int kk = 0; kk < ksteps; ++kk) {
+          const uint64_t ad = smem_desc_sw128(aa + kk * 32, 16, 1024);
+          mma_ss(tmem, ad, smem_desc_sw128(wa + kk * 2048, kSlab, 1024), idesc_a, k > 0 || kk > 0);
+          if (n_b > 0) mma_ss(tmem + 192, ad, smem_desc_sw128(wa + 3 * kSlab + kk * 2048, kSlab, 1024), idesc_b, k > 0 || kk > 0);
+        }
+        mma_commit(&bar->empty[s]);
+      }
+      if (ok) mma_commit(&bar->done);
+    }
+  } else {
+    const int quarter = warp & 3, row = m0 + quarter * 32 + lane;
+    const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16);
+    if (mbar_wait(&bar->done, 0, dev_status, abort_flag)) {
+      tc_fence_after();
+      __nv_bfloat16* dst = c + (size_t)(row < M ? row : 0) * N + n0;
+      for (int j = 0; j < n_cols; j += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + j, r);
+        tmem_wait_ld();
+        if (row < M) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 8) {
+            if (j + e < n_cols) {
+              __align__(16) __nv_bfloat162 q[4];
+#pragma unroll
+              for (int u = 0; u < 4; ++u)
+                q[u] = __floats2bfloat162_rn(__uint_as_float(r[e + 2 * u]), __uint_as_float(r[e + 2 * u + 1]));
+              *reinterpret_cast<uint4*>(dst + j + e) = *reinterpret_cast<const uint4*>(q);
+            }
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, ncols);
+  }
+}
+
+}  // namespace
+
+bool linear_tc_shape_ok(int M, int N, int K) { return M >= 1 && N >= 8 && K >= 8 && N % 8 == 0 && K % 8 == 0; }
+
+// c[i] = a * w[i] for i < n_mats (1..3); a [M][K], w[i] [K][N], c[i] [M][N], all bf16 row-major.
+cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* const* w, void* const* c, int n_mats,
+                             uint32_t* dev_status, cudaStream_t s) {
+  CUtensorMap ta, tw[3];
+  const uint64_t adims[2] = {(uint64_t)K, (uint64_t)M};
+  const uint64_t astr[1] = {(uint64_t)K * 2};
+  const uint32_t abox[2] = {64, 128};
+  if (!encode_tmap_16bit(&ta, a, 2, adims, astr, abox)) return cudaErrorInvalidValue;
+  const uint64_t wdims[2] = {(uint64_t)N, (uint64_t)K};
+  const uint64_t wstr[1] = {(uint64_t)N * 2};
+  const uint32_t wbox[2] = {64, 64};
+  GemmOut out;
+  for (int i = 0; i < 3; ++i) {
+    const int j = i < n_mats ? i : 0;
+    if (!encode_tmap_16bit(&tw[i], w[j], 2, wdims, wstr, wbox)) return cudaErrorInvalidValue;
+    out.c[i] = (__nv_bfloat16*)c[j];
+  }
+  const int slabs = ((N < kColBlock ? N : kColBlock) + 63) / 64;
+  const int stage_bytes = kABytes + slabs * kSlab;
+  int stages = (222 * 1024) / stage_bytes;
+  stages = stages > 4 ? 4 : stages;
+  const int nk = (K + kKC - 1) / kKC;
+  if (stages > nk) stages = nk;
+  const int smem = 1024 + stages * stage_bytes + 256;
+  static bool attr = false;
+  if (!attr) {
+    cudaError_t e = cudaFuncSetAttribute(linear_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    attr = true;
+  }
+  dim3 grid((M + 127) / 128, (N + kColBlock - 1) / kColBlock, n_mats);
+  cudaError_t e = launch_dependent(linear_rows_kernel, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out, M, N, K,
+                                   stages, dev_status);
+  count_launch();
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+}  // namespace toma

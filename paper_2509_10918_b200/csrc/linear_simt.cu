@@ -267,6 +267,31 @@ cudaError_t launch_unmerge_simt(const Geom& g, const void* w, const void* y, voi
   return cudaGetLastError();
 }
 
+// c[m][n] = sum_k a[m][k] w[k][n] (plain projection; fp32 mode and shapes the tensor-core kernel does not take).
+template <typename T>
+struct LinearOp {
+  static constexpr bool a_k_contig = true, b_k_contig = false;
+  int M, N, K;
+  const T* a_;
+  const T* w_;
+  T* c_;
+  __device__ __forceinline__ float a(int, int m, int k) const { return to_f32(a_[(size_t)m * K + k]); }
+  __device__ __forceinline__ float b(int, int k, int n) const { return to_f32(w_[(size_t)k * N + n]); }
+  template <typename AccT>
+  __device__ __forceinline__ void store(int, int m, int n, AccT v) const { from_f32(c_[(size_t)m * N + n], (float)v); }
+};
+
+cudaError_t launch_linear_simt(int M, int N, int K, bool f32, const void* a, const void* w, void* c, cudaStream_t s) {
+  if (f32) {
+    LinearOp<float> op{M, N, K, (const float*)a, (const float*)w, (float*)c};
+    run_gemm<LinearOp<float>, float>(op, 1, s);
+  } else {
+    LinearOp<__nv_bfloat16> op{M, N, K, (const __nv_bfloat16*)a, (const __nv_bfloat16*)w, (__nv_bfloat16*)c};
+    run_gemm<LinearOp<__nv_bfloat16>, float>(op, 1, s);
+  }
+  return cudaGetLastError();
+}
+
 // gidx[b][p * D_loc + k] = image token of tile p's k-th pick.
 __global__ void global_idx_kernel(const int32_t* __restrict__ idx, int32_t* __restrict__ gidx, int P, int Dloc, int tiles_x,
                                   int th, int tw, int W, int total) {

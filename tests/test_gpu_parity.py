@@ -362,6 +362,25 @@ def test_global_merge_block_parity_at_benchmark_size(toma):
         assert_close(to_host64(out), want, cfg.dtype, f"global-merge block step {step}")
 
 
+@pytest.mark.parametrize("dtype,m,n,k", [
+    ("bf16", 4096, 640, 640), ("bf16", 4096, 1920, 640), ("bf16", 1000, 72, 200), ("bf16", 130, 320, 64),
+    ("bf16", 128, 328, 640), ("bf16", 2560, 3072, 3072), ("f32", 300, 96, 160),
+])
+def test_linear_parity(toma, dtype, m, n, k):
+    """Projection c = a w through toma_linear: ragged rows, a partial last k-step, partial column blocks."""
+    a_host = gen.round_to_dtype(gen.normal(0, (91, m, k), m * k).reshape(m, k).astype(np.float32), dtype)
+    w_host = gen.round_to_dtype((gen.normal(0, (92, n, k), k * n).reshape(k, n) / np.sqrt(k)).astype(np.float32), dtype)
+    a, w = to_dev(a_host, dtype), to_dev(w_host, dtype)
+    c = torch.full((m, n), float("nan"), dtype=a.dtype, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    toma.toma_linear(a, w, c, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rows = np.unique(np.concatenate([[0, m - 1], np.random.default_rng(m).choice(m, size=min(m, 200), replace=False)]))
+    assert not torch.isnan(c).any()
+    assert_close(to_host64(c)[rows], O.linear(a_host[rows], w_host), dtype, "linear")
+
+
 def test_block_replays_from_a_cuda_graph(toma):
     """A reuse step and a refresh step captured into CUDA graphs (the calls never allocate or synchronise,
     and their dependent launches are capturable) replay to the same bits as direct calls."""

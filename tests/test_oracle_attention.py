@@ -47,3 +47,15 @@ def test_heads_are_independent_column_blocks_and_match_library():
     assert np.allclose(got, want.numpy(), atol=1e-12)
     rows = np.array([0, 5, 36])
     assert np.allclose(O.attention(q, k, v, h, query_rows=rows), got[rows])
+
+
+def test_linear_matches_explicit_loops():
+    rng = np.random.default_rng(5)
+    a, w = rng.normal(size=(5, 7)), rng.normal(size=(7, 3))
+    want = np.zeros((5, 3))
+    for i in range(5):
+        for j in range(3):
+            for k in range(7):
+                want[i, j] += a[i, k] * w[k, j]
+    assert np.allclose(O.linear(a, w), want, rtol=0, atol=1e-13)
+    assert np.array_equal(O.linear(a, np.eye(7)), a)
