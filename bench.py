@@ -230,7 +230,53 @@ def other_workloads(toma, torch, flush, peaks):
                       "full_attention_tflops": 4.0 * B * N * N * d / full / 1e6}
         del x, y, idx, w, ws
         torch.cuda.empty_cache()
+    out["cfg3_attention_module"] = attention_module_workload(toma, torch, flush)
     return out
+
+
+def attention_module_workload(toma, torch, flush):
+    """The benchmark workload with the whole attention module as the wrapped F: Q/K/V projections, attention and
+    output projection on the merged tokens (toma_block_proj) against the same module on all tokens
+    (toma_attention_proj).  Random N(0, 1/d) projection weights."""
+    import gen
+    cfg = gen.config("cfg3")
+    desc = toma.desc_from_config(cfg)
+    tdt = toma.torch_dtype(desc)
+    x = torch.from_numpy(gen.features(cfg)).cuda().to(tdt)
+    y = torch.empty_like(x)
+    d = cfg.dim
+    ws_w = [torch.from_numpy((gen.normal(0, (96, i, d), d * d).reshape(d, d) / d ** 0.5).astype("float32")).cuda().to(tdt)
+            for i in range(4)]
+    idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    B, N = cfg.batch, cfg.n_tokens
+    ws_full = torch.empty(toma.toma_attention_proj_workspace_bytes(B, N, cfg.n_heads, cfg.head_dim, cfg.dtype),
+                          dtype=torch.uint8, device="cuda")
+
+    def t_us(fn, reps=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(1e3 * e0.elapsed_time(e1))
+        return statistics.median(ts)
+
+    k = cfg.reuse_interval
+    refresh = t_us(lambda: toma.toma_block_proj(desc, 0, x, *ws_w, y, idx, w, ws, None))
+    reuse_us = t_us(lambda: toma.toma_block_proj(desc, 1, x, *ws_w, y, idx, w, ws, None))
+    full = t_us(lambda: toma.toma_attention_proj(B, N, cfg.n_heads, cfg.head_dim, cfg.dtype, x, *ws_w, y, ws_full, None))
+    mean = (refresh + (k - 1) * reuse_us) / k
+    m = B * (cfg.n_merged + cfg.n_extra)
+    qkv = t_us(lambda: toma.toma_linear(x.view(B * N, d)[:m], ws_w[0], y.view(B * N, d)[:m]))
+    return {"tokens": B * N, "reuse_interval": k, "refresh_us": refresh, "reuse_us": reuse_us, "block_mean_us": mean,
+            "full_module_us": full, "speedup_vs_full_module": full / mean,
+            "one_projection_us": qkv, "one_projection_tflops": 2.0 * m * d * d / qkv / 1e6}
 
 
 def main():

@@ -186,6 +186,23 @@ TOMA_API toma_status toma_linear(int32_t m, int32_t n, int32_t k, int32_t dtype,
 TOMA_API toma_status toma_block(const toma_desc* desc, int32_t step, const void* x, void* out, int32_t* idx_state,
                        void* w_state, void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream);
 
+/* toma_block with the whole attention module as the wrapped F (Algorithm 3 applies F to the merged tokens,
+ * so the module's projections shrink with them): Q = X_m wq, K = X_m wk, V = X_m wv, attention, then wo,
+ * then the unmerge.  wq, wk, wv, wo: [dim][dim] row-major [in][out], device, dtype of x.  Everything else as
+ * toma_block (same workspace size). */
+TOMA_API toma_status toma_block_proj(const toma_desc* desc, int32_t step, const void* x, const void* wq, const void* wk,
+                                     const void* wv, const void* wo, void* out, int32_t* idx_state, void* w_state, void* ws,
+                                     size_t ws_bytes, uint32_t* dev_status, void* stream);
+
+/* The same attention module on all tokens, without ToMA: out = attention(x wq, x wk, x wv) wo.  The
+ * full-token baseline of toma_block_proj.  x, out [batch][len][n_heads*head_dim];
+ * ws: device scratch of toma_attention_proj_workspace_bytes(), 16-byte aligned. */
+TOMA_API size_t toma_attention_proj_workspace_bytes(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim,
+                                                    int32_t dtype);
+TOMA_API toma_status toma_attention_proj(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim, int32_t dtype,
+                                         const void* x, const void* wq, const void* wk, const void* wv, const void* wo,
+                                         void* out, void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream);
+
 /* toma_block for callers whose tokens live in HOST memory (Algorithm 3 end to end, copies included):
  * copy x_host -> x_dev, run toma_block(x_dev -> out_dev), copy out_dev -> out_host.
  *   x_host, out_host: HOST buffers of batch*(N + n_extra)*dim elements, caller-owned.  Page-locked

@@ -277,7 +277,7 @@ class BlockState:
 def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid_w: int,
                tile_h: int, tile_w: int, merge_ratio: float, tau: float, n_heads: int,
                reuse_interval: int, n_extra: int = 0, round_fn=None, weight_reuse_interval: int = 0,
-               global_merge: bool = False):
+               global_merge: bool = False, proj=None):
     """One ToMA-wrapped attention call (Algorithm 3) on x [B, N + n_extra, d].
 
     Selection and weights are recomputed when step % reuse_interval == 0 and
@@ -292,6 +292,10 @@ def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid
     tile, merge over the whole image) the D destinations of an image, in the same tile-major pick
     order, form one destination set and Sec. 4.2's weights, merge and unmerge are applied once to all
     N image tokens; state.w is then [B, 1, D, N].
+
+    With proj = (wq, wk, wv, wo), each [d, d] as [in, out], the wrapped module is the whole attention
+    module: attention(X_m wq, X_m wk, X_m wv) wo (Algorithm 3 applies F to the merged tokens; App. C's
+    4 d^2 N term).  round_fn is then also applied to q, k, v and to the projected output.
 
     `round_fn`, if given, is applied to the merged and to the attended tensor; it
     lets a test mirror the storage rounding between stages.  Returns
@@ -331,10 +335,15 @@ def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid
         merged[b, D:] = x[b, N:]
     if round_fn is not None:
         merged = round_fn(merged)
+    rnd = (lambda t: t) if round_fn is None else round_fn
     attended = np.empty_like(merged)
     for b in range(B):
-        attended[b] = attention(merged[b], merged[b], merged[b], n_heads)
-    if round_fn is not None:
+        if proj is None:
+            attended[b] = attention(merged[b], merged[b], merged[b], n_heads)
+        else:
+            q, k, v = (rnd(linear(merged[b], w)) for w in proj[:3])
+            attended[b] = rnd(linear(rnd(attention(q, k, v, n_heads)), proj[3]))
+    if round_fn is not None and proj is None:
         attended = round_fn(attended)
     out = np.empty((B, n_all, d), dtype=np.float64)
     for b in range(B):

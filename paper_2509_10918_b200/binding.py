@@ -21,7 +21,8 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_RATIO", "ERR_TA
 
 EXPORTS = ["toma_select_static", "toma_launch_counter", "toma_workspace_bytes", "toma_weights_bytes", "toma_dest_per_tile", "toma_validate", "toma_status_str",
            "toma_select", "toma_merge_weights", "toma_merge", "toma_attention_workspace_bytes", "toma_attention_plan", "toma_attention",
-           "toma_unmerge", "toma_block", "toma_block_host", "toma_linear",
+           "toma_unmerge", "toma_block", "toma_block_host", "toma_linear", "toma_block_proj", "toma_attention_proj_workspace_bytes",
+           "toma_attention_proj",
            "toma_weights_export", "toma_weights_import"]
 
 
@@ -82,6 +83,12 @@ def _load() -> ctypes.CDLL:
     lib.toma_block.restype = c_int32
     lib.toma_block.argtypes = [P, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p,
                                c_void_p]
+    lib.toma_block_proj.restype = c_int32
+    lib.toma_block_proj.argtypes = [P, c_int32] + [c_void_p] * 9 + [c_size_t, c_void_p, c_void_p]
+    lib.toma_attention_proj_workspace_bytes.restype = c_size_t
+    lib.toma_attention_proj_workspace_bytes.argtypes = [c_int32] * 5
+    lib.toma_attention_proj.restype = c_int32
+    lib.toma_attention_proj.argtypes = [c_int32] * 5 + [c_void_p] * 7 + [c_size_t, c_void_p, c_void_p]
     lib.toma_linear.restype = c_int32
     lib.toma_linear.argtypes = [c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.toma_block_host.restype = c_int32
@@ -234,6 +241,22 @@ def toma_linear(a, w, c, dev_status=None):
     n = w.shape[1]
     code = TOMA_F32 if a.dtype == torch.float32 else TOMA_BF16
     _check(lib.toma_linear(m, n, k, code, _ptr(a), _ptr(w), _ptr(c), _ptr(dev_status), _stream()), "toma_linear")
+
+
+def toma_block_proj(desc, step, x, wq, wk, wv, wo, out, idx_state, w_state, ws, dev_status=None):
+    _check(lib.toma_block_proj(ctypes.byref(desc), step, _ptr(x), _ptr(wq), _ptr(wk), _ptr(wv), _ptr(wo), _ptr(out),
+                               _ptr(idx_state), _ptr(w_state), _ptr(ws), ws.numel() * ws.element_size(), _ptr(dev_status),
+                               _stream()), "toma_block_proj")
+
+
+def toma_attention_proj_workspace_bytes(batch, length, n_heads, head_dim, dtype) -> int:
+    return int(lib.toma_attention_proj_workspace_bytes(batch, length, n_heads, head_dim, _dtype_code(dtype)))
+
+
+def toma_attention_proj(batch, length, n_heads, head_dim, dtype, x, wq, wk, wv, wo, out, ws, dev_status=None):
+    _check(lib.toma_attention_proj(batch, length, n_heads, head_dim, _dtype_code(dtype), _ptr(x), _ptr(wq), _ptr(wk),
+                                   _ptr(wv), _ptr(wo), _ptr(out), _ptr(ws), ws.numel() * ws.element_size(),
+                                   _ptr(dev_status), _stream()), "toma_attention_proj")
 
 
 def toma_block_host(desc, step, x_host, out_host, x_dev, out_dev, idx_state, w_state, ws, dev_status=None,

@@ -70,6 +70,8 @@ WsLayout ws_layout(const Geom& g) {
   l.xm_off = off;     off = align_up(off + (size_t)g.B * g.Lm * g.d * esz, 256);
   l.att_off = off;    off = align_up(off + (size_t)g.B * g.Lm * g.d * esz, 256);
   l.att_ws_off = off; off = align_up(off + attention_ws_bytes(g.B, g.Lm, g.heads, g.dh, g.f32), 256);
+  // q, k, v and the projected attention output of toma_block_proj (four merged-size tensors)
+  l.proj_off = off;   off = align_up(off + 4 * align_up((size_t)g.B * g.Lm * g.d * esz, 256), 256);
   l.total = off;
   return l;
 }
@@ -283,12 +285,21 @@ toma_status toma_linear(int32_t m, int32_t n, int32_t k, int32_t dtype, const vo
   return cuda_ok(do_linear(m, n, k, dtype == TOMA_F32, a, ws, cs, 1, dev_status, (cudaStream_t)stream));
 }
 
-toma_status toma_block(const toma_desc* desc, int32_t step, const void* x, void* out, int32_t* idx_state,
-                       void* w_state, void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream) {
+// The wrapped module F: attention over the merged tokens with Q = K = V = X_m, or, with projection weights
+// (proj = {wq, wk, wv, wo}, each [dim][dim], row-major [in][out]), the whole attention module
+// (X_m wq, X_m wk, X_m wv -> attention -> wo).
+static toma_status block_impl(const toma_desc* desc, int32_t step, const void* x, const void* const* proj, void* out,
+                              int32_t* idx_state, void* w_state, void* ws, size_t ws_bytes, uint32_t* dev_status,
+                              void* stream) {
   Geom g;
   toma_status st = make_geom(desc, &g);
   if (st != TOMA_OK) return st;
   if (!x || !out || !idx_state || !w_state) return TOMA_ERR_NULL;
+  if (proj)
+    for (int i = 0; i < 4; ++i) {
+      if (!proj[i]) return TOMA_ERR_NULL;
+      if (misaligned(proj[i])) return TOMA_ERR_SHAPE;
+    }
   if (step < 0) return TOMA_ERR_SHAPE;
   if (misaligned(x) || misaligned(out) || misaligned(w_state)) return TOMA_ERR_SHAPE;
   if (!attention_supported_simt(g.dh)) return TOMA_ERR_UNSUPPORTED;
@@ -308,8 +319,65 @@ toma_status toma_block(const toma_desc* desc, int32_t step, const void* x, void*
   bool tickets_clean = false;
   const size_t ticket_bytes = attention_on_tc(g.dh, g.f32) ? attention_tc_ticket_bytes(g.B, g.Lm, g.heads) : 0;
   if (e == cudaSuccess) e = do_merge(g, w_state, x, xm, wsb + l.att_ws_off, ticket_bytes, &tickets_clean, dev_status, s);
-  if (e == cudaSuccess) e = do_attention(g.B, g.Lm, g.heads, g.dh, g.f32, xm, xm, xm, att, wsb + l.att_ws_off, tickets_clean, dev_status, s);
-  if (e == cudaSuccess) e = do_unmerge(g, w_state, att, out, dev_status, s);
+  if (!proj) {
+    if (e == cudaSuccess) e = do_attention(g.B, g.Lm, g.heads, g.dh, g.f32, xm, xm, xm, att, wsb + l.att_ws_off, tickets_clean, dev_status, s);
+    if (e == cudaSuccess) e = do_unmerge(g, w_state, att, out, dev_status, s);
+    return cuda_ok(e);
+  }
+  const size_t one = align_up((size_t)g.B * g.Lm * g.d * (g.f32 ? 4 : 2), 256);
+  void* qkv[3] = {wsb + l.proj_off, wsb + l.proj_off + one, wsb + l.proj_off + 2 * one};
+  void* y = wsb + l.proj_off + 3 * one;
+  const int rows = g.B * g.Lm;
+  if (e == cudaSuccess) e = do_linear(rows, g.d, g.d, g.f32, xm, proj, qkv, 3, dev_status, s);
+  if (e == cudaSuccess) e = do_attention(g.B, g.Lm, g.heads, g.dh, g.f32, qkv[0], qkv[1], qkv[2], att, wsb + l.att_ws_off, tickets_clean, dev_status, s);
+  void* ys[1] = {y};
+  if (e == cudaSuccess) e = do_linear(rows, g.d, g.d, g.f32, att, proj + 3, ys, 1, dev_status, s);
+  if (e == cudaSuccess) e = do_unmerge(g, w_state, y, out, dev_status, s);
+  return cuda_ok(e);
+}
+
+toma_status toma_block(const toma_desc* desc, int32_t step, const void* x, void* out, int32_t* idx_state,
+                       void* w_state, void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream) {
+  return block_impl(desc, step, x, nullptr, out, idx_state, w_state, ws, ws_bytes, dev_status, stream);
+}
+
+toma_status toma_block_proj(const toma_desc* desc, int32_t step, const void* x, const void* wq, const void* wk,
+                            const void* wv, const void* wo, void* out, int32_t* idx_state, void* w_state, void* ws,
+                            size_t ws_bytes, uint32_t* dev_status, void* stream) {
+  const void* proj[4] = {wq, wk, wv, wo};
+  return block_impl(desc, step, x, proj, out, idx_state, w_state, ws, ws_bytes, dev_status, stream);
+}
+
+size_t toma_attention_proj_workspace_bytes(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim, int32_t dtype) {
+  if ((dtype != TOMA_BF16 && dtype != TOMA_F32) || batch < 1 || len < 1 || n_heads < 1 || head_dim < 1) return 0;
+  const size_t one = align_up((size_t)batch * len * n_heads * head_dim * (dtype == TOMA_F32 ? 4 : 2), 256);
+  return 4 * one + align_up(attention_ws_bytes(batch, len, n_heads, head_dim, dtype == TOMA_F32), 256);
+}
+
+toma_status toma_attention_proj(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim, int32_t dtype, const void* x,
+                                const void* wq, const void* wk, const void* wv, const void* wo, void* out, void* ws,
+                                size_t ws_bytes, uint32_t* dev_status, void* stream) {
+  if (dtype != TOMA_BF16 && dtype != TOMA_F32) return TOMA_ERR_DTYPE;
+  if (batch < 1 || len < 1 || n_heads < 1 || head_dim < 1) return TOMA_ERR_SHAPE;
+  if (!x || !wq || !wk || !wv || !wo || !out) return TOMA_ERR_NULL;
+  if (misaligned(x) || misaligned(wq) || misaligned(wk) || misaligned(wv) || misaligned(wo) || misaligned(out)) return TOMA_ERR_SHAPE;
+  if (!attention_supported_simt(head_dim)) return TOMA_ERR_UNSUPPORTED;
+  const bool f32 = dtype == TOMA_F32;
+  const int d = n_heads * head_dim;
+  if (d % 8) return TOMA_ERR_SHAPE;
+  if (!ws || misaligned(ws) || ws_bytes < toma_attention_proj_workspace_bytes(batch, len, n_heads, head_dim, dtype)) return TOMA_ERR_WORKSPACE;
+  cudaStream_t s = (cudaStream_t)stream;
+  char* wsb = (char*)ws;
+  const size_t one = align_up((size_t)batch * len * d * (f32 ? 4 : 2), 256);
+  void* qkv[3] = {wsb, wsb + one, wsb + 2 * one};
+  void* att = wsb + 3 * one;
+  void* att_ws = wsb + 4 * one;
+  const void* proj[4] = {wq, wk, wv, wo};
+  const int rows = batch * len;
+  cudaError_t e = do_linear(rows, d, d, f32, x, proj, qkv, 3, dev_status, s);
+  if (e == cudaSuccess) e = do_attention(batch, len, n_heads, head_dim, f32, qkv[0], qkv[1], qkv[2], att, att_ws, false, dev_status, s);
+  void* outs[1] = {out};
+  if (e == cudaSuccess) e = do_linear(rows, d, d, f32, att, proj + 3, outs, 1, dev_status, s);
   return cuda_ok(e);
 }
 

@@ -33,7 +33,7 @@ toma_status make_geom(const toma_desc* desc, Geom* g);
 
 // Workspace carve-up (all offsets 256-byte aligned).
 struct WsLayout {
-  size_t y_off, sq_off, logits_off, wts_off, gidx_off, xm_off, att_off, att_ws_off, total;
+  size_t y_off, sq_off, logits_off, wts_off, gidx_off, xm_off, att_off, att_ws_off, proj_off, total;
 };
 WsLayout ws_layout(const Geom& g);
 // Geometry the weights, the merge and the unmerge work in: g itself, or, with global merge, the image as

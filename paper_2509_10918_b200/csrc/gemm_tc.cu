@@ -20,7 +20,6 @@ namespace {
 constexpr int kKC = 64;                  // contraction elements per stage
 constexpr int kSlab = kKC * 128;         // [64 k][64 n] slab of W, 128-byte rows
 constexpr int kABytes = 128 * 128;       // [128 m][64 k] slab of A
-constexpr int kColBlock = 320;           // output columns per CTA
 
 struct GemmBars {
   uint64_t full[4], empty[4], done;
@@ -32,6 +31,10 @@ struct GemmOut {
   __nv_bfloat16* c[3];
 };
 
+// kCols = 320: two accumulators (192 + 128 columns), 512 tensor-memory columns, one CTA per SM, deep ring.
+// kCols = 256: one accumulator, 256 tensor-memory columns, two CTAs per SM, for grids that would otherwise
+// spill into a second wave or leave most SMs idle.
+template <int kCols>
 __global__ void __launch_bounds__(192, 1)
 linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w0,
                    const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2, GemmOut out, int M,
@@ -39,16 +42,17 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * 128, n0 = blockIdx.y * kColBlock;
+  constexpr int kFirst = kCols == 320 ? 3 : 4;  // 64-column slabs of the first accumulator
+  const int m0 = blockIdx.x * 128, n0 = blockIdx.y * kCols;
   const CUtensorMap* tm_w = blockIdx.z == 0 ? &tm_w0 : blockIdx.z == 1 ? &tm_w1 : &tm_w2;
   __nv_bfloat16* c = out.c[blockIdx.z];
-  const int n_cols = min(kColBlock, N - n0);     // columns of this CTA (multiple of 8)
+  const int n_cols = min(kCols, N - n0);         // columns of this CTA (multiple of 8)
   const int slabs = (n_cols + 63) / 64;
-  const int n_a = min(slabs, 3) * 64, n_b = (slabs - min(slabs, 3)) * 64;
+  const int n_a = min(slabs, kFirst) * 64, n_b = (slabs - min(slabs, kFirst)) * 64;
   const int stage_bytes = kABytes + slabs * kSlab;
   GemmBars* bar = reinterpret_cast<GemmBars*>(smem + stages * stage_bytes);
   const int nk = (K + kKC - 1) / kKC;
-  constexpr uint32_t ncols = 512;
+  constexpr uint32_t ncols = kCols == 320 ? 512 : 256;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -95,7 +99,7 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
         for (int kk = 0; kk < ksteps; ++kk) {
           const uint64_t ad = smem_desc_sw128(aa + kk * 32, 16, 1024);
           mma_ss(tmem, ad, smem_desc_sw128(wa + kk * 2048, kSlab, 1024), idesc_a, k > 0 || kk > 0);
-          if (n_b > 0) mma_ss(tmem + 192, ad, smem_desc_sw128(wa + 3 * kSlab + kk * 2048, kSlab, 1024), idesc_b, k > 0 || kk > 0);
+          if (n_b > 0) mma_ss(tmem + kFirst * 64, ad, smem_desc_sw128(wa + kFirst * kSlab + kk * 2048, kSlab, 1024), idesc_b, k > 0 || kk > 0);
         }
         mma_commit(&bar->empty[s]);
       }
@@ -155,22 +159,33 @@ cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* con
     if (!encode_tmap_16bit(&tw[i], w[j], 2, wdims, wstr, wbox)) return cudaErrorInvalidValue;
     out.c[i] = (__nv_bfloat16*)c[j];
   }
-  const int slabs = ((N < kColBlock ? N : kColBlock) + 63) / 64;
+  // Column block: 320 (one CTA per SM, deep ring) unless that grid overflows the SMs into a second wave or
+  // fills less than half of them while the 256-column form (two CTAs per SM) fits one wave.
+  int sms = 148, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int mb = (M + 127) / 128;
+  const int ctas320 = mb * ((N + 319) / 320) * n_mats, ctas256 = mb * ((N + 255) / 256) * n_mats;
+  const bool narrow = ctas256 <= 2 * sms && (ctas320 > sms || 2 * ctas320 < sms);
+  const int cols = narrow ? 256 : 320;
+  const int slabs = ((N < cols ? N : cols) + 63) / 64;
   const int stage_bytes = kABytes + slabs * kSlab;
-  int stages = (222 * 1024) / stage_bytes;
-  stages = stages > 4 ? 4 : stages;
+  int stages = ((narrow ? 110 : 222) * 1024) / stage_bytes;
+  stages = stages > 4 ? 4 : stages < 1 ? 1 : stages;
   const int nk = (K + kKC - 1) / kKC;
   if (stages > nk) stages = nk;
   const int smem = 1024 + stages * stage_bytes + 256;
   static bool attr = false;
   if (!attr) {
-    cudaError_t e = cudaFuncSetAttribute(linear_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(linear_rows_kernel<320>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(linear_rows_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr = true;
   }
-  dim3 grid((M + 127) / 128, (N + kColBlock - 1) / kColBlock, n_mats);
-  cudaError_t e = launch_dependent(linear_rows_kernel, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out, M, N, K,
-                                   stages, dev_status);
+  dim3 grid(mb, (N + cols - 1) / cols, n_mats);
+  cudaError_t e = narrow ? launch_dependent(linear_rows_kernel<256>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out,
+                                            M, N, K, stages, dev_status)
+                         : launch_dependent(linear_rows_kernel<320>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out,
+                                            M, N, K, stages, dev_status);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }

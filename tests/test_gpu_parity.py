@@ -381,6 +381,67 @@ def test_linear_parity(toma, dtype, m, n, k):
     assert_close(to_host64(c)[rows], O.linear(a_host[rows], w_host), dtype, "linear")
 
 
+def _proj_weights(cfg, seed=93):
+    """Four [d, d] projection matrices N(0, 1/d), rounded to the storage dtype."""
+    d = cfg.dim
+    return [gen.round_to_dtype((gen.normal(0, (seed, i, d), d * d).reshape(d, d) / np.sqrt(d)).astype(np.float32), cfg.dtype)
+            for i in range(4)]
+
+
+def _storage_rounding(dtype):
+    return (lambda t: gen.round_to_dtype(np.asarray(t, dtype=np.float32), dtype).astype(np.float64)) if dtype == "bf16" \
+        else (lambda t: np.asarray(t, dtype=np.float32).astype(np.float64))
+
+
+@pytest.mark.parametrize("name,over", [("cfg2", dict(batch=1)), ("cfg3", dict(batch=1)), ("cfg1", {}),
+                                       ("cfg2", dict(batch=1, grid_h=16, grid_w=16, n_extra=9))],
+                         ids=["cfg2", "cfg3", "cfg1-f32", "extra-tokens"])
+def test_block_with_projections_parity(toma, name, over):
+    """toma_block_proj: the wrapped module is the whole attention module (Q/K/V projections, attention, output
+    projection) on the merged tokens.  The oracle mirrors the storage rounding between stages."""
+    cfg = gen.config(name, steps=2, reuse_interval=2, **over)
+    desc = toma.desc_from_config(cfg)
+    w_host = _proj_weights(cfg)
+    w_dev = [to_dev(w, cfg.dtype) for w in w_host]
+    idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    st = O.BlockState()
+    kw = dict(grid_h=cfg.grid_h, grid_w=cfg.grid_w, tile_h=cfg.tile_h, tile_w=cfg.tile_w, merge_ratio=cfg.merge_ratio,
+              tau=cfg.tau, n_heads=cfg.n_heads, reuse_interval=2, n_extra=cfg.n_extra,
+              proj=[x.astype(np.float64) for x in w_host], round_fn=_storage_rounding(cfg.dtype))
+    for step, x_host in enumerate(gen.feature_sequence(cfg)):
+        x = to_dev(x_host, cfg.dtype)
+        out = torch.empty_like(x)
+        toma.toma_block_proj(desc, step, x, *w_dev, out, idx, w, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        want, _, _ = O.block_step(x_host, step, st, **kw)
+        assert np.array_equal(idx.cpu().numpy().astype(np.int64), st.idx)
+        assert_close(to_host64(out), want, cfg.dtype, f"block with projections, step {step}")
+
+
+@pytest.mark.parametrize("dtype,B,L,h,dh", [("bf16", 2, 1024, 10, 64), ("bf16", 1, 600, 3, 128), ("f32", 1, 200, 2, 64)])
+def test_attention_module_with_projections_parity(toma, dtype, B, L, h, dh):
+    """toma_attention_proj (the full-token baseline of toma_block_proj) against the oracle."""
+    d = h * dh
+    cfg = gen.config("cfg2", batch=B, dim=d, n_heads=h, head_dim=dh, dtype=dtype)
+    x_host = gen.round_to_dtype(gen.normal(0, (94, L, d), B * L * d).reshape(B, L, d).astype(np.float32), dtype)
+    w_host = _proj_weights(cfg, seed=95)
+    x, w_dev = to_dev(x_host, dtype), [to_dev(w, dtype) for w in w_host]
+    out = torch.empty_like(x)
+    ws = torch.empty(toma.toma_attention_proj_workspace_bytes(B, L, h, dh, dtype), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    toma.toma_attention_proj(B, L, h, dh, dtype, x, *w_dev, out, ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rnd = _storage_rounding(dtype)
+    got = to_host64(out)
+    for b in range(B):
+        q, k, v = (rnd(O.linear(x_host[b], w)) for w in w_host[:3])
+        want = O.linear(rnd(O.attention(q, k, v, h)), w_host[3])
+        assert_close(got[b], want, dtype, f"attention module b={b}")
+
+
 def test_block_replays_from_a_cuda_graph(toma):
     """A reuse step and a refresh step captured into CUDA graphs (the calls never allocate or synchronise,
     and their dependent launches are capturable) replay to the same bits as direct calls."""
