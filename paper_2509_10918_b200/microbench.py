@@ -3,7 +3,7 @@
     python -m paper_2509_10918_b200.microbench --stage attention --workload cfg3 [--full-length] [--reps 50]
     python -m paper_2509_10918_b200.microbench --stage merge --workload cfg2
 
-Stages: select, weights, merge, attention, unmerge, block.  Prints one JSON line with median / min
+Stages: select, weights, merge, attention, unmerge, block, linear (--mnk m,n,k).  Prints one JSON line with median / min
 microseconds and the derived GB/s or TFLOP/s.  Also the command to run under ncu when a single
 kernel is to be profiled on a small case (--reps 3 --no-flush).
 """
@@ -22,7 +22,7 @@ if ROOT not in sys.path:
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--stage", required=True, choices=["select", "weights", "merge", "attention", "unmerge", "block"])
+    ap.add_argument("--stage", required=True, choices=["select", "weights", "merge", "attention", "unmerge", "block", "linear"])
     ap.add_argument("--workload", default="cfg3")
     ap.add_argument("--ratio", type=float, default=None)
     ap.add_argument("--full-length", action="store_true", help="attention over all N tokens instead of the merged D")
@@ -30,12 +30,35 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--no-flush", action="store_true")
     ap.add_argument("--global-merge", action="store_true", help="weights / merge / unmerge over the whole image")
+    ap.add_argument("--mnk", default="4096,1920,640", help="stage linear: rows, columns, contraction length")
     args = ap.parse_args()
 
     import torch
 
     import gen
     import paper_2509_10918_b200 as toma
+
+    if args.stage == "linear":  # projection c = a w, bf16
+        m, n, k = (int(v) for v in args.mnk.split(","))
+        a = torch.randn(m, k, device="cuda").bfloat16()
+        wmat = (torch.randn(k, n, device="cuda") / k ** 0.5).bfloat16()
+        c = torch.empty(m, n, device="cuda", dtype=torch.bfloat16)
+        flush = None if args.no_flush else torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        times = []
+        for it in range(args.warmup + args.reps):
+            if flush is not None:
+                flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            toma.toma_linear(a, wmat, c)
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                times.append(1e3 * e0.elapsed_time(e1))
+        med = statistics.median(times)
+        print(json.dumps({"stage": "linear", "m": m, "n": n, "k": k, "median_us": med, "min_us": min(times),
+                          "tflops_median": 2.0 * m * n * k / med / 1e6}))
+        return
 
     cfg = gen.config(args.workload) if args.ratio is None else gen.config(args.workload, merge_ratio=args.ratio)
     desc = toma.desc_from_config(cfg, global_merge=args.global_merge)
