@@ -85,7 +85,16 @@ typedef struct {
                                       weights, merge and unmerge run over all N image tokens (the paper's default
                                       variant, Sec. 5).  Merged rows keep the tile-major pick order; the weight
                                       buffer then holds A~^T as [batch][N][D] and is far larger */
+  int32_t unmerge_mode;            /* matrix toma_unmerge applies (Sec. 4.2.2): TOMA_UNMERGE_TRANSPOSE (0), the
+                                      transpose A~^T of the merge weights, Algorithm 3's choice;
+                                      TOMA_UNMERGE_SHARES (1), the transpose A^T of the column-stochastic
+                                      softmax matrix before its rows are normalised: every source token gets
+                                      the convex combination of the destinations' outputs given by its own
+                                      softmax shares, so a constant input comes back unchanged.  A non-zero mode
+                                      keeps a second matrix in the weight buffer (twice the size) */
 } toma_desc;
+
+enum { TOMA_UNMERGE_TRANSPOSE = 0, TOMA_UNMERGE_SHARES = 1 };
 
 /* Host-only helpers.  Return 0 / negative on an invalid descriptor. */
 TOMA_API size_t toma_workspace_bytes(const toma_desc* desc);   /* scratch needed by select / merge_weights / block */
@@ -225,6 +234,10 @@ TOMA_API toma_status toma_block_host(const toma_desc* desc, int32_t step, const 
  * one-hot matrix makes merge a hard ToMeSD-style merge, Sec. 4.2). */
 TOMA_API toma_status toma_weights_export(const toma_desc* desc, const void* w, float* dense, void* stream);
 TOMA_API toma_status toma_weights_import(const toma_desc* desc, const float* dense, void* w, void* stream);
+/* The matrix toma_unmerge applies, transposed back to dense fp32 [batch][P][D_loc][N_loc]: A~ itself with
+ * TOMA_UNMERGE_TRANSPOSE, the second matrix of the weight buffer otherwise.  With a non-zero unmerge_mode
+ * toma_weights_import fills both matrices with `dense`. */
+TOMA_API toma_status toma_unmerge_weights_export(const toma_desc* desc, const void* w, float* dense, void* stream);
 
 #ifdef __cplusplus
 }

@@ -188,6 +188,21 @@ def select_tile_definition(x_tile: np.ndarray, d_loc: int) -> np.ndarray:
 # ----------------------------------------------------------------------------
 
 
+def softmax_shares(x_tile: np.ndarray, idx: np.ndarray, tau: float) -> np.ndarray:
+    """A [D_loc, N_loc] for one region: the softmax of Sec. 4.2.1 before its rows are normalised.
+
+    logits  L_ik = <X[idx_i], X_k> / (tau * sqrt(d));  A_ik = softmax over the destination axis i,
+    separately for every source token k, so every column of A sums to 1.
+    """
+    x = np.asarray(x_tile, dtype=np.float64)
+    d = x.shape[1]
+    dest = x[np.asarray(idx, dtype=np.int64)]
+    L = (dest @ x.T) / (tau * np.sqrt(float(d)))
+    L = L - L.max(axis=0, keepdims=True)
+    E = np.exp(L)
+    return E / E.sum(axis=0, keepdims=True)
+
+
 def merge_weights(x_tile: np.ndarray, idx: np.ndarray, tau: float) -> np.ndarray:
     """A~ [D_loc, N_loc] for one region.
 
@@ -198,13 +213,7 @@ def merge_weights(x_tile: np.ndarray, idx: np.ndarray, tau: float) -> np.ndarray
               shares that sum to 1)
     A~_ik   = A_ik / sum_k' A_ik'  (row normalisation; Algorithm 3, A / A.sum(-1))
     """
-    x = np.asarray(x_tile, dtype=np.float64)
-    d = x.shape[1]
-    dest = x[np.asarray(idx, dtype=np.int64)]
-    L = (dest @ x.T) / (tau * np.sqrt(float(d)))
-    L = L - L.max(axis=0, keepdims=True)
-    E = np.exp(L)
-    A = E / E.sum(axis=0, keepdims=True)
+    A = softmax_shares(x_tile, idx, tau)
     Z = A.sum(axis=1, keepdims=True)
     return A / Z
 
@@ -215,7 +224,10 @@ def merge(w: np.ndarray, x_tile: np.ndarray) -> np.ndarray:
 
 
 def unmerge(w: np.ndarray, y_tile: np.ndarray) -> np.ndarray:
-    """X'_unmerged = A~^T X'  (Sec. 4.2.2, transpose unmerge)."""
+    """X'_unmerged = A~^T X'  (Sec. 4.2.2, transpose unmerge).
+
+    Passing the column-stochastic A of softmax_shares instead of A~ gives the "shares" variant: every
+    source token receives the convex combination sum_i A_ik X'_i of the destinations' outputs."""
     return np.asarray(w, dtype=np.float64).T @ np.asarray(y_tile, dtype=np.float64)
 
 
@@ -271,13 +283,14 @@ class BlockState:
     """Cached selection and weights of one batch (what Sec. 4.3.2 reuses)."""
     idx: Optional[np.ndarray] = None      # [B, P, D_loc] local indices, pick order
     w: Optional[np.ndarray] = None        # [B, P, D_loc, N_loc]
+    u: Optional[np.ndarray] = None        # matrix the unmerge applies (w itself, or the shares A), same shape
     margins: List[float] = field(default_factory=list)
 
 
 def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid_w: int,
                tile_h: int, tile_w: int, merge_ratio: float, tau: float, n_heads: int,
                reuse_interval: int, n_extra: int = 0, round_fn=None, weight_reuse_interval: int = 0,
-               global_merge: bool = False, proj=None):
+               global_merge: bool = False, proj=None, unmerge_mode: str = "transpose"):
     """One ToMA-wrapped attention call (Algorithm 3) on x [B, N + n_extra, d].
 
     Selection and weights are recomputed when step % reuse_interval == 0 and
@@ -296,6 +309,9 @@ def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid
     With proj = (wq, wk, wv, wo), each [d, d] as [in, out], the wrapped module is the whole attention
     module: attention(X_m wq, X_m wk, X_m wv) wo (Algorithm 3 applies F to the merged tokens; App. C's
     4 d^2 N term).  round_fn is then also applied to q, k, v and to the projected output.
+
+    unmerge_mode "transpose" applies A~^T (Algorithm 3); "shares" applies A^T, the softmax matrix
+    before row normalisation (columns sum to 1).
 
     `round_fn`, if given, is applied to the merged and to the attended tensor; it
     lets a test mirror the storage rounding between stages.  Returns
@@ -316,15 +332,22 @@ def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid
             for p in range(P):
                 state.idx[b, p], mg = select_tile(x[b, ids[p]], d_loc)
                 state.margins.append(mg)
+    if unmerge_mode not in ("transpose", "shares"):
+        raise ValueError(unmerge_mode)
     if refresh_w and global_merge:
         state.w = np.empty((B, 1, D, N), dtype=np.float64)
+        state.u = np.empty_like(state.w)
         for b in range(B):
-            state.w[b, 0] = merge_weights(x[b, :N], global_destinations(state.idx[b], ids), tau)
+            state.u[b, 0] = softmax_shares(x[b, :N], global_destinations(state.idx[b], ids), tau)
+            state.w[b, 0] = state.u[b, 0] / state.u[b, 0].sum(axis=1, keepdims=True)
     elif refresh_w:
         state.w = np.empty((B, P, d_loc, n_loc), dtype=np.float64)
+        state.u = np.empty_like(state.w)
         for b in range(B):
             for p in range(P):
-                state.w[b, p] = merge_weights(x[b, ids[p]], state.idx[b, p], tau)
+                state.u[b, p] = softmax_shares(x[b, ids[p]], state.idx[b, p], tau)
+                state.w[b, p] = state.u[b, p] / state.u[b, p].sum(axis=1, keepdims=True)
+    u = state.w if unmerge_mode == "transpose" else state.u
     merged = np.empty((B, D + n_extra, d), dtype=np.float64)
     for b in range(B):
         if global_merge:
@@ -348,10 +371,10 @@ def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid
     out = np.empty((B, n_all, d), dtype=np.float64)
     for b in range(B):
         if global_merge:
-            out[b, :N] = unmerge(state.w[b, 0], attended[b, :D])
+            out[b, :N] = unmerge(u[b, 0], attended[b, :D])
         else:
             for p in range(P):
-                out[b, ids[p]] = unmerge(state.w[b, p], attended[b, p * d_loc:(p + 1) * d_loc])
+                out[b, ids[p]] = unmerge(u[b, p], attended[b, p * d_loc:(p + 1) * d_loc])
         out[b, N:] = attended[b, D:]
     return out, merged, attended
 

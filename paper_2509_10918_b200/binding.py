@@ -23,7 +23,9 @@ EXPORTS = ["toma_select_static", "toma_launch_counter", "toma_workspace_bytes", 
            "toma_select", "toma_merge_weights", "toma_merge", "toma_attention_workspace_bytes", "toma_attention_plan", "toma_attention",
            "toma_unmerge", "toma_block", "toma_block_host", "toma_linear", "toma_block_proj", "toma_attention_proj_workspace_bytes",
            "toma_attention_proj",
-           "toma_weights_export", "toma_weights_import"]
+           "toma_weights_export", "toma_weights_import", "toma_unmerge_weights_export"]
+
+UNMERGE_MODES = {"transpose": 0, "shares": 1}
 
 
 class TomaDesc(Structure):
@@ -33,7 +35,7 @@ class TomaDesc(Structure):
         ("merge_ratio", c_float), ("tau", c_float),
         ("reuse_interval", c_int32), ("weight_reuse_interval", c_int32),
         ("n_heads", c_int32), ("head_dim", c_int32), ("n_extra", c_int32), ("dtype", c_int32),
-        ("global_merge", c_int32),
+        ("global_merge", c_int32), ("unmerge_mode", c_int32),
     ]
 
 
@@ -98,6 +100,8 @@ def _load() -> ctypes.CDLL:
     lib.toma_weights_export.argtypes = [P, c_void_p, c_void_p, c_void_p]
     lib.toma_weights_import.restype = c_int32
     lib.toma_weights_import.argtypes = [P, c_void_p, c_void_p, c_void_p]
+    lib.toma_unmerge_weights_export.restype = c_int32
+    lib.toma_unmerge_weights_export.argtypes = [P, c_void_p, c_void_p, c_void_p]
     return lib
 
 
@@ -105,10 +109,12 @@ lib = _load()
 
 
 def make_desc(*, batch, grid_h, grid_w, dim, tile_h, tile_w, merge_ratio, tau, n_heads, head_dim, dtype,
-              reuse_interval=1, weight_reuse_interval=0, n_extra=0, global_merge=False) -> TomaDesc:
+              reuse_interval=1, weight_reuse_interval=0, n_extra=0, global_merge=False,
+              unmerge_mode="transpose") -> TomaDesc:
     code = {"bf16": TOMA_BF16, "f32": TOMA_F32, TOMA_BF16: TOMA_BF16, TOMA_F32: TOMA_F32}[dtype]
     return TomaDesc(batch, grid_h, grid_w, dim, tile_h, tile_w, merge_ratio, tau, reuse_interval,
-                    weight_reuse_interval, n_heads, head_dim, n_extra, code, 1 if global_merge else 0)
+                    weight_reuse_interval, n_heads, head_dim, n_extra, code, 1 if global_merge else 0,
+                    UNMERGE_MODES.get(unmerge_mode, unmerge_mode))
 
 
 def desc_from_config(cfg, **overrides) -> TomaDesc:
@@ -279,6 +285,11 @@ def toma_block_host(desc, step, x_host, out_host, x_dev, out_dev, idx_state, w_s
 
 def toma_weights_export(desc, w, dense):
     _check(lib.toma_weights_export(ctypes.byref(desc), _ptr(w), _ptr(dense), _stream()), "toma_weights_export")
+
+
+def toma_unmerge_weights_export(desc, w, dense):
+    _check(lib.toma_unmerge_weights_export(ctypes.byref(desc), _ptr(w), _ptr(dense), _stream()),
+           "toma_unmerge_weights_export")
 
 
 def toma_weights_import(desc, dense, w):

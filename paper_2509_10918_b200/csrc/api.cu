@@ -38,6 +38,8 @@ toma_status make_geom(const toma_desc* desc, Geom* g) {
   if (desc->global_merge != 0 && desc->global_merge != 1) return TOMA_ERR_SHAPE;
   g->global_merge = desc->global_merge == 1;
   if (g->global_merge && (long long)g->N * g->D > (1ll << 27)) return TOMA_ERR_UNSUPPORTED;  // dense D x N weights per image
+  if (desc->unmerge_mode != TOMA_UNMERGE_TRANSPOSE && desc->unmerge_mode != TOMA_UNMERGE_SHARES) return TOMA_ERR_SHAPE;
+  g->unmerge_mode = desc->unmerge_mode;
   g->logit_scale = (float)(1.0 / ((double)desc->tau * sqrt((double)desc->dim)));
   return TOMA_OK;
 }
@@ -46,6 +48,16 @@ static bool attention_on_tc(int dh, bool f32) { return !f32 && (dh == 64 || dh =
 
 static size_t attention_ws_bytes(int B, int L, int heads, int dh, bool f32) {
   return attention_on_tc(dh, f32) ? attention_tc_workspace_bytes(B, L, heads, dh) : 0;
+}
+
+// Bytes of one matrix of the weight buffer (one fp32 plane, or a hi and a lo bf16 plane, per region).
+static size_t weight_matrix_bytes(const Geom& g) {
+  const Geom gm = merge_geom(g);
+  return (size_t)gm.B * gm.P * gm.Nloc * gm.Dloc * 4;
+}
+// The matrix toma_unmerge reads.
+static const void* unmerge_matrix(const Geom& g, const void* w) {
+  return g.unmerge_mode == TOMA_UNMERGE_TRANSPOSE ? w : (const char*)w + weight_matrix_bytes(g);
 }
 
 Geom merge_geom(const Geom& g) {
@@ -112,9 +124,10 @@ static cudaError_t do_weights(const Geom& g, const void* x, const int32_t* idx, 
     if (e != cudaSuccess) return e;
     idx = gidx;
   }
+  void* wu = g.unmerge_mode == TOMA_UNMERGE_SHARES ? (char*)w + weight_matrix_bytes(g) : nullptr;
   if (weights_tc_supported(gm))
-    return launch_weights_tc(gm, x, idx, w, (float*)(ws + l.logits_off), ws + l.wts_off, dev_status, s);
-  return launch_weights_simt(gm, x, idx, w, (float*)(ws + l.logits_off), s);
+    return launch_weights_tc(gm, x, idx, w, wu, (float*)(ws + l.logits_off), ws + l.wts_off, dev_status, s);
+  return launch_weights_simt(gm, x, idx, w, wu, (float*)(ws + l.logits_off), s);
 }
 
 // `zero`, `zero_bytes`: a region to clear on the side; *zeroed says whether the path taken did it.
@@ -133,6 +146,7 @@ static cudaError_t do_merge(const Geom& g_sel, const void* w, const void* x, voi
 static cudaError_t do_unmerge(const Geom& g_sel, const void* w, const void* y, void* out, uint32_t* dev_status,
                               cudaStream_t s) {
   const Geom g = merge_geom(g_sel);
+  w = unmerge_matrix(g_sel, w);
   if (linear_tc_supported(g)) {
     cudaError_t e = launch_unmerge_tc(g, w, y, out, dev_status, s);
     return e != cudaSuccess ? e : launch_copy_extra(g, y, out, false, s);
@@ -168,8 +182,7 @@ size_t toma_workspace_bytes(const toma_desc* desc) {
 size_t toma_weights_bytes(const toma_desc* desc) {
   Geom g;
   if (make_geom(desc, &g) != TOMA_OK) return 0;
-  const Geom gm = merge_geom(g);
-  return (size_t)gm.B * gm.P * gm.Nloc * gm.Dloc * 4;  // one fp32 plane, or a hi and a lo bf16 plane
+  return weight_matrix_bytes(g) * (g.unmerge_mode == TOMA_UNMERGE_TRANSPOSE ? 1 : 2);
 }
 
 int32_t toma_dest_per_tile(const toma_desc* desc) {
@@ -421,7 +434,18 @@ toma_status toma_weights_import(const toma_desc* desc, const float* dense, void*
   toma_status st = make_geom(desc, &g);
   if (st != TOMA_OK) return st;
   if (!w || !dense) return TOMA_ERR_NULL;
-  return cuda_ok(launch_weights_import(merge_geom(g), dense, w, (cudaStream_t)stream));
+  cudaError_t e = launch_weights_import(merge_geom(g), dense, w, (cudaStream_t)stream);
+  if (e == cudaSuccess && g.unmerge_mode != TOMA_UNMERGE_TRANSPOSE)
+    e = launch_weights_import(merge_geom(g), dense, (char*)w + weight_matrix_bytes(g), (cudaStream_t)stream);
+  return cuda_ok(e);
+}
+
+toma_status toma_unmerge_weights_export(const toma_desc* desc, const void* w, float* dense, void* stream) {
+  Geom g;
+  toma_status st = make_geom(desc, &g);
+  if (st != TOMA_OK) return st;
+  if (!w || !dense) return TOMA_ERR_NULL;
+  return cuda_ok(launch_weights_export(merge_geom(g), unmerge_matrix(g, w), dense, (cudaStream_t)stream));
 }
 
 }  // extern "C"

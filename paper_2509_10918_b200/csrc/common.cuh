@@ -25,6 +25,7 @@ struct Geom {
   int heads, dh;
   bool f32;
   bool global_merge;  // weights / merge / unmerge over the whole image (selection stays per tile)
+  int unmerge_mode;   // TOMA_UNMERGE_*: a non-zero mode keeps a second matrix behind A~^T in the weight buffer
   float logit_scale;  // 1 / (tau * sqrt(d))
   long long tokens_all() const { return (long long)N + n_extra; }
 };
@@ -50,7 +51,8 @@ cudaError_t launch_gram_ffma(const Geom& g, const __nv_bfloat16* y, int16_t* sq,
 bool gram_tc_supported(const Geom& g);
 cudaError_t launch_gram_tc(const Geom& g, const __nv_bfloat16* y, int16_t* sq, uint32_t* dev_status, cudaStream_t s);
 cudaError_t launch_greedy(const Geom& g, const int16_t* sq, int32_t* idx, cudaStream_t s);
-cudaError_t launch_weights_simt(const Geom& g, const void* x, const int32_t* idx, void* w, float* logits,
+// `wu`: where the un-normalised shares A^T go in the weight buffer's layout, or nullptr.
+cudaError_t launch_weights_simt(const Geom& g, const void* x, const int32_t* idx, void* w, void* wu, float* logits,
                                 cudaStream_t s);
 cudaError_t launch_merge_simt(const Geom& g, const void* w, const void* x, void* xm, cudaStream_t s);
 cudaError_t launch_unmerge_simt(const Geom& g, const void* w, const void* y, void* out, cudaStream_t s);
@@ -58,8 +60,8 @@ cudaError_t launch_attention_simt(int B, int L, int heads, int dh, bool f32, con
                                   const void* v, void* o, cudaStream_t s);
 bool weights_tc_supported(const Geom& g);
 size_t weights_tc_scratch_bytes(const Geom& g);
-cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, void* w, float* shares, void* scratch,
-                              uint32_t* dev_status, cudaStream_t s);
+cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, void* w, void* wu, float* shares,
+                              void* scratch, uint32_t* dev_status, cudaStream_t s);
 bool linear_tc_supported(const Geom& g);
 // `zero` / `zero_bytes` (multiple of 4, may be 0): a region the kernel clears on the side.
 cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* xm, void* zero, size_t zero_bytes,

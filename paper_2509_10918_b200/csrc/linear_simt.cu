@@ -167,10 +167,11 @@ __global__ void __launch_bounds__(128) softmax_dest_kernel(float* __restrict__ l
   for (int i = 0; i < Dloc; ++i) L[(size_t)i * Nloc] *= inv;
 }
 
-// Row normalisation: one warp per (tile, destination i); writes A~^T[k][i] = A_ik / sum_k' A_ik'.
+// Row normalisation: one warp per (tile, destination i); writes A~^T[k][i] = A_ik / sum_k' A_ik'
+// and, when wu is given, the shares themselves, A^T[k][i] = A_ik, in the same layout.
 template <typename WT>
-__global__ void __launch_bounds__(256) rownorm_kernel(const float* __restrict__ A, WT* __restrict__ w, int Nloc,
-                                                      int Dloc, int rows_total) {
+__global__ void __launch_bounds__(256) rownorm_kernel(const float* __restrict__ A, WT* __restrict__ w, WT* __restrict__ wu,
+                                                      int Nloc, int Dloc, int rows_total) {
   const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (row >= rows_total) return;
@@ -183,9 +184,11 @@ __global__ void __launch_bounds__(256) rownorm_kernel(const float* __restrict__ 
   const float inv = z > 0.f ? 1.f / z : 0.f;
   const size_t plane = (size_t)Nloc * Dloc;
   for (int k = lane; k < Nloc; k += 32) w_store(w, batch, (size_t)k * Dloc + i, plane, a[k] * inv);
+  if (wu)
+    for (int k = lane; k < Nloc; k += 32) w_store(wu, batch, (size_t)k * Dloc + i, plane, a[k]);
 }
 
-cudaError_t launch_weights_simt(const Geom& g, const void* x, const int32_t* idx, void* w, float* logits,
+cudaError_t launch_weights_simt(const Geom& g, const void* x, const int32_t* idx, void* w, void* wu, float* logits,
                                 cudaStream_t s) {
   const int batches = g.B * g.P;
   if (g.f32) {
@@ -200,9 +203,9 @@ cudaError_t launch_weights_simt(const Geom& g, const void* x, const int32_t* idx
   const int rows = batches * g.Dloc;
   const int blocks = (rows * 32 + 255) / 256;
   if (g.f32)
-    rownorm_kernel<float><<<blocks, 256, 0, s>>>(logits, (float*)w, g.Nloc, g.Dloc, rows);
+    rownorm_kernel<float><<<blocks, 256, 0, s>>>(logits, (float*)w, (float*)wu, g.Nloc, g.Dloc, rows);
   else
-    rownorm_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(logits, (__nv_bfloat16*)w, g.Nloc, g.Dloc, rows);
+    rownorm_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(logits, (__nv_bfloat16*)w, (__nv_bfloat16*)wu, g.Nloc, g.Dloc, rows);
   count_launch();
   return cudaGetLastError();
 }

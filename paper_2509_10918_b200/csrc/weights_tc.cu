@@ -229,7 +229,8 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
 
 __global__ void __launch_bounds__(256)
 weights_normalise_kernel(const float* __restrict__ shares, const float* __restrict__ zpart, __nv_bfloat16* __restrict__ w,
-                         int Nloc, int Dloc, int mblocks) {
+                         __nv_bfloat16* __restrict__ wu, int Nloc, int Dloc, int mblocks) {
+  // wu (may be null): the shares themselves, A^T, in the same two-plane layout
   // grid (blocks over the tile's [N_loc][D_loc] plane in groups of four destinations, tile)
   extern __shared__ float zs[];  // reciprocal row sums of the tile's D_loc destinations
   dependency_wait();  // launched with programmatic stream serialisation
@@ -257,6 +258,16 @@ weights_normalise_kernel(const float* __restrict__ shares, const float* __restri
     }
     *reinterpret_cast<uint2*>(t + r) = *reinterpret_cast<const uint2*>(hi);
     *reinterpret_cast<uint2*>(t + plane + r) = *reinterpret_cast<const uint2*>(lo);
+    if (wu) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        hi[e] = __float2bfloat16_rn(in[e]);
+        lo[e] = __float2bfloat16_rn(in[e] - __bfloat162float(hi[e]));
+      }
+      __nv_bfloat16* u = wu + batch * 2 * plane;
+      *reinterpret_cast<uint2*>(u + r) = *reinterpret_cast<const uint2*>(hi);
+      *reinterpret_cast<uint2*>(u + plane + r) = *reinterpret_cast<const uint2*>(lo);
+    }
   }
 }
 
@@ -344,8 +355,8 @@ size_t weights_tc_scratch_bytes(const Geom& g) {  // gathered destinations + par
   return dest + tiles * (g.Nloc / m_tok) * g.Dloc * 4 + 256;
 }
 
-cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, void* w, float* shares, void* scratch,
-                              uint32_t* dev_status, cudaStream_t s) {
+cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, void* w, void* wu, float* shares,
+                              void* scratch, uint32_t* dev_status, cudaStream_t s) {
   const size_t tiles = (size_t)g.B * g.P;
   WParams p;
   p.P = g.P; p.tiles_x = g.tiles_x; p.th = g.th; p.tw = g.tw; p.W = g.W; p.Nloc = g.Nloc; p.Dloc = g.Dloc; p.d = g.d;
@@ -418,7 +429,7 @@ cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, 
     attr3 = true;
   }
   le = launch_dependent(weights_normalise_kernel, dim3((unsigned)nblocks, (unsigned)tiles), dim3(256), (size_t)g.Dloc * 4, s,
-                        (const float*)shares, zsrc, (__nv_bfloat16*)w, g.Nloc, g.Dloc, zblocks);
+                        (const float*)shares, zsrc, (__nv_bfloat16*)w, (__nv_bfloat16*)wu, g.Nloc, g.Dloc, zblocks);
   count_launch();
   return le != cudaSuccess ? le : cudaGetLastError();
 }

@@ -28,6 +28,12 @@ def test_every_declared_symbol_is_exported(toma):
     assert declared == set(toma.EXPORTS)
 
 
+def test_binding_declares_argument_types_for_every_entry_point(toma):
+    # without argtypes ctypes passes a Python int as a 32-bit C int and a device pointer loses its upper half
+    for name in toma.EXPORTS:
+        assert getattr(toma.lib, name).argtypes is not None, f"{name}: ctypes argtypes not declared"
+
+
 def _desc(toma, **kw):
     base = dict(batch=2, grid_h=64, grid_w=64, dim=640, tile_h=16, tile_w=16, merge_ratio=0.5, tau=0.1, n_heads=10,
                 head_dim=64, dtype="bf16")
@@ -51,12 +57,16 @@ def test_descriptor_validation(toma):
     d = _desc(toma)
     d.dtype = 5
     assert toma.toma_validate(d) == DTYPE
+    assert toma.toma_validate(_desc(toma, unmerge_mode="shares")) == OK
+    assert toma.toma_validate(_desc(toma, unmerge_mode=2)) == SHAPE
+    assert toma.toma_validate(_desc(toma, unmerge_mode=-1)) == SHAPE
 
 
 def test_sizes(toma):
     d = _desc(toma)
     assert toma.toma_dest_per_tile(d) == 128
     assert toma.toma_weights_bytes(d) == 2 * 16 * 256 * 128 * 4  # hi + lo bf16 planes
+    assert toma.toma_weights_bytes(_desc(toma, unmerge_mode="shares")) == 2 * toma.toma_weights_bytes(d)  # A~^T and A^T
     assert toma.toma_workspace_bytes(d) > 0
     assert toma.toma_dest_per_tile(_desc(toma, merge_ratio=0.25)) == 192
     assert toma.toma_dest_per_tile(_desc(toma, merge_ratio=0.75)) == 64

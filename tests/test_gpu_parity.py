@@ -362,6 +362,97 @@ def test_global_merge_block_parity_at_benchmark_size(toma):
         assert_close(to_host64(out), want, cfg.dtype, f"global-merge block step {step}")
 
 
+SHARES = [
+    # name, overrides, global merge
+    ("cfg1", {}, False),                                   # fp32, FFMA weights path
+    ("cfg2", dict(batch=1), False),                        # 8x8 tiles
+    ("cfg3", dict(batch=1), False),                        # the benchmark's tile shape
+    ("cfg4", dict(grid_h=32, grid_w=32, n_extra=7), False),  # 3072 channels, 128-wide heads, text tokens
+    ("cfg2", dict(batch=2, grid_h=32, grid_w=32, tile_h=8, tile_w=8, dim=128, n_heads=2, head_dim=64), True),
+    ("cfg3", dict(batch=1, grid_h=32, grid_w=32, merge_ratio=0.25), True),  # 768 destinations: blocked weights
+]
+
+
+@pytest.mark.parametrize("name,over,global_merge", SHARES, ids=[str(i) for i in range(len(SHARES))])
+def test_shares_unmerge_parity(toma, name, over, global_merge):
+    """unmerge_mode "shares": toma_unmerge applies A^T, the softmax matrix before row normalisation.  The
+    merge side is untouched; the second matrix of the weight buffer is the oracle's A; a constant comes
+    back as the same constant (columns of A sum to 1); the unmerged tensor matches the oracle's."""
+    cfg = gen.config(name, **over)
+    x_host = gen.features(cfg)
+    run = Run(toma, cfg, x_host, global_merge=global_merge, unmerge_mode="shares")
+    ref = Run(toma, cfg, x_host, global_merge=global_merge)
+    assert toma.toma_weights_bytes(run.desc) == 2 * toma.toma_weights_bytes(ref.desc)
+    idx = run.select()
+    ref.idx.copy_(run.idx)
+    N, D = cfg.n_tokens, cfg.n_merged
+    shape = (cfg.batch, 1, D, N) if global_merge else (cfg.batch, cfg.n_tiles, cfg.d_loc, cfg.n_loc)
+    for r in (run, ref):
+        r.t.toma_merge_weights(r.desc, r.x, r.idx, r.w, r.ws, r.status)
+        r.ok()
+    nb = toma.toma_weights_bytes(ref.desc)
+    assert torch.equal(run.w[:nb], ref.w[:nb]), "the merge matrix must not depend on the unmerge mode"
+    dense_u = torch.empty(shape, dtype=torch.float32, device="cuda")
+    toma.toma_unmerge_weights_export(run.desc, run.w, dense_u)
+    dense_t = torch.empty(shape, dtype=torch.float32, device="cuda")
+    toma.toma_unmerge_weights_export(ref.desc, ref.w, dense_t)
+    dense_w = torch.empty(shape, dtype=torch.float32, device="cuda")
+    toma.toma_weights_export(ref.desc, ref.w, dense_w)
+    torch.cuda.synchronize()
+    assert torch.equal(dense_t, dense_w), "transpose mode: the unmerge matrix is the merge matrix"
+    A = dense_u.cpu().numpy().astype(np.float64)
+    assert np.all(A >= 0) and np.abs(A.sum(axis=2) - 1.0).max() < (1e-5 if cfg.dtype == "f32" else 2e-3)
+    merged = run.merge()
+    assert np.array_equal(merged, ref.merge())
+    y_dev = run.attend()
+    y_host = to_host64(y_dev)
+    unmerged = run.unmerge(y_dev)
+    const = torch.full_like(y_dev, 1.5)
+    back = run.unmerge(const)
+    assert np.abs(back - 1.5).max() <= (1e-5 if cfg.dtype == "f32" else 2 ** -7), "partition of unity"
+    ids = O.tile_token_ids(cfg.grid_h, cfg.grid_w, cfg.tile_h, cfg.tile_w)
+    w_abs = 2e-5 if cfg.dtype == "f32" else 6e-4
+    if global_merge:
+        for b in range(cfg.batch):
+            x_img = x_host[b, :N].astype(np.float64)
+            want = O.softmax_shares(x_img, O.global_destinations(idx[b], ids), cfg.tau)
+            assert np.abs(A[b, 0] - want).max() <= w_abs
+            assert_close(unmerged[b, :N], O.unmerge(want, y_host[b, :D]), cfg.dtype, "global shares unmerge")
+    else:
+        got, want_u = [], []
+        for b, p in sample_tiles(cfg, 8):
+            xt = tile_tokens(cfg, x_host, b, p)
+            want = O.softmax_shares(xt, idx[b, p], cfg.tau)
+            assert np.abs(A[b, p] - want).max() <= w_abs, f"shares differ in tile ({b},{p})"
+            got.append(unmerged[b, ids[p]])
+            want_u.append(O.unmerge(want, y_host[b, p * cfg.d_loc:(p + 1) * cfg.d_loc]))
+        assert_close(np.stack(got), np.stack(want_u), cfg.dtype, "shares unmerge")
+    if cfg.n_extra:
+        assert np.array_equal(unmerged[:, N:], y_host[:, D:])
+
+
+@pytest.mark.parametrize("global_merge", [False, True])
+def test_block_with_shares_unmerge_parity(toma, global_merge):
+    """toma_block with unmerge_mode "shares" over a refresh, a weights-only and a reuse step."""
+    cfg = gen.config("cfg3", batch=1, steps=4, reuse_interval=4, grid_h=32, grid_w=32)
+    desc = toma.desc_from_config(cfg, global_merge=global_merge, unmerge_mode="shares", weight_reuse_interval=2)
+    idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    st = O.BlockState()
+    kw = dict(grid_h=cfg.grid_h, grid_w=cfg.grid_w, tile_h=cfg.tile_h, tile_w=cfg.tile_w, merge_ratio=cfg.merge_ratio,
+              tau=cfg.tau, n_heads=cfg.n_heads, reuse_interval=4, weight_reuse_interval=2, global_merge=global_merge,
+              unmerge_mode="shares")
+    for step, x_host in enumerate(gen.feature_sequence(cfg)):
+        x = to_dev(x_host, cfg.dtype)
+        out = torch.empty_like(x)
+        toma.toma_block(desc, step, x, out, idx, w, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        want, _, _ = O.block_step(x_host, step, st, **kw)
+        assert np.array_equal(idx.cpu().numpy().astype(np.int64), st.idx)
+        assert_close(to_host64(out), want, cfg.dtype, f"shares block step {step}")
+
+
 @pytest.mark.parametrize("dtype,m,n,k", [
     ("bf16", 4096, 640, 640), ("bf16", 4096, 1920, 640), ("bf16", 1000, 72, 200), ("bf16", 130, 320, 64),
     ("bf16", 128, 328, 640), ("bf16", 2560, 3072, 3072), ("f32", 300, 96, 160),

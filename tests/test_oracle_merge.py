@@ -182,3 +182,79 @@ def test_global_merge_reduces_to_tile_merge_for_one_tile_and_sees_across_tiles()
     # largest entry of the column is still the destination it copies
     w2 = O.merge_weights(x2[0, :64], gidx, c.tau)
     assert np.argmax(w2[:, other] * w2.shape[1]) == 0 or np.argmax(w2[:, other]) == 0
+
+
+def test_softmax_shares_closed_form_and_relation_to_merge_weights():
+    """The matrix of the "shares" unmerge: columns sum to 1 (a token's shares over the destinations),
+    A~ is A with its rows rescaled, and the closed form of the two-destination case."""
+    x = np.array([[1.0, 0, 0, 0], [0, 1.0, 0, 0], [math.log(3.0), 0, 0, 0]])
+    idx = np.array([0, 1])
+    A = O.softmax_shares(x, idx, 0.5)              # tau*sqrt(d) = 1
+    assert A[:, 2] == pytest.approx([3 / 4, 1 / 4])
+    e = math.e
+    assert A[:, 0] == pytest.approx([e / (e + 1), 1 / (e + 1)])  # destination 0 against itself and against 1
+    c = gen.config("cfg2", batch=1)
+    tile = O.split_regions(gen.features(c)[0], c.grid_h, c.grid_w, c.tile_h, c.tile_w)[3]
+    idx, _ = O.select_tile(tile, c.d_loc)
+    A = O.softmax_shares(tile, idx, c.tau)
+    w = O.merge_weights(tile, idx, c.tau)
+    assert np.all(A >= 0) and np.allclose(A.sum(axis=0), 1.0, atol=1e-12)
+    assert np.allclose(w * A.sum(axis=1, keepdims=True), A, rtol=1e-12, atol=0)
+
+
+def test_shares_unmerge_is_a_partition_of_unity_and_beats_the_transpose_on_round_trips():
+    """With the column-stochastic matrix every source token receives a convex combination of the
+    destinations' outputs: a constant comes back unchanged, outputs stay inside the destinations'
+    range, and unmerge(merge(x)) is closer to x than with A~^T, whose columns sum to about D/N."""
+    c = gen.config("cfg2", batch=1)
+    tile = O.split_regions(gen.features(c)[0], c.grid_h, c.grid_w, c.tile_h, c.tile_w)[5].astype(np.float64)
+    idx, _ = O.select_tile(tile, c.d_loc)
+    A = O.softmax_shares(tile, idx, c.tau)
+    w = O.merge_weights(tile, idx, c.tau)
+    const = np.full((c.d_loc, 7), 2.5)
+    assert np.allclose(O.unmerge(A, const), 2.5, atol=1e-12)
+    assert not np.allclose(O.unmerge(w, const), 2.5, atol=0.1)   # the transpose attenuates
+    y = np.random.default_rng(3).normal(size=(c.d_loc, 5))
+    un = O.unmerge(A, y)
+    assert np.all(un <= y.max(axis=0) + 1e-12) and np.all(un >= y.min(axis=0) - 1e-12)
+    merged = O.merge(w, tile)
+    err_t = np.linalg.norm(O.unmerge(w, merged) - tile) / np.linalg.norm(tile)
+    err_s = np.linalg.norm(O.unmerge(A, merged) - tile) / np.linalg.norm(tile)
+    assert err_s < err_t
+    # explicit loops: out_k = sum_i A_ik y_i
+    k = 11
+    assert np.allclose(un[k], sum(A[i, k] * y[i] for i in range(c.d_loc)), atol=1e-12)
+
+
+def test_shares_unmerge_on_orthogonal_groups_copies_the_prototype_output():
+    d, groups, rep = 16, 4, 3
+    x = np.repeat(np.eye(d)[:groups] * 3.0, rep, axis=0)
+    x = x + 0.01 * np.arange(x.size).reshape(x.shape) / x.size
+    idx, _ = O.select_tile(x, groups)
+    A = O.softmax_shares(x, idx, 0.05)  # cold softmax: hard assignment
+    member = np.repeat(np.arange(groups), rep)
+    y = np.arange(groups * d, dtype=np.float64).reshape(groups, d)
+    un = O.unmerge(A, y)
+    for k in range(groups * rep):
+        j = list(member[idx]).index(member[k])
+        assert np.allclose(un[k], y[j], atol=1e-5)   # (y_j / rep with the transpose unmerge)
+
+
+def test_block_step_unmerge_modes_differ_only_in_the_unmerge():
+    c = gen.config("cfg2", batch=1, grid_h=16, grid_w=16, dim=64, n_heads=1, head_dim=64)
+    x = gen.features(c)
+    kw = dict(grid_h=16, grid_w=16, tile_h=c.tile_h, tile_w=c.tile_w, merge_ratio=0.5, tau=c.tau, n_heads=1,
+              reuse_interval=1)
+    st_t, st_s = O.BlockState(), O.BlockState()
+    out_t, merged_t, att_t = O.block_step(x, 0, st_t, **kw)
+    out_s, merged_s, att_s = O.block_step(x, 0, st_s, unmerge_mode="shares", **kw)
+    assert np.array_equal(merged_t, merged_s) and np.array_equal(att_t, att_s)
+    assert np.array_equal(st_t.w, st_s.w) and np.array_equal(st_t.idx, st_s.idx)
+    ids = O.tile_token_ids(16, 16, c.tile_h, c.tile_w)
+    d_loc = c.d_loc
+    p = 2
+    want = st_s.u[0, p].T @ att_s[0, p * d_loc:(p + 1) * d_loc]
+    assert np.allclose(out_s[0, ids[p]], want, atol=1e-12)
+    assert not np.allclose(out_s, out_t, atol=1e-3)
+    with pytest.raises(ValueError):
+        O.block_step(x, 0, O.BlockState(), unmerge_mode="nope", **kw)
