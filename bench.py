@@ -231,6 +231,7 @@ def other_workloads(toma, torch, flush, peaks):
         del x, y, idx, w, ws
         torch.cuda.empty_cache()
     out["cfg3_attention_module"] = attention_module_workload(toma, torch, flush)
+    out["cfg3_mlp_module"] = mlp_module_workload(toma, torch, flush)
     return out
 
 
@@ -277,6 +278,47 @@ def attention_module_workload(toma, torch, flush):
     return {"tokens": B * N, "reuse_interval": k, "refresh_us": refresh, "reuse_us": reuse_us, "block_mean_us": mean,
             "full_module_us": full, "speedup_vs_full_module": full / mean,
             "one_projection_us": qkv, "one_projection_tflops": 2.0 * m * d * d / qkv / 1e6}
+
+
+def mlp_module_workload(toma, torch, flush):
+    """The benchmark workload with the MLP as the wrapped F (hidden width 4 d, GELU): toma_block_mlp on the
+    merged tokens against the same MLP on all tokens (toma_mlp).  Random N(0, 1/fan-in) weights."""
+    import gen
+    cfg = gen.config("cfg3")
+    desc = toma.desc_from_config(cfg)
+    tdt = toma.torch_dtype(desc)
+    x = torch.from_numpy(gen.features(cfg)).cuda().to(tdt)
+    y = torch.empty_like(x)
+    d, f = cfg.dim, 4 * cfg.dim
+    w1 = torch.from_numpy((gen.normal(0, (99, 1, d, f), d * f).reshape(d, f) / d ** 0.5).astype("float32")).cuda().to(tdt)
+    w2 = torch.from_numpy((gen.normal(0, (99, 2, d, f), d * f).reshape(f, d) / f ** 0.5).astype("float32")).cuda().to(tdt)
+    idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    B, N = cfg.batch, cfg.n_tokens
+    ws_full = torch.empty(toma.toma_mlp_workspace_bytes(B * N, d, f, cfg.dtype), dtype=torch.uint8, device="cuda")
+
+    def t_us(fn, reps=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(1e3 * e0.elapsed_time(e1))
+        return statistics.median(ts)
+
+    k = cfg.reuse_interval
+    refresh = t_us(lambda: toma.toma_block_mlp(desc, 0, x, w1, w2, y, idx, w, ws, None))
+    reuse_us = t_us(lambda: toma.toma_block_mlp(desc, 1, x, w1, w2, y, idx, w, ws, None))
+    full = t_us(lambda: toma.toma_mlp(B * N, d, f, cfg.dtype, x, w1, w2, y, ws_full, None))
+    mean = (refresh + (k - 1) * reuse_us) / k
+    return {"tokens": B * N, "hidden": f, "reuse_interval": k, "refresh_us": refresh, "reuse_us": reuse_us,
+            "block_mean_us": mean, "full_module_us": full, "speedup_vs_full_module": full / mean,
+            "full_module_tflops": 4.0 * B * N * d * f / full / 1e6}
 
 
 def main():

@@ -212,6 +212,23 @@ TOMA_API toma_status toma_attention_proj(int32_t batch, int32_t len, int32_t n_h
                                          const void* x, const void* wq, const void* wk, const void* wv, const void* wo,
                                          void* out, void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream);
 
+/* toma_block with the MLP as the wrapped F (Sec. 4.2.2: the merged tokens go through "Attention/MLP"):
+ * merge, H = GELU(X_m w1), Y = H w2, unmerge.  GELU(v) = v Phi(v) with the exact normal distribution
+ * function (erf), applied to the fp32 accumulator before H is stored in the dtype of x.
+ *   w1 [dim][hidden], w2 [hidden][dim]: row-major [in][out], device, dtype of x, no biases;
+ *   hidden: a multiple of 8, at most 4 * dim (H lives in the block's workspace).  TOMA_ERR_SHAPE otherwise.
+ * Everything else as toma_block (same workspace size; n_heads / head_dim are validated but unused). */
+TOMA_API toma_status toma_block_mlp(const toma_desc* desc, int32_t step, const void* x, const void* w1, const void* w2,
+                                    int32_t hidden, void* out, int32_t* idx_state, void* w_state, void* ws, size_t ws_bytes,
+                                    uint32_t* dev_status, void* stream);
+
+/* The same MLP on all rows, without ToMA: out = GELU(x w1) w2, x and out [rows][dim].  The full-token baseline
+ * of toma_block_mlp.  ws: device scratch of toma_mlp_workspace_bytes() (the hidden tensor), 16-byte aligned;
+ * bf16 needs dim and hidden multiples of 8. */
+TOMA_API size_t toma_mlp_workspace_bytes(int32_t rows, int32_t dim, int32_t hidden, int32_t dtype);
+TOMA_API toma_status toma_mlp(int32_t rows, int32_t dim, int32_t hidden, int32_t dtype, const void* x, const void* w1,
+                              const void* w2, void* out, void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream);
+
 /* toma_block for callers whose tokens live in HOST memory (Algorithm 3 end to end, copies included):
  * copy x_host -> x_dev, run toma_block(x_dev -> out_dev), copy out_dev -> out_host.
  *   x_host, out_host: HOST buffers of batch*(N + n_extra)*dim elements, caller-owned.  Page-locked

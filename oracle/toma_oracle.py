@@ -15,6 +15,7 @@ configs are pinned only through those properties.
 """
 from __future__ import annotations
 
+import math
 from dataclasses import dataclass, field
 from typing import List, Optional, Tuple
 
@@ -242,6 +243,23 @@ def linear(a: np.ndarray, w: np.ndarray) -> np.ndarray:
     return np.asarray(a, dtype=np.float64) @ np.asarray(w, dtype=np.float64)
 
 
+_erf = np.vectorize(math.erf, otypes=[np.float64])
+
+
+def gelu(v: np.ndarray) -> np.ndarray:
+    """GELU(v) = v * Phi(v) with the exact standard normal distribution function
+    Phi(v) = (1 + erf(v / sqrt 2)) / 2: the activation of the wrapped MLP."""
+    v = np.asarray(v, dtype=np.float64)
+    return 0.5 * v * (1.0 + _erf(v / math.sqrt(2.0)))
+
+
+def mlp(x: np.ndarray, w1: np.ndarray, w2: np.ndarray, round_fn=None) -> np.ndarray:
+    """The MLP as the wrapped module F (Sec. 4.2.2, "Attention/MLP"): GELU(x w1) w2, no biases.
+    round_fn, if given, mirrors the storage rounding of the hidden tensor and of the result."""
+    rnd = (lambda t: t) if round_fn is None else round_fn
+    return rnd(linear(rnd(gelu(linear(x, w1))), w2))
+
+
 def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, n_heads: int,
               query_rows: Optional[np.ndarray] = None) -> np.ndarray:
     """Multi-head softmax(Q K^T / sqrt(dh)) V for one batch item.
@@ -290,7 +308,7 @@ class BlockState:
 def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid_w: int,
                tile_h: int, tile_w: int, merge_ratio: float, tau: float, n_heads: int,
                reuse_interval: int, n_extra: int = 0, round_fn=None, weight_reuse_interval: int = 0,
-               global_merge: bool = False, proj=None, unmerge_mode: str = "transpose"):
+               global_merge: bool = False, proj=None, unmerge_mode: str = "transpose", mlp_weights=None):
     """One ToMA-wrapped attention call (Algorithm 3) on x [B, N + n_extra, d].
 
     Selection and weights are recomputed when step % reuse_interval == 0 and
@@ -309,6 +327,9 @@ def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid
     With proj = (wq, wk, wv, wo), each [d, d] as [in, out], the wrapped module is the whole attention
     module: attention(X_m wq, X_m wk, X_m wv) wo (Algorithm 3 applies F to the merged tokens; App. C's
     4 d^2 N term).  round_fn is then also applied to q, k, v and to the projected output.
+
+    With mlp_weights = (w1 [d, f], w2 [f, d]) the wrapped module is the MLP GELU(X_m w1) w2 instead of
+    attention; round_fn is then applied to the hidden tensor and to the MLP's output.
 
     unmerge_mode "transpose" applies A~^T (Algorithm 3); "shares" applies A^T, the softmax matrix
     before row normalisation (columns sum to 1).
@@ -361,12 +382,14 @@ def block_step(x: np.ndarray, step: int, state: BlockState, *, grid_h: int, grid
     rnd = (lambda t: t) if round_fn is None else round_fn
     attended = np.empty_like(merged)
     for b in range(B):
-        if proj is None:
+        if mlp_weights is not None:
+            attended[b] = mlp(merged[b], mlp_weights[0], mlp_weights[1], round_fn)
+        elif proj is None:
             attended[b] = attention(merged[b], merged[b], merged[b], n_heads)
         else:
             q, k, v = (rnd(linear(merged[b], w)) for w in proj[:3])
             attended[b] = rnd(linear(rnd(attention(q, k, v, n_heads)), proj[3]))
-    if round_fn is not None and proj is None:
+    if round_fn is not None and proj is None and mlp_weights is None:
         attended = round_fn(attended)
     out = np.empty((B, n_all, d), dtype=np.float64)
     for b in range(B):

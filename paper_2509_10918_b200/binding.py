@@ -22,7 +22,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_RATIO", "ERR_TA
 EXPORTS = ["toma_select_static", "toma_launch_counter", "toma_workspace_bytes", "toma_weights_bytes", "toma_dest_per_tile", "toma_validate", "toma_status_str",
            "toma_select", "toma_merge_weights", "toma_merge", "toma_attention_workspace_bytes", "toma_attention_plan", "toma_attention",
            "toma_unmerge", "toma_block", "toma_block_host", "toma_linear", "toma_block_proj", "toma_attention_proj_workspace_bytes",
-           "toma_attention_proj",
+           "toma_attention_proj", "toma_block_mlp", "toma_mlp_workspace_bytes", "toma_mlp",
            "toma_weights_export", "toma_weights_import", "toma_unmerge_weights_export"]
 
 UNMERGE_MODES = {"transpose": 0, "shares": 1}
@@ -91,6 +91,12 @@ def _load() -> ctypes.CDLL:
     lib.toma_attention_proj_workspace_bytes.argtypes = [c_int32] * 5
     lib.toma_attention_proj.restype = c_int32
     lib.toma_attention_proj.argtypes = [c_int32] * 5 + [c_void_p] * 7 + [c_size_t, c_void_p, c_void_p]
+    lib.toma_block_mlp.restype = c_int32
+    lib.toma_block_mlp.argtypes = [P, c_int32, c_void_p, c_void_p, c_void_p, c_int32] + [c_void_p] * 4 + [c_size_t, c_void_p, c_void_p]
+    lib.toma_mlp_workspace_bytes.restype = c_size_t
+    lib.toma_mlp_workspace_bytes.argtypes = [c_int32] * 4
+    lib.toma_mlp.restype = c_int32
+    lib.toma_mlp.argtypes = [c_int32] * 4 + [c_void_p] * 5 + [c_size_t, c_void_p, c_void_p]
     lib.toma_linear.restype = c_int32
     lib.toma_linear.argtypes = [c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.toma_block_host.restype = c_int32
@@ -263,6 +269,23 @@ def toma_attention_proj(batch, length, n_heads, head_dim, dtype, x, wq, wk, wv, 
     _check(lib.toma_attention_proj(batch, length, n_heads, head_dim, _dtype_code(dtype), _ptr(x), _ptr(wq), _ptr(wk),
                                    _ptr(wv), _ptr(wo), _ptr(out), _ptr(ws), ws.numel() * ws.element_size(),
                                    _ptr(dev_status), _stream()), "toma_attention_proj")
+
+
+def toma_block_mlp(desc, step, x, w1, w2, out, idx_state, w_state, ws, dev_status=None):
+    """w1 [dim][hidden], w2 [hidden][dim]; hidden is read from w1's shape."""
+    hidden = int(w1.shape[1])
+    _check(lib.toma_block_mlp(ctypes.byref(desc), step, _ptr(x), _ptr(w1), _ptr(w2), hidden, _ptr(out), _ptr(idx_state),
+                              _ptr(w_state), _ptr(ws), ws.numel() * ws.element_size(), _ptr(dev_status), _stream()),
+           "toma_block_mlp")
+
+
+def toma_mlp_workspace_bytes(rows, dim, hidden, dtype) -> int:
+    return int(lib.toma_mlp_workspace_bytes(rows, dim, hidden, _dtype_code(dtype)))
+
+
+def toma_mlp(rows, dim, hidden, dtype, x, w1, w2, out, ws, dev_status=None):
+    _check(lib.toma_mlp(rows, dim, hidden, _dtype_code(dtype), _ptr(x), _ptr(w1), _ptr(w2), _ptr(out), _ptr(ws),
+                        ws.numel() * ws.element_size(), _ptr(dev_status), _stream()), "toma_mlp")
 
 
 def toma_block_host(desc, step, x_host, out_host, x_dev, out_dev, idx_state, w_state, ws, dev_status=None,

@@ -277,10 +277,10 @@ toma_status toma_attention(int32_t batch, int32_t len, int32_t n_heads, int32_t 
 
 // c[i] = a w[i] for n_mats weight / output pairs
 static cudaError_t do_linear(int M, int N, int K, bool f32, const void* a, const void* const* w, void* const* c, int n_mats,
-                             uint32_t* dev_status, cudaStream_t s) {
-  if (!f32 && linear_tc_shape_ok(M, N, K)) return launch_linear_tc(M, N, K, a, w, c, n_mats, dev_status, s);
+                             int act, uint32_t* dev_status, cudaStream_t s) {
+  if (!f32 && linear_tc_shape_ok(M, N, K)) return launch_linear_tc(M, N, K, a, w, c, n_mats, act, dev_status, s);
   for (int i = 0; i < n_mats; ++i) {
-    cudaError_t e = launch_linear_simt(M, N, K, f32, a, w[i], c[i], s);
+    cudaError_t e = launch_linear_simt(M, N, K, f32, a, w[i], c[i], act, s);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
@@ -295,15 +295,16 @@ toma_status toma_linear(int32_t m, int32_t n, int32_t k, int32_t dtype, const vo
   if (dtype == TOMA_BF16 && (n % 8 || k % 8)) return TOMA_ERR_SHAPE;  // 16-byte rows
   const void* ws[1] = {w};
   void* cs[1] = {c};
-  return cuda_ok(do_linear(m, n, k, dtype == TOMA_F32, a, ws, cs, 1, dev_status, (cudaStream_t)stream));
+  return cuda_ok(do_linear(m, n, k, dtype == TOMA_F32, a, ws, cs, 1, kActNone, dev_status, (cudaStream_t)stream));
 }
 
 // The wrapped module F: attention over the merged tokens with Q = K = V = X_m, or, with projection weights
 // (proj = {wq, wk, wv, wo}, each [dim][dim], row-major [in][out]), the whole attention module
-// (X_m wq, X_m wk, X_m wv -> attention -> wo).
-static toma_status block_impl(const toma_desc* desc, int32_t step, const void* x, const void* const* proj, void* out,
-                              int32_t* idx_state, void* w_state, void* ws, size_t ws_bytes, uint32_t* dev_status,
-                              void* stream) {
+// (X_m wq, X_m wk, X_m wv -> attention -> wo); or, with mlp = {w1 [dim][hidden], w2 [hidden][dim]}, the MLP
+// GELU(X_m w1) w2.
+static toma_status block_impl(const toma_desc* desc, int32_t step, const void* x, const void* const* proj,
+                              const void* const* mlp, int hidden, void* out, int32_t* idx_state, void* w_state, void* ws,
+                              size_t ws_bytes, uint32_t* dev_status, void* stream) {
   Geom g;
   toma_status st = make_geom(desc, &g);
   if (st != TOMA_OK) return st;
@@ -313,6 +314,12 @@ static toma_status block_impl(const toma_desc* desc, int32_t step, const void* x
       if (!proj[i]) return TOMA_ERR_NULL;
       if (misaligned(proj[i])) return TOMA_ERR_SHAPE;
     }
+  if (mlp) {
+    if (!mlp[0] || !mlp[1]) return TOMA_ERR_NULL;
+    if (misaligned(mlp[0]) || misaligned(mlp[1])) return TOMA_ERR_SHAPE;
+    // the hidden tensor lives in the four merged-size slots of the projection scratch
+    if (hidden < 8 || hidden % 8 || hidden > 4 * g.d) return TOMA_ERR_SHAPE;
+  }
   if (step < 0) return TOMA_ERR_SHAPE;
   if (misaligned(x) || misaligned(out) || misaligned(w_state)) return TOMA_ERR_SHAPE;
   if (!attention_supported_simt(g.dh)) return TOMA_ERR_UNSUPPORTED;
@@ -332,6 +339,15 @@ static toma_status block_impl(const toma_desc* desc, int32_t step, const void* x
   bool tickets_clean = false;
   const size_t ticket_bytes = attention_on_tc(g.dh, g.f32) ? attention_tc_ticket_bytes(g.B, g.Lm, g.heads) : 0;
   if (e == cudaSuccess) e = do_merge(g, w_state, x, xm, wsb + l.att_ws_off, ticket_bytes, &tickets_clean, dev_status, s);
+  if (mlp) {
+    const int rows = g.B * g.Lm;
+    void* hid[1] = {wsb + l.proj_off};
+    void* ys[1] = {att};
+    if (e == cudaSuccess) e = do_linear(rows, hidden, g.d, g.f32, xm, mlp, hid, 1, kActGelu, dev_status, s);
+    if (e == cudaSuccess) e = do_linear(rows, g.d, hidden, g.f32, hid[0], mlp + 1, ys, 1, kActNone, dev_status, s);
+    if (e == cudaSuccess) e = do_unmerge(g, w_state, att, out, dev_status, s);
+    return cuda_ok(e);
+  }
   if (!proj) {
     if (e == cudaSuccess) e = do_attention(g.B, g.Lm, g.heads, g.dh, g.f32, xm, xm, xm, att, wsb + l.att_ws_off, tickets_clean, dev_status, s);
     if (e == cudaSuccess) e = do_unmerge(g, w_state, att, out, dev_status, s);
@@ -341,24 +357,55 @@ static toma_status block_impl(const toma_desc* desc, int32_t step, const void* x
   void* qkv[3] = {wsb + l.proj_off, wsb + l.proj_off + one, wsb + l.proj_off + 2 * one};
   void* y = wsb + l.proj_off + 3 * one;
   const int rows = g.B * g.Lm;
-  if (e == cudaSuccess) e = do_linear(rows, g.d, g.d, g.f32, xm, proj, qkv, 3, dev_status, s);
+  if (e == cudaSuccess) e = do_linear(rows, g.d, g.d, g.f32, xm, proj, qkv, 3, kActNone, dev_status, s);
   if (e == cudaSuccess) e = do_attention(g.B, g.Lm, g.heads, g.dh, g.f32, qkv[0], qkv[1], qkv[2], att, wsb + l.att_ws_off, tickets_clean, dev_status, s);
   void* ys[1] = {y};
-  if (e == cudaSuccess) e = do_linear(rows, g.d, g.d, g.f32, att, proj + 3, ys, 1, dev_status, s);
+  if (e == cudaSuccess) e = do_linear(rows, g.d, g.d, g.f32, att, proj + 3, ys, 1, kActNone, dev_status, s);
   if (e == cudaSuccess) e = do_unmerge(g, w_state, y, out, dev_status, s);
   return cuda_ok(e);
 }
 
 toma_status toma_block(const toma_desc* desc, int32_t step, const void* x, void* out, int32_t* idx_state,
                        void* w_state, void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream) {
-  return block_impl(desc, step, x, nullptr, out, idx_state, w_state, ws, ws_bytes, dev_status, stream);
+  return block_impl(desc, step, x, nullptr, nullptr, 0, out, idx_state, w_state, ws, ws_bytes, dev_status, stream);
+}
+
+toma_status toma_block_mlp(const toma_desc* desc, int32_t step, const void* x, const void* w1, const void* w2,
+                           int32_t hidden, void* out, int32_t* idx_state, void* w_state, void* ws, size_t ws_bytes,
+                           uint32_t* dev_status, void* stream) {
+  const void* mlp[2] = {w1, w2};
+  return block_impl(desc, step, x, nullptr, mlp, hidden, out, idx_state, w_state, ws, ws_bytes, dev_status, stream);
+}
+
+size_t toma_mlp_workspace_bytes(int32_t rows, int32_t dim, int32_t hidden, int32_t dtype) {
+  if ((dtype != TOMA_BF16 && dtype != TOMA_F32) || rows < 1 || dim < 1 || hidden < 1) return 0;
+  return align_up((size_t)rows * hidden * (dtype == TOMA_F32 ? 4 : 2), 256);
+}
+
+toma_status toma_mlp(int32_t rows, int32_t dim, int32_t hidden, int32_t dtype, const void* x, const void* w1, const void* w2,
+                     void* out, void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream) {
+  if (dtype != TOMA_BF16 && dtype != TOMA_F32) return TOMA_ERR_DTYPE;
+  if (rows < 1 || dim < 1 || hidden < 1) return TOMA_ERR_SHAPE;
+  if (!x || !w1 || !w2 || !out) return TOMA_ERR_NULL;
+  if (misaligned(x) || misaligned(w1) || misaligned(w2) || misaligned(out)) return TOMA_ERR_SHAPE;
+  if (dtype == TOMA_BF16 && (dim % 8 || hidden % 8)) return TOMA_ERR_SHAPE;  // 16-byte rows
+  if (!ws || misaligned(ws) || ws_bytes < toma_mlp_workspace_bytes(rows, dim, hidden, dtype)) return TOMA_ERR_WORKSPACE;
+  const bool f32 = dtype == TOMA_F32;
+  cudaStream_t s = (cudaStream_t)stream;
+  const void* w1s[1] = {w1};
+  const void* w2s[1] = {w2};
+  void* hid[1] = {ws};
+  void* outs[1] = {out};
+  cudaError_t e = do_linear(rows, hidden, dim, f32, x, w1s, hid, 1, kActGelu, dev_status, s);
+  if (e == cudaSuccess) e = do_linear(rows, dim, hidden, f32, ws, w2s, outs, 1, kActNone, dev_status, s);
+  return cuda_ok(e);
 }
 
 toma_status toma_block_proj(const toma_desc* desc, int32_t step, const void* x, const void* wq, const void* wk,
                             const void* wv, const void* wo, void* out, int32_t* idx_state, void* w_state, void* ws,
                             size_t ws_bytes, uint32_t* dev_status, void* stream) {
   const void* proj[4] = {wq, wk, wv, wo};
-  return block_impl(desc, step, x, proj, out, idx_state, w_state, ws, ws_bytes, dev_status, stream);
+  return block_impl(desc, step, x, proj, nullptr, 0, out, idx_state, w_state, ws, ws_bytes, dev_status, stream);
 }
 
 size_t toma_attention_proj_workspace_bytes(int32_t batch, int32_t len, int32_t n_heads, int32_t head_dim, int32_t dtype) {
@@ -387,10 +434,10 @@ toma_status toma_attention_proj(int32_t batch, int32_t len, int32_t n_heads, int
   void* att_ws = wsb + 4 * one;
   const void* proj[4] = {wq, wk, wv, wo};
   const int rows = batch * len;
-  cudaError_t e = do_linear(rows, d, d, f32, x, proj, qkv, 3, dev_status, s);
+  cudaError_t e = do_linear(rows, d, d, f32, x, proj, qkv, 3, kActNone, dev_status, s);
   if (e == cudaSuccess) e = do_attention(batch, len, n_heads, head_dim, f32, qkv[0], qkv[1], qkv[2], att, att_ws, false, dev_status, s);
   void* outs[1] = {out};
-  if (e == cudaSuccess) e = do_linear(rows, d, d, f32, att, proj + 3, outs, 1, dev_status, s);
+  if (e == cudaSuccess) e = do_linear(rows, d, d, f32, att, proj + 3, outs, 1, kActNone, dev_status, s);
   return cuda_ok(e);
 }
 

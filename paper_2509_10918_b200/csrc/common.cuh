@@ -83,10 +83,12 @@ cudaError_t launch_attention_tc(int B, int L, int heads, int dh, const void* q, 
 cudaError_t launch_global_idx(const Geom& g, const int32_t* idx, int32_t* gidx, cudaStream_t s);
 // Projection c = a w (a [M][K], w [K][N], c [M][N], row-major): tensor-core form for bf16 (up to three
 // weight / output pairs sharing a), FFMA form otherwise.
+// `act`: kActNone, or kActGelu to apply the exact (erf) GELU to the fp32 result before it is stored.
+constexpr int kActNone = 0, kActGelu = 1;
 bool linear_tc_shape_ok(int M, int N, int K);
-cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* const* w, void* const* c, int n_mats,
+cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* const* w, void* const* c, int n_mats, int act,
                              uint32_t* dev_status, cudaStream_t s);
-cudaError_t launch_linear_simt(int M, int N, int K, bool f32, const void* a, const void* w, void* c, cudaStream_t s);
+cudaError_t launch_linear_simt(int M, int N, int K, bool f32, const void* a, const void* w, void* c, int act, cudaStream_t s);
 cudaError_t launch_weights_export(const Geom& g, const void* w, float* dense, cudaStream_t s);
 cudaError_t launch_weights_import(const Geom& g, const float* dense, void* w, cudaStream_t s);
 
@@ -97,6 +99,9 @@ __device__ __forceinline__ float to_f32(__half v) { return __half2float(v); }
 __device__ __forceinline__ void from_f32(float& o, float v) { o = v; }
 __device__ __forceinline__ void from_f32(__nv_bfloat16& o, float v) { o = __float2bfloat16_rn(v); }
 __device__ __forceinline__ void from_f32(__half& o, float v) { o = __float2half_rn(v); }
+
+// GELU(v) = v * Phi(v), Phi the standard normal distribution function.
+__device__ __forceinline__ float gelu(float v) { return 0.5f * v * (1.f + erff(v * 0.70710678118654752f)); }
 
 // Global row of image token (tile p, local slot l) inside one batch item.
 __device__ __forceinline__ int tile_token(int p, int l, int tiles_x, int th, int tw, int W) {

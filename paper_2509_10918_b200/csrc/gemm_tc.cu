@@ -7,7 +7,8 @@
 // W the MN-major one exactly as stored ([k][n] row-major), so neither is transposed or copied.
 // blockIdx.z selects one of up to three weight / output pairs that share A (Q, K and V in one
 // launch).  Warp 0 feeds a TMA ring, warp 1 issues the MMAs, warps 2..5 write each token row's
-// columns as one contiguous run.
+// columns as one contiguous run, after the activation when one is asked for (the first layer of the
+// MLP, the other module ToMA wraps).
 #include "common.cuh"
 #include "tc.cuh"
 
@@ -38,7 +39,7 @@ template <int kCols>
 __global__ void __launch_bounds__(192, 1)
 linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w0,
                    const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2, GemmOut out, int M,
-                   int N, int K, int stages, uint32_t* dev_status) {
+                   int N, int K, int stages, int act, uint32_t* dev_status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -115,6 +116,10 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
         uint32_t r[32];
         tmem_ld32(taddr + j, r);
         tmem_wait_ld();
+        if (act == kActGelu) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(gelu(__uint_as_float(r[e])));
+        }
         if (row < M) {
 #pragma unroll
           for (int e = 0; e < 32; e += 8) {
@@ -143,7 +148,7 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
 bool linear_tc_shape_ok(int M, int N, int K) { return M >= 1 && N >= 8 && K >= 8 && N % 8 == 0 && K % 8 == 0; }
 
 // c[i] = a * w[i] for i < n_mats (1..3); a [M][K], w[i] [K][N], c[i] [M][N], all bf16 row-major.
-cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* const* w, void* const* c, int n_mats,
+cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* const* w, void* const* c, int n_mats, int act,
                              uint32_t* dev_status, cudaStream_t s) {
   CUtensorMap ta, tw[3];
   const uint64_t adims[2] = {(uint64_t)K, (uint64_t)M};
@@ -183,9 +188,9 @@ cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* con
   }
   dim3 grid(mb, (N + cols - 1) / cols, n_mats);
   cudaError_t e = narrow ? launch_dependent(linear_rows_kernel<256>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out,
-                                            M, N, K, stages, dev_status)
+                                            M, N, K, stages, act, dev_status)
                          : launch_dependent(linear_rows_kernel<320>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out,
-                                            M, N, K, stages, dev_status);
+                                            M, N, K, stages, act, dev_status);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }

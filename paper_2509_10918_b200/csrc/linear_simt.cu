@@ -278,18 +278,22 @@ struct LinearOp {
   const T* a_;
   const T* w_;
   T* c_;
+  int act;
   __device__ __forceinline__ float a(int, int m, int k) const { return to_f32(a_[(size_t)m * K + k]); }
   __device__ __forceinline__ float b(int, int k, int n) const { return to_f32(w_[(size_t)k * N + n]); }
   template <typename AccT>
-  __device__ __forceinline__ void store(int, int m, int n, AccT v) const { from_f32(c_[(size_t)m * N + n], (float)v); }
+  __device__ __forceinline__ void store(int, int m, int n, AccT v) const {
+    const float f = (float)v;
+    from_f32(c_[(size_t)m * N + n], act == kActGelu ? gelu(f) : f);
+  }
 };
 
-cudaError_t launch_linear_simt(int M, int N, int K, bool f32, const void* a, const void* w, void* c, cudaStream_t s) {
+cudaError_t launch_linear_simt(int M, int N, int K, bool f32, const void* a, const void* w, void* c, int act, cudaStream_t s) {
   if (f32) {
-    LinearOp<float> op{M, N, K, (const float*)a, (const float*)w, (float*)c};
+    LinearOp<float> op{M, N, K, (const float*)a, (const float*)w, (float*)c, act};
     run_gemm<LinearOp<float>, float>(op, 1, s);
   } else {
-    LinearOp<__nv_bfloat16> op{M, N, K, (const __nv_bfloat16*)a, (const __nv_bfloat16*)w, (__nv_bfloat16*)c};
+    LinearOp<__nv_bfloat16> op{M, N, K, (const __nv_bfloat16*)a, (const __nv_bfloat16*)w, (__nv_bfloat16*)c, act};
     run_gemm<LinearOp<__nv_bfloat16>, float>(op, 1, s);
   }
   return cudaGetLastError();

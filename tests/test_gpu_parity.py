@@ -533,6 +533,67 @@ def test_attention_module_with_projections_parity(toma, dtype, B, L, h, dh):
         assert_close(got[b], want, dtype, f"attention module b={b}")
 
 
+def _mlp_weights(cfg, hidden, seed=97):
+    """w1 [d, f] ~ N(0, 1/d) and w2 [f, d] ~ N(0, 1/f), rounded to the storage dtype."""
+    d = cfg.dim
+    w1 = gen.normal(0, (seed, 1, d, hidden), d * hidden).reshape(d, hidden) / np.sqrt(d)
+    w2 = gen.normal(0, (seed, 2, d, hidden), d * hidden).reshape(hidden, d) / np.sqrt(hidden)
+    return [gen.round_to_dtype(w.astype(np.float32), cfg.dtype) for w in (w1, w2)]
+
+
+@pytest.mark.parametrize("dtype,rows,d,f", [("bf16", 2048, 640, 2560), ("bf16", 300, 128, 512), ("bf16", 1000, 64, 40),
+                                            ("f32", 130, 64, 96)])
+def test_mlp_parity(toma, dtype, rows, d, f):
+    """toma_mlp (the full-token baseline of toma_block_mlp): GELU(x w1) w2 against the oracle, which rounds the
+    hidden tensor to the storage dtype as the kernels do."""
+    cfg = gen.config("cfg2", batch=1, dim=d, n_heads=1, head_dim=d, dtype=dtype)
+    x_host = gen.round_to_dtype(gen.normal(0, (98, rows, d), rows * d).reshape(rows, d).astype(np.float32), dtype)
+    w_host = _mlp_weights(cfg, f)
+    x, w1, w2 = to_dev(x_host, dtype), to_dev(w_host[0], dtype), to_dev(w_host[1], dtype)
+    out = torch.empty_like(x)
+    ws = torch.empty(toma.toma_mlp_workspace_bytes(rows, d, f, dtype), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    toma.toma_mlp(rows, d, f, dtype, x, w1, w2, out, ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    pick = np.unique(np.concatenate([[0, rows - 1], np.random.default_rng(rows).choice(rows, size=min(rows, 160), replace=False)]))
+    want = O.mlp(x_host[pick], w_host[0], w_host[1], _storage_rounding(dtype))
+    assert_close(to_host64(out)[pick], want, dtype, "mlp")
+    # the hidden tensor itself: GELU of the first projection, in storage dtype
+    hid = ws[: rows * f * (4 if dtype == "f32" else 2)].view(torch.float32 if dtype == "f32" else torch.bfloat16).reshape(rows, f)
+    assert_close(to_host64(hid)[pick], O.gelu(O.linear(x_host[pick], w_host[0])), dtype, "mlp hidden")
+
+
+@pytest.mark.parametrize("name,over,hidden", [("cfg2", dict(batch=1), 5120), ("cfg3", dict(batch=1), 2560), ("cfg1", {}, 320),
+                                              ("cfg2", dict(batch=1, grid_h=16, grid_w=16, n_extra=9), 1288)],
+                         ids=["cfg2", "cfg3", "cfg1-f32", "extra-tokens"])
+def test_block_with_mlp_parity(toma, name, over, hidden):
+    """toma_block_mlp: the wrapped module is the MLP on the merged tokens; a refresh step and a reuse step."""
+    cfg = gen.config(name, steps=2, reuse_interval=2, **over)
+    desc = toma.desc_from_config(cfg)
+    w_host = _mlp_weights(cfg, hidden)
+    w1, w2 = (to_dev(w, cfg.dtype) for w in w_host)
+    idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    st = O.BlockState()
+    kw = dict(grid_h=cfg.grid_h, grid_w=cfg.grid_w, tile_h=cfg.tile_h, tile_w=cfg.tile_w, merge_ratio=cfg.merge_ratio,
+              tau=cfg.tau, n_heads=cfg.n_heads, reuse_interval=2, n_extra=cfg.n_extra,
+              mlp_weights=[x.astype(np.float64) for x in w_host], round_fn=_storage_rounding(cfg.dtype))
+    for step, x_host in enumerate(gen.feature_sequence(cfg)):
+        x = to_dev(x_host, cfg.dtype)
+        out = torch.empty_like(x)
+        toma.toma_block_mlp(desc, step, x, w1, w2, out, idx, w, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        want, _, _ = O.block_step(x_host, step, st, **kw)
+        assert np.array_equal(idx.cpu().numpy().astype(np.int64), st.idx)
+        assert_close(to_host64(out), want, cfg.dtype, f"block with MLP, step {step}")
+    # a hidden width beyond four times the model width does not fit the block's workspace
+    wide = torch.zeros((cfg.dim, 4 * cfg.dim + 8), dtype=x.dtype, device="cuda")
+    with pytest.raises(toma.TomaError):
+        toma.toma_block_mlp(desc, 0, x, wide, w2, out, idx, w, ws, status)
+
+
 def test_block_replays_from_a_cuda_graph(toma):
     """A reuse step and a refresh step captured into CUDA graphs (the calls never allocate or synchronise,
     and their dependent launches are capturable) replay to the same bits as direct calls."""

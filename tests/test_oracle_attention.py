@@ -1,6 +1,7 @@
 """Pins for the attention oracle (Eq. 1 with tau = 1): textbook special cases and a
 library second opinion."""
 import numpy as np
+import pytest
 import torch
 
 from oracle import toma_oracle as O
@@ -59,3 +60,38 @@ def test_linear_matches_explicit_loops():
                 want[i, j] += a[i, k] * w[k, j]
     assert np.allclose(O.linear(a, w), want, rtol=0, atol=1e-13)
     assert np.array_equal(O.linear(a, np.eye(7)), a)
+
+
+def test_gelu_closed_forms_and_library_second_opinion():
+    import math
+    import torch
+    # Phi(1) = 0.8413447460685429 (standard normal table), Phi(0) = 1/2
+    assert O.gelu(np.array([0.0]))[0] == 0.0
+    assert O.gelu(np.array([1.0]))[0] == pytest.approx(0.8413447460685429, abs=1e-15)
+    assert O.gelu(np.array([-1.0]))[0] == pytest.approx(-0.15865525393145707, abs=1e-15)
+    v = np.linspace(-6, 6, 241)
+    g = O.gelu(v)
+    assert np.allclose(g - O.gelu(-v), v, atol=1e-14)            # Phi(v) + Phi(-v) = 1
+    assert np.allclose(g[v > 5.5], v[v > 5.5], atol=1e-7) and np.all(np.abs(g[v < -5.5]) < 1e-7)
+    assert g.min() == pytest.approx(-0.16997, abs=1e-4)           # the dip near v = -0.7518
+    want = torch.nn.functional.gelu(torch.from_numpy(v), approximate="none").numpy()
+    assert np.allclose(g, want, atol=1e-14)
+    # not the tanh approximation: the two differ by up to 5e-4
+    tanh_form = 0.5 * v * (1 + np.tanh(math.sqrt(2 / math.pi) * (v + 0.044715 * v ** 3)))
+    assert np.abs(g - tanh_form).max() > 1e-4
+
+
+def test_mlp_is_two_projections_around_gelu():
+    rng = np.random.default_rng(9)
+    x, w1, w2 = rng.normal(size=(6, 8)), rng.normal(size=(8, 12)) / 3, rng.normal(size=(12, 8)) / 3
+    h = np.zeros((6, 12))
+    for i in range(6):
+        for j in range(12):
+            h[i, j] = sum(x[i, k] * w1[k, j] for k in range(8))
+    want = O.gelu(h) @ w2
+    assert np.allclose(O.mlp(x, w1, w2), want, atol=1e-13)
+    # rounding hook: applied to the hidden tensor and to the result
+    r = lambda t: np.round(t * 16) / 16
+    assert np.array_equal(O.mlp(x, w1, w2, r), r(r(O.gelu(h)) @ w2))
+    # a zero first layer gives GELU(0) = 0 everywhere
+    assert np.array_equal(O.mlp(x, np.zeros_like(w1), w2), np.zeros((6, 8)))
