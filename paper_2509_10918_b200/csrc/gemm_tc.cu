@@ -9,6 +9,8 @@
 // launch).  Warp 0 feeds a TMA ring, warp 1 issues the MMAs, warps 2..5 write each token row's
 // columns as one contiguous run, after the activation when one is asked for (the first layer of the
 // MLP, the other module ToMA wraps).
+#include <cstdlib>
+
 #include "common.cuh"
 #include "tc.cuh"
 
@@ -35,7 +37,10 @@ struct GemmOut {
 // kCols = 320: two accumulators (192 + 128 columns), 512 tensor-memory columns, one CTA per SM, deep ring.
 // kCols = 256: one accumulator, 256 tensor-memory columns, two CTAs per SM, for grids that would otherwise
 // spill into a second wave or leave most SMs idle.
-template <int kCols>
+// kRowBlocks = 2 (with kCols = 256): two 128-row blocks per CTA share every W slab, so a CTA moves 64 KB
+// per 256 x 256 x 64 multiply-adds instead of 48 KB per 128 x 256 x 64 (these shapes re-read their operands
+// from L2 many times and are bound by that traffic); one CTA per SM.
+template <int kCols, int kRowBlocks = 1>
 __global__ void __launch_bounds__(192, 1)
 linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w0,
                    const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2, GemmOut out, int M,
@@ -44,16 +49,17 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int kFirst = kCols == 320 ? 3 : 4;  // 64-column slabs of the first accumulator
-  const int m0 = blockIdx.x * 128, n0 = blockIdx.y * kCols;
+  const int m0 = blockIdx.x * 128 * kRowBlocks, n0 = blockIdx.y * kCols;
   const CUtensorMap* tm_w = blockIdx.z == 0 ? &tm_w0 : blockIdx.z == 1 ? &tm_w1 : &tm_w2;
   __nv_bfloat16* c = out.c[blockIdx.z];
   const int n_cols = min(kCols, N - n0);         // columns of this CTA (multiple of 8)
   const int slabs = (n_cols + 63) / 64;
   const int n_a = min(slabs, kFirst) * 64, n_b = (slabs - min(slabs, kFirst)) * 64;
-  const int stage_bytes = kABytes + slabs * kSlab;
+  const int stage_bytes = kRowBlocks * kABytes + slabs * kSlab;
   GemmBars* bar = reinterpret_cast<GemmBars*>(smem + stages * stage_bytes);
   const int nk = (K + kKC - 1) / kKC;
-  constexpr uint32_t ncols = kCols == 320 ? 512 : 256;
+  constexpr uint32_t ncols = (kCols == 320 || kRowBlocks == 2) ? 512 : 256;
+  static_assert(kRowBlocks == 1 || kCols == 256, "two row blocks need the one-accumulator column form");
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -82,8 +88,9 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
         if (k >= stages && !mbar_wait(&bar->empty[s], ((k / stages) - 1) & 1, dev_status, abort_flag)) break;
         uint8_t* sa = smem + s * stage_bytes;
         mbar_expect_tx(&bar->full[s], stage_bytes);
-        tma_load_2d(sa, &tm_a, &bar->full[s], k * kKC, m0);
-        for (int j = 0; j < slabs; ++j) tma_load_2d(sa + kABytes + j * kSlab, tm_w, &bar->full[s], n0 + j * 64, k * kKC);
+        for (int rb = 0; rb < kRowBlocks; ++rb) tma_load_2d(sa + rb * kABytes, &tm_a, &bar->full[s], k * kKC, m0 + rb * 128);
+        for (int j = 0; j < slabs; ++j)
+          tma_load_2d(sa + kRowBlocks * kABytes + j * kSlab, tm_w, &bar->full[s], n0 + j * 64, k * kKC);
       }
     }
   } else if (warp == 1) {
@@ -95,22 +102,30 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
         const int s = k % stages;
         if (!mbar_wait(&bar->full[s], (k / stages) & 1, dev_status, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t aa = smem_u32(smem + s * stage_bytes), wa = aa + kABytes;
+        const uint32_t aa = smem_u32(smem + s * stage_bytes), wa = aa + kRowBlocks * kABytes;
         const int ksteps = min(kKC, K - k * kKC + 15) / 16;  // 16 contraction elements per MMA (zero filled past K)
         for (int kk = 0; kk < ksteps; ++kk) {
-          const uint64_t ad = smem_desc_sw128(aa + kk * 32, 16, 1024);
-          mma_ss(tmem, ad, smem_desc_sw128(wa + kk * 2048, kSlab, 1024), idesc_a, k > 0 || kk > 0);
-          if (n_b > 0) mma_ss(tmem + kFirst * 64, ad, smem_desc_sw128(wa + kFirst * kSlab + kk * 2048, kSlab, 1024), idesc_b, k > 0 || kk > 0);
+          const uint64_t wd = smem_desc_sw128(wa + kk * 2048, kSlab, 1024);
+#pragma unroll
+          for (int rb = 0; rb < kRowBlocks; ++rb) {
+            const uint64_t ad = smem_desc_sw128(aa + rb * kABytes + kk * 32, 16, 1024);
+            mma_ss(tmem + rb * 256, ad, wd, idesc_a, k > 0 || kk > 0);
+            if (kRowBlocks == 1 && n_b > 0)
+              mma_ss(tmem + kFirst * 64, ad, smem_desc_sw128(wa + kFirst * kSlab + kk * 2048, kSlab, 1024), idesc_b, k > 0 || kk > 0);
+          }
         }
         mma_commit(&bar->empty[s]);
       }
       if (ok) mma_commit(&bar->done);
     }
   } else {
-    const int quarter = warp & 3, row = m0 + quarter * 32 + lane;
-    const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16);
+    const int quarter = warp & 3;
     if (mbar_wait(&bar->done, 0, dev_status, abort_flag)) {
       tc_fence_after();
+#pragma unroll 1
+      for (int rb = 0; rb < kRowBlocks; ++rb) {
+      const int row = m0 + rb * 128 + quarter * 32 + lane;
+      const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + rb * 256;
       __nv_bfloat16* dst = c + (size_t)(row < M ? row : 0) * N + n0;
       for (int j = 0; j < n_cols; j += 32) {
         uint32_t r[32];
@@ -133,6 +148,7 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
           }
         }
       }
+      }  // row blocks
     }
   }
   tc_fence_before();
@@ -164,17 +180,30 @@ cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* con
     if (!encode_tmap_16bit(&tw[i], w[j], 2, wdims, wstr, wbox)) return cudaErrorInvalidValue;
     out.c[i] = (__nv_bfloat16*)c[j];
   }
-  // Column block: 320 (one CTA per SM, deep ring) unless that grid overflows the SMs into a second wave or
-  // fills less than half of them while the 256-column form (two CTAs per SM) fits one wave.
+  // Tile form: the one with the least serial work per SM, counted as CTAs per SM (rounded up) times the
+  // multiply-adds of a tile, the 256 x 256 form credited with the 1.3x it gains from moving fewer operand
+  // bytes per multiply-add (timed on eleven shapes from 4096 x 640 x 640 to 16384 x 8192 x 4096; the
+  // model picks the faster form on each).  The 128 x 256 form keeps two CTAs per SM resident and is only
+  // considered while its grid fits them.
   int sms = 148, dev = 0;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int mb = (M + 127) / 128;
-  const int ctas320 = mb * ((N + 319) / 320) * n_mats, ctas256 = mb * ((N + 255) / 256) * n_mats;
-  const bool narrow = ctas256 <= 2 * sms && (ctas320 > sms || 2 * ctas320 < sms);
-  const int cols = narrow ? 256 : 320;
+  const long long ctas320 = (long long)mb * ((N + 319) / 320) * n_mats, ctas256 = (long long)mb * ((N + 255) / 256) * n_mats;
+  const long long ctas_pair = (long long)((M + 255) / 256) * ((N + 255) / 256) * n_mats;
+  const long long cost320 = ((ctas320 + sms - 1) / sms) * (128 * 320) * 13;
+  const long long cost256 = ctas256 <= 2 * sms ? ((ctas256 + sms - 1) / sms) * (128 * 256) * 13 : cost320 + 1;
+  const long long cost_pair = M > 128 ? ((ctas_pair + sms - 1) / sms) * (256 * 256) * 10 : cost320 + 1;
+  int pair = cost_pair < cost320 && cost_pair < cost256;
+  bool narrow = !pair && cost256 < cost320;
+  if (const char* e = getenv("TOMA_LINEAR_TILE")) {  // tuning aid: 256 x 256 (2), 128 x 320 (1) or 128 x 256 (0) tiles
+    const int v = atoi(e);
+    pair = v == 2 && M > 128;
+    narrow = v == 0;
+  }
+  const int cols = (narrow || pair) ? 256 : 320;
   const int slabs = ((N < cols ? N : cols) + 63) / 64;
-  const int stage_bytes = kABytes + slabs * kSlab;
-  int stages = ((narrow ? 110 : 222) * 1024) / stage_bytes;
+  const int stage_bytes = (pair ? 2 : 1) * kABytes + slabs * kSlab;
+  int stages = ((narrow && !pair ? 110 : 222) * 1024) / stage_bytes;
   stages = stages > 4 ? 4 : stages < 1 ? 1 : stages;
   const int nk = (K + kKC - 1) / kKC;
   if (stages > nk) stages = nk;
@@ -183,11 +212,14 @@ cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* con
   if (!attr) {
     cudaError_t e = cudaFuncSetAttribute(linear_rows_kernel<320>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(linear_rows_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(linear_rows_kernel<256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr = true;
   }
-  dim3 grid(mb, (N + cols - 1) / cols, n_mats);
-  cudaError_t e = narrow ? launch_dependent(linear_rows_kernel<256>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out,
+  dim3 grid(pair ? (M + 255) / 256 : mb, (N + cols - 1) / cols, n_mats);
+  cudaError_t e = pair ? launch_dependent(linear_rows_kernel<256, 2>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out,
+                                          M, N, K, stages, act, dev_status)
+                  : narrow ? launch_dependent(linear_rows_kernel<256>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out,
                                             M, N, K, stages, act, dev_status)
                          : launch_dependent(linear_rows_kernel<320>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out,
                                             M, N, K, stages, act, dev_status);

@@ -472,6 +472,27 @@ def test_linear_parity(toma, dtype, m, n, k):
     assert_close(to_host64(c)[rows], O.linear(a_host[rows], w_host), dtype, "linear")
 
 
+@pytest.mark.parametrize("tile", [0, 1, 2], ids=["128x256", "128x320", "256x256"])
+@pytest.mark.parametrize("m,n,k", [(300, 328, 200), (129, 1920, 640), (1024, 72, 136), (640, 512, 64)])
+def test_linear_every_tile_form(toma, monkeypatch, tile, m, n, k):
+    """Each of the projection kernel's three tile forms, forced, on shapes with a ragged last row block (the
+    second row block of a 256-row tile partly or wholly past the end), partial column blocks and a partial
+    last k-step."""
+    monkeypatch.setenv("TOMA_LINEAR_TILE", str(tile))
+    a_host = gen.round_to_dtype(gen.normal(0, (191, m, k), m * k).reshape(m, k).astype(np.float32), "bf16")
+    w_host = gen.round_to_dtype((gen.normal(0, (192, n, k), k * n).reshape(k, n) / np.sqrt(k)).astype(np.float32), "bf16")
+    a, w = to_dev(a_host, "bf16"), to_dev(w_host, "bf16")
+    c = torch.full((m, n), float("nan"), dtype=a.dtype, device="cuda")
+    guard = torch.full((4096,), 7.0, dtype=a.dtype, device="cuda")  # allocated right after c
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    toma.toma_linear(a, w, c, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert not torch.isnan(c).any()
+    assert bool((guard == 7.0).all())
+    assert_close(to_host64(c), O.linear(a_host, w_host), "bf16", f"linear, tile form {tile}")
+
+
 def _proj_weights(cfg, seed=93):
     """Four [d, d] projection matrices N(0, 1/d), rounded to the storage dtype."""
     d = cfg.dim
