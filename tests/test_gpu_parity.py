@@ -715,6 +715,8 @@ EDGE = [
     dict(grid_h=16, grid_w=16, tile_h=16, tile_w=8, dim=72, n_heads=1, head_dim=72, merge_ratio=0.3),  # odd dim, ragged D_loc
     dict(grid_h=8, grid_w=8, tile_h=8, tile_w=8, dim=64, n_heads=1, merge_ratio=0.0),        # keep everything
     dict(grid_h=16, grid_w=16, tile_h=8, tile_w=8, dim=64, n_heads=1, merge_ratio=0.5, n_extra=7),
+    dict(grid_h=16, grid_w=16, tile_h=8, tile_w=8, dim=4096, n_heads=32, head_dim=128, merge_ratio=0.5),  # widest supported token
+    dict(grid_h=16, grid_w=16, tile_h=8, tile_w=8, dim=16, n_heads=1, head_dim=16, merge_ratio=0.5),     # narrow token
 ]
 
 
