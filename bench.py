@@ -102,20 +102,22 @@ def blas_threads():
 
 
 def cpu_baseline(cfg):
-    """The oracle as it stands, timed on this machine's host cores on batch item 0: one refresh
-    step and one reuse step, combined with the schedule's 2:8 mix."""
+    """The oracle as it stands, timed on this machine's host cores over the workload's whole step schedule
+    (two refresh and eight reuse steps of the full batch: about ten seconds of CPU work)."""
     import gen
     from oracle import toma_oracle as O
-    seq = list(gen.feature_sequence(cfg, 2))
+    seq = list(gen.feature_sequence(cfg, cfg.steps))
     st = O.BlockState()
-    t_refresh = oracle_step_seconds(cfg, seq[0][:1], 0, st)
-    t_reuse = oracle_step_seconds(cfg, seq[1][:1], 1, st)
+    times = [oracle_step_seconds(cfg, x, t, st) for t, x in enumerate(seq)]
     k = cfg.reuse_interval
-    per_cycle = t_refresh + (k - 1) * t_reuse
-    tokens = k * (cfg.n_tokens + cfg.n_extra)
-    return {"value": tokens / per_cycle, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-            "sample": f"batch item 0 of {cfg.batch}: one refresh step ({t_refresh:.2f} s) and one reuse step "
-                      f"({t_reuse:.2f} s), weighted 1:{k - 1} as in the schedule",
+    refresh = [dt for t, dt in enumerate(times) if t % k == 0]
+    reuse = [dt for t, dt in enumerate(times) if t % k != 0]
+    tokens = len(seq) * cfg.batch * (cfg.n_tokens + cfg.n_extra)
+    t_refresh = sum(refresh) / max(len(refresh), 1)
+    t_reuse = sum(reuse) / max(len(reuse), 1)
+    return {"value": tokens / sum(times), "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": f"the whole schedule once, all {cfg.batch} batch items: {len(refresh)} refresh steps ({t_refresh:.2f} s each) "
+                      f"and {len(reuse)} reuse steps ({t_reuse:.2f} s each), {sum(times):.1f} s in all",
             "refresh_s": t_refresh, "reuse_s": t_reuse}
 
 
