@@ -124,31 +124,31 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
       tc_fence_after();
 #pragma unroll 1
       for (int rb = 0; rb < kRowBlocks; ++rb) {
-      const int row = m0 + rb * 128 + quarter * 32 + lane;
-      const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + rb * 256;
-      __nv_bfloat16* dst = c + (size_t)(row < M ? row : 0) * N + n0;
-      for (int j = 0; j < n_cols; j += 32) {
-        uint32_t r[32];
-        tmem_ld32(taddr + j, r);
-        tmem_wait_ld();
-        if (act == kActGelu) {
+        const int row = m0 + rb * 128 + quarter * 32 + lane;
+        const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + rb * 256;
+        __nv_bfloat16* dst = c + (size_t)(row < M ? row : 0) * N + n0;
+        for (int j = 0; j < n_cols; j += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + j, r);
+          tmem_wait_ld();
+          if (act == kActGelu) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(gelu(__uint_as_float(r[e])));
-        }
-        if (row < M) {
+            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(gelu(__uint_as_float(r[e])));
+          }
+          if (row < M) {
 #pragma unroll
-          for (int e = 0; e < 32; e += 8) {
-            if (j + e < n_cols) {
-              __align__(16) __nv_bfloat162 q[4];
+            for (int e = 0; e < 32; e += 8) {
+              if (j + e < n_cols) {
+                __align__(16) __nv_bfloat162 q[4];
 #pragma unroll
-              for (int u = 0; u < 4; ++u)
-                q[u] = __floats2bfloat162_rn(__uint_as_float(r[e + 2 * u]), __uint_as_float(r[e + 2 * u + 1]));
-              *reinterpret_cast<uint4*>(dst + j + e) = *reinterpret_cast<const uint4*>(q);
+                for (int u = 0; u < 4; ++u)
+                  q[u] = __floats2bfloat162_rn(__uint_as_float(r[e + 2 * u]), __uint_as_float(r[e + 2 * u + 1]));
+                *reinterpret_cast<uint4*>(dst + j + e) = *reinterpret_cast<const uint4*>(q);
+              }
             }
           }
         }
       }
-      }  // row blocks
     }
   }
   tc_fence_before();
