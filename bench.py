@@ -275,7 +275,7 @@ def attention_module_workload(toma, torch, flush):
     reuse_us = t_us(lambda: toma.toma_block_proj(desc, 1, x, *ws_w, y, idx, w, ws, None))
     full = t_us(lambda: toma.toma_attention_proj(B, N, cfg.n_heads, cfg.head_dim, cfg.dtype, x, *ws_w, y, ws_full, None))
     mean = (refresh + (k - 1) * reuse_us) / k
-    m = B * (cfg.n_merged + cfg.n_extra)
+    m = B * (cfg.n_tiles * toma.toma_dest_per_tile(desc) + cfg.n_extra)
     qkv = t_us(lambda: toma.toma_linear(x.view(B * N, d)[:m], ws_w[0], y.view(B * N, d)[:m]))
     return {"tokens": B * N, "reuse_interval": k, "refresh_us": refresh, "reuse_us": reuse_us, "block_mean_us": mean,
             "full_module_us": full, "speedup_vs_full_module": full / mean,
@@ -373,7 +373,8 @@ def main():
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
     B, N, d = cfg.batch, cfg.n_tokens + cfg.n_extra, cfg.dim
-    Lm = cfg.n_merged + cfg.n_extra
+    d_loc = toma.toma_dest_per_tile(desc)
+    Lm = cfg.n_tiles * d_loc + cfg.n_extra
 
     def block(t):
         toma.toma_block(desc, t % cycle, xs[t % cycle], out, idx, w, ws, status)
@@ -453,7 +454,7 @@ def main():
     esz = 2 if cfg.dtype == "bf16" else 4
     att_flops = 4.0 * B * Lm * Lm * d
     att_tf = att_flops / (stage_ms["attention"] * 1e-3) / 1e12
-    mrg_bytes = B * (cfg.n_tokens * d * esz + cfg.n_merged * d * esz + cfg.n_tiles * cfg.n_loc * cfg.d_loc * esz)
+    mrg_bytes = B * (cfg.n_tokens * d * esz + cfg.n_tiles * d_loc * d * esz + cfg.n_tiles * cfg.n_loc * d_loc * esz)
     # traffic: dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this workload,
     # from the ncu capture summarised in profiles/attention_tc_cfg3_cfg5a.md (only valid for the default workload)
     traffic = 5331200 + 225024 if args.workload == "cfg3" else None

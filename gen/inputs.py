@@ -116,14 +116,6 @@ class TomaConfig:
     def n_tiles(self) -> int:
         return (self.grid_h // self.tile_h) * (self.grid_w // self.tile_w)
 
-    @property
-    def d_loc(self) -> int:
-        return self.n_loc - int(np.floor(float(np.float32(self.merge_ratio)) * self.n_loc + 0.5))
-
-    @property
-    def n_merged(self) -> int:
-        return self.n_tiles * self.d_loc
-
     def with_(self, **kw) -> "TomaConfig":
         return replace(self, **kw)
 

@@ -104,6 +104,14 @@ TOMA_API toma_status toma_validate(const toma_desc* desc);
 TOMA_API const char* toma_status_str(toma_status s);
 /* Total number of kernels this library has launched in this process (monotonic; for benchmarks). */
 TOMA_API uint64_t toma_launch_counter(void);
+/* TEST-ONLY: overrides launch heuristics so that the parity tests can drive every code path of the
+ * attention kernel's work plan (Eq. 1) and every tile form of the projection kernel (App. C's 4 d^2 N
+ * term).  The library itself never calls it and reads no environment variable; results do not depend
+ * on these settings, only the launch configuration does.  Process-wide; not for concurrent use.
+ *   attention_split: 0 = whole work units per CTA, 1 = spans cut at single key tiles, other = heuristic
+ *   attention_ctas : > 0 = number of persistent CTAs (clamped to the scratch capacity), else heuristic
+ *   linear_tile    : 1 = 128 x 256, 2 = 128 x 320, 3 = 256 x 256 tiles, else heuristic */
+TOMA_API void toma_test_set_tuning(int32_t attention_split, int32_t attention_ctas, int32_t linear_tile);
 
 /* Destination selection (Sec. 4.1, Algorithm 2) inside every tile.
  *   x   [batch][N + n_extra][dim]  in
@@ -155,7 +163,7 @@ TOMA_API size_t toma_attention_workspace_bytes(int32_t batch, int32_t len, int32
                                                int32_t dtype);
 
 /* Host-only diagnostic: how toma_attention would cut this shape's work across its persistent CTAs.
- * A work unit is (batch, head, 128 queries); an iteration is one 64-key tile of a unit; CTA g runs the
+ * A work unit is (batch, head, 256 queries); an iteration is one 64-key tile of a unit; CTA g runs the
  * iterations bounds[g] .. bounds[g+1]-1 of the units laid end to end.
  *   info[0] = number of CTAs G, info[1] = 1 if units are split between CTAs (cut at single key
  *   tiles) or 0 if every CTA gets whole units, info[2] = work units, info[3] = key tiles per unit.

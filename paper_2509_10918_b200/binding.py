@@ -19,7 +19,7 @@ TOMA_BF16, TOMA_F32 = 0, 1
 STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_RATIO", "ERR_TAU", "ERR_WORKSPACE",
                 "ERR_UNSUPPORTED", "ERR_CUDA", "ERR_TIMEOUT", "ERR_SCRATCH_LIMIT"]
 
-EXPORTS = ["toma_select_static", "toma_launch_counter", "toma_workspace_bytes", "toma_weights_bytes", "toma_dest_per_tile", "toma_validate", "toma_status_str",
+EXPORTS = ["toma_select_static", "toma_launch_counter", "toma_test_set_tuning", "toma_workspace_bytes", "toma_weights_bytes", "toma_dest_per_tile", "toma_validate", "toma_status_str",
            "toma_select", "toma_merge_weights", "toma_merge", "toma_attention_workspace_bytes", "toma_attention_plan", "toma_attention",
            "toma_unmerge", "toma_block", "toma_block_host", "toma_linear", "toma_block_proj", "toma_attention_proj_workspace_bytes",
            "toma_attention_proj", "toma_block_mlp", "toma_mlp_workspace_bytes", "toma_mlp",
@@ -61,6 +61,8 @@ def _load() -> ctypes.CDLL:
     lib.toma_dest_per_tile.argtypes = [P]
     lib.toma_launch_counter.restype = ctypes.c_uint64
     lib.toma_launch_counter.argtypes = []
+    lib.toma_test_set_tuning.restype = None
+    lib.toma_test_set_tuning.argtypes = [c_int32, c_int32, c_int32]
     lib.toma_validate.restype = c_int32
     lib.toma_validate.argtypes = [P]
     lib.toma_status_str.restype = c_char_p
@@ -165,6 +167,11 @@ def toma_workspace_bytes(desc: TomaDesc) -> int:
 
 def toma_weights_bytes(desc: TomaDesc) -> int:
     return lib.toma_weights_bytes(ctypes.byref(desc))
+
+
+def toma_test_set_tuning(attention_split: int = -1, attention_ctas: int = 0, linear_tile: int = 0) -> None:
+    """Test-only: force the attention work plan / the projection tile form (defaults restore the heuristics)."""
+    lib.toma_test_set_tuning(attention_split, attention_ctas, linear_tile)
 
 
 def toma_dest_per_tile(desc: TomaDesc) -> int:

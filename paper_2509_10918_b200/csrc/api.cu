@@ -499,5 +499,22 @@ toma_status toma_unmerge_weights_export(const toma_desc* desc, const void* w, fl
 
 namespace toma {
 std::atomic<unsigned long long> g_launches{0};
+std::atomic<int> g_tune_attention_split{-1}, g_tune_attention_ctas{0}, g_tune_linear_tile{0};
+
+int sm_count() {
+  static std::atomic<int> cached[64];
+  int dev = 0, v = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (dev >= 0 && dev < 64 && (v = cached[dev].load(std::memory_order_relaxed)) > 0) return v;
+  if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v < 1) return 148;
+  if (dev >= 0 && dev < 64) cached[dev].store(v, std::memory_order_relaxed);
+  return v;
+}
 }
 extern "C" uint64_t toma_launch_counter(void) { return (uint64_t)toma::g_launches.load(); }
+
+extern "C" void toma_test_set_tuning(int32_t attention_split, int32_t attention_ctas, int32_t linear_tile) {
+  toma::g_tune_attention_split.store(attention_split == 0 || attention_split == 1 ? attention_split : -1);
+  toma::g_tune_attention_ctas.store(attention_ctas > 0 ? attention_ctas : 0);
+  toma::g_tune_linear_tile.store(linear_tile >= 1 && linear_tile <= 3 ? linear_tile : 0);
+}

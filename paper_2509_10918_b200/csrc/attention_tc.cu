@@ -1,36 +1,39 @@
 // Attention core softmax(Q K^T / sqrt(dh)) V (Eq. 1 with tau = 1) on the sm_100a tensor
 // cores, bf16 in / bf16 out, fp32 softmax and accumulation.
 //
-// Work unit = (batch, head, 128 queries); one iteration = one 64-key tile of a unit.  The launch is
-// persistent, two CTAs per SM, and the units' iterations, laid end to end, are cut into one equal
-// contiguous span per CTA, so that every CTA runs the same number of key tiles whatever the unit
-// count (a launch of whole units leaves most SMs idle in its last wave: 320 units on 296 CTA slots
-// took as long as 592).  A span that covers only part of a unit's keys leaves the unnormalised
-// accumulator, the reference maximum and the row sum of its piece in global scratch; the warp that
-// arrives last at the (unit, warp) ticket adds the pieces up and writes the output rows.  Nobody
-// waits for another CTA.
+// Work unit = (batch, head, 256 queries) = two 128-row query tiles that share every K/V tile; one
+// iteration = one 64-key tile of a unit.  The launch is persistent, one CTA per SM, and the units'
+// iterations, laid end to end, are cut into one contiguous span per CTA, so that every CTA runs the
+// same number of key tiles whatever the unit count.  A span that covers only part of a unit's keys
+// leaves the unnormalised accumulator, the reference maximum and the row sum of its piece in global
+// scratch; the warp that arrives last at the (unit, warp) ticket adds the pieces up and writes the
+// output rows.  Nobody waits for another CTA.
 //
-// Inside a CTA warp 4 feeds K and V tiles through a TMA ring, warps 5 and 6 issue tcgen05 MMAs,
-// warp 7 publishes a partial first piece (memory fence and tickets, off everybody else's path),
-// warps 0..3 (one thread per query row) run the online softmax straight out of tensor memory:
-//   S_j = Q K_j^T          -> tensor memory, two 64-column buffers; S_{j+1} is issued before the
-//                             softmax of tile j has finished, so the softmax warps never wait for a
-//                             round trip through the MMA warp
-//   P_j = 2^(S_j*c - m)    -> written back over S_j's first 32 columns as bf16 and used as the
-//                             A operand (from tensor memory) of  O += P_j V_j
-//   row sums (head_dim 64) -> a second tiny MMA, P_j x ones[64 x 16], accumulates sum_k P_jk in
-//                             tensor memory: exactly the bf16 P that multiplies V, so P can be
-//                             produced by truncation (one byte-permute per pair, no conversion on
-//                             the XU pipe) without biasing the normalised result
+// Inside a CTA (12 warps): warps 0..3 run the online softmax of query tile 0, warps 4..7 that of
+// query tile 1 (one thread per query row, straight out of tensor memory), warp 8 feeds Q, K and V
+// through TMA rings, one elected thread of warp 9 issues every tcgen05 MMA, warp 10 publishes a
+// partial first piece (memory fence and tickets, off everybody else's path).
+//   S_q,j = Q_q K_j^T      -> tensor memory, two 64-column buffers per query tile.  MMAs issued by
+//                             one thread execute in order, so S_q,j+2 is issued right behind the
+//                             product that reads P_q,j out of the same buffer, without a round trip
+//                             through a barrier: a softmax warp group always finds its next S tile
+//                             complete, and the tensor pipe, the two softmax groups and the loads
+//                             overlap instead of taking turns.
+//   P_q,j = 2^(S*c - m)    -> written back over S_q,j's first 32 columns as bf16 and used as the
+//                             A operand (from tensor memory) of  O_q += P_q,j V_j
+//   row sums (head_dim 64) -> the B operand of that product is [V_j | 1]: 16 extra columns of ones
+//                             accumulate sum_k P_jk behind O in tensor memory: exactly the bf16 P
+//                             that multiplies V, so P can be produced by truncation (one
+//                             byte-permute per pair, no conversion on the XU pipe) without biasing
+//                             the normalised result
 //   running maximum        -> O (and the row sums) are rescaled only when the maximum grew by more
 //                             than 2^8; the final division by the row sum makes a stale maximum exact
-//   exponentials           -> a quarter of them are a degree-3 polynomial on the FMA pipe (relative
+//   exponentials           -> part of them are a degree-3 polynomial on the FMA pipe (relative
 //                             error 7.5e-5, far below bf16 resolution of P), the rest MUFU ex2
 // The whole S row of a tile (64 fp32) is fetched with one tensor-memory round trip and kept in
 // registers for both the maximum and the exponentials.
-// Keys past the sequence end are zero-filled by TMA and masked out.
-#include <cstdlib>
-
+// Keys past the sequence end are zero-filled by TMA and masked out; query rows past the end are
+// computed on zeros and not written.
 #include "common.cuh"
 #include "tc.cuh"
 
@@ -40,37 +43,44 @@ using namespace tc;
 
 namespace {
 
-constexpr int kBM = 128;  // queries per CTA
-constexpr int kBN = 64;   // keys per tile
+constexpr int kBM = 128;      // rows of one query tile = threads of one softmax warp group
+constexpr int kUM = 2 * kBM;  // queries per work unit
+constexpr int kBN = 64;       // keys per tile
+constexpr int kThreads = 384;
 constexpr float kRescaleThreshold = 8.0f;
 
 template <int DH>
 struct AttCfg {
-  static constexpr int kStages = DH == 64 ? 4 : 2;         // K ring depth = V ring depth
+  static constexpr int kStages = 4;                        // K/V ring depth (S runs two tiles ahead of P V)
+  static constexpr int kQBufs = DH == 64 ? 2 : 1;          // Q buffers: the next unit's Q lands under this unit's tail
   static constexpr int kChunks = DH / 64;                  // 64-column (128-byte) slabs per row
   static constexpr int kQSlab = kBM * 128;                 // 128 query rows x 128 B
+  static constexpr int kQTile = kChunks * kQSlab;          // one query tile
+  static constexpr int kQBytes = 2 * kQTile;               // both query tiles of a unit
   static constexpr int kKvSlab = kBN * 128;                // 64 key rows x 128 B
-  static constexpr int kQBytes = kChunks * kQSlab;
   static constexpr int kKvBytes = kChunks * kKvSlab;       // one K or V tile
   static constexpr int kOnesBytes = kBN * 128;             // [64 keys][64] bf16 ones: the N chunk after V in the PV operand
-  static constexpr int kSmemBytes = 1024 + kQBytes + 2 * kStages * kKvBytes + kOnesBytes + 256;
+  static constexpr int kBarBytes = 512;
+  static constexpr int kSmemBytes = 1024 + kQBufs * kQBytes + 2 * kStages * kKvBytes + kOnesBytes + kBarBytes;
   static constexpr bool kSumMma = DH == 64;                // row sums on the tensor pipe, truncated P
-  static constexpr int kTmemCols = 256;
-  static constexpr int kColS = 0, kColO = 128;  // S buffers at columns 0 and 64; O (and, behind it, the row sums) at 128
+  static constexpr int kTmemCols = 512;
+  // S buffer (q, b) at column (2 q + b) * 64; O_q (and, behind it, the row sums) from column 256
+  static constexpr int kColS = 0, kColO = 256, kOStride = DH == 64 ? 96 : 128;
 };
 
 struct Barriers {
-  uint64_t q_full, q_empty;           // per piece: Q landed / every S MMA of the piece has read Q
-  uint64_t k_full[4], v_empty[4];     // per tile: K and V landed / PV MMAs of the tile done
-  uint64_t s_full[2], p_full[2];      // per tile: S ready for the softmax / P ready for the PV MMAs
-  uint64_t o_done, o_free;            // per piece: accumulator complete / epilogue has read it
+  uint64_t q_full[2], q_empty[2];     // per piece: Q landed / every S MMA of the piece has read Q
+  uint64_t k_full[4], kv_empty[4];    // per tile: K and V landed / every MMA that reads them is done
+  uint64_t s_full[2][2], p_full[2][2];  // per tile and query tile: S ready for the softmax / P ready for the PV MMAs
+  uint64_t o_done[2], o_free[2];      // per piece and query tile: accumulator complete / epilogue has read it
   uint64_t pub_ready, pub_done;       // first partial piece: written by the softmax warps / published, tickets drawn
-  uint32_t first_ticket[4];           // per softmax warp: ticket its first (partial) piece drew
+  uint32_t first_ticket[8];           // per softmax warp: ticket its first (partial) piece drew
   uint32_t others_done;               // set by the publisher when the span's last unit has all its other pieces in scratch
-  uint32_t poll_stop;                 // set by softmax warp 0 when the answer is no longer needed
+  uint32_t poll_stop[2];              // set by each softmax group when the answer is no longer needed
   uint32_t tmem_base;
   int abort_flag;
 };
+static_assert(sizeof(Barriers) <= 512, "barrier block outgrew its reservation");
 
 // The iterations [0, T) are cut into G spans at multiples of `quantum`: with T / quantum = q * G + r,
 // the first r spans hold q + 1 quanta and the others q.
@@ -99,9 +109,33 @@ __device__ __forceinline__ Piece piece_at(int it, int it_end, int nblk) {
   return p;
 }
 
-// Scratch of one piece: O as [DH / 4][128 rows] float4, then m[128], l[128].
+// A position in the CTA's span for the single-thread roles: `n` counts key tiles across pieces (ring
+// slots, S buffers and their barrier phases follow n), `pc` counts pieces (phases of the per-piece
+// barriers), `j` is the tile inside the current piece of `cnt` tiles.
+struct Cursor {
+  int it, it_end, nblk, j, cnt, pc, n;
+  __device__ __forceinline__ void load() {
+    const int left = it_end - it, in_unit = nblk - it % nblk;
+    cnt = left < in_unit ? left : in_unit;
+  }
+  __device__ __forceinline__ void init(int b, int e, int nb) {
+    it = b, it_end = e, nblk = nb, j = 0, pc = 0, n = 0;
+    load();
+  }
+  __device__ __forceinline__ bool valid() const { return it < it_end; }
+  __device__ __forceinline__ bool last_of_piece() const { return j + 1 == cnt; }
+  __device__ __forceinline__ void next() {
+    ++n;
+    if (++j == cnt) {
+      it += cnt, ++pc, j = 0;
+      load();
+    }
+  }
+};
+
+// Scratch of one piece: O as [DH / 4][256 rows] float4, then m[256], l[256].
 template <int DH>
-__host__ __device__ constexpr size_t piece_floats() { return (size_t)kBM * DH + 2 * kBM; }
+__host__ __device__ constexpr size_t piece_floats() { return (size_t)kUM * DH + 2 * kUM; }
 
 __device__ __forceinline__ float ex2_mufu(float x) {
   float y;
@@ -246,11 +280,11 @@ __device__ __forceinline__ void store_row32(__nv_bfloat16* dst, const uint32_t (
   }
 }
 
-// Where the output rows of unit u start for this thread's query row (nullptr past the sequence end).
+// Where the output rows of unit u start for query row `row` (0..255) of the unit (nullptr past the sequence end).
 template <int DH>
 __device__ __forceinline__ __nv_bfloat16* out_row(__nv_bfloat16* o, int u, int row, int L, int heads) {
-  const int nq = (L + kBM - 1) / kBM;
-  const int bh = u / nq, qi = (u - bh * nq) * kBM + row, b = bh / heads, h = bh - b * heads;
+  const int nq = (L + kUM - 1) / kUM;
+  const int bh = u / nq, qi = (u - bh * nq) * kUM + row, b = bh / heads, h = bh - b * heads;
   if (qi >= L) return nullptr;
   return o + ((size_t)b * L + qi) * ((size_t)heads * DH) + (size_t)h * DH;
 }
@@ -271,7 +305,7 @@ __device__ __forceinline__ const float* slot_of(const float* pieces, const Spans
 template <int DH>
 __device__ __noinline__ void combine_rows(const float* pieces, Spans sp, int u, int g_first, int g_last, int row,
                                           __nv_bfloat16* dst) {
-  constexpr size_t kM = (size_t)kBM * DH, kL = (size_t)kBM * DH + kBM;
+  constexpr size_t kM = (size_t)kUM * DH, kL = (size_t)kUM * DH + kUM;
   float M = -INFINITY;
   for (int g = g_first; g <= g_last; g += 2) {
     const float* sa = slot_of<DH>(pieces, sp, g, u);
@@ -296,8 +330,8 @@ __device__ __noinline__ void combine_rows(const float* pieces, Spans sp, int u, 
         float4 va[8], vb[8];
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-          va[q] = __ldcg(reinterpret_cast<const float4*>(sa) + (size_t)(half * 16 + c * 8 + q) * kBM + row);
-          vb[q] = __ldcg(reinterpret_cast<const float4*>(sb) + (size_t)(half * 16 + c * 8 + q) * kBM + row);
+          va[q] = __ldcg(reinterpret_cast<const float4*>(sa) + (size_t)(half * 16 + c * 8 + q) * kUM + row);
+          vb[q] = __ldcg(reinterpret_cast<const float4*>(sb) + (size_t)(half * 16 + c * 8 + q) * kUM + row);
         }
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -337,7 +371,7 @@ __device__ __forceinline__ uint32_t ld_acquire_cta(const uint32_t* smem_word) {
 }
 
 // Publishes this warp's 32 rows of a piece and takes the (unit, warp) ticket.  Returns the number
-// of contributors that had taken it before.
+// of contributors that had taken it before.  Called by whole warps only.
 __device__ __forceinline__ uint32_t take_ticket(uint32_t* ticket, int lane) {
   __threadfence();
   __syncwarp();
@@ -346,33 +380,42 @@ __device__ __forceinline__ uint32_t take_ticket(uint32_t* ticket, int lane) {
   return __shfl_sync(0xffffffffu, t, 0);
 }
 
+// The per-thread view of a softmax thread: its query tile, its row in the unit, its accumulator.
+struct Row {
+  int q;        // query tile (softmax warp group) 0 or 1
+  int warp;     // softmax warp 0..7 = ticket column
+  int lane;
+  int row;      // query row inside the unit, 0..255
+  uint32_t ob;  // tensor-memory address of this row's accumulator
+};
+
 // End of a piece that covers all keys of its unit (the only kind when units are kept whole), run by
 // the softmax warps: wait for the accumulator, normalise, write the rows out.  Returns false when
 // the wait ran out.
 template <int DH>
-__device__ __forceinline__ bool finish_whole(uint32_t ob, Barriers* bar, int pos, int pc, int row, float l, __nv_bfloat16* o,
-                                             int L, int heads, uint32_t* dev_status) {
+__device__ __forceinline__ bool finish_whole(const Row& t, Barriers* bar, int unit, int pc, float l, __nv_bfloat16* o, int L,
+                                             int heads, uint32_t* dev_status) {
   using C = AttCfg<DH>;
-  if (!mbar_wait(&bar->o_done, pc & 1, dev_status, &bar->abort_flag)) return false;
+  if (!mbar_wait(&bar->o_done[t.q], pc & 1, dev_status, &bar->abort_flag)) return false;
   tc_fence_after();
   if (C::kSumMma) {
     uint32_t rs[16];
-    tmem_ld16(ob + DH, rs);
+    tmem_ld16(t.ob + DH, rs);
     tmem_wait_ld();
     l = __uint_as_float(rs[0]);
   }
-  __nv_bfloat16* dst = out_row<DH>(o, pos, row, L, heads);
+  __nv_bfloat16* dst = out_row<DH>(o, unit, t.row, L, heads);
   const float inv = 1.f / l;
 #pragma unroll
   for (int c = 0; c < DH / 32; ++c) {
     uint32_t r[32];
-    tmem_ld32(ob + c * 32, r);
+    tmem_ld32(t.ob + c * 32, r);
     tmem_wait_ld();
     if (dst) store_row32(dst + c * 32, r, inv);
   }
   tc_fence_before();
   __syncwarp();
-  if ((row & 31) == 0) mbar_arrive(&bar->o_free);  // the next piece's first PV product may overwrite the accumulator
+  if (t.lane == 0) mbar_arrive(&bar->o_free[t.q]);  // the next piece's first PV product may overwrite the accumulator
   return true;
 }
 
@@ -385,16 +428,18 @@ __device__ __forceinline__ bool finish_whole(uint32_t ob, Barriers* bar, int pos
 //     ticket is drawn; the warp that draws a unit's last ticket adds its pieces up.  A last piece
 //     does that here; a first piece, with more of the span to come, hands the fence and the
 //     tickets' round trips to the publisher thread and looks at the outcome in settle_first_piece.
+// Every decision that ends in a warp-wide operation is taken once per warp (lane 0 reads, the warp
+// gets the value by shuffle), so a warp always goes one way as a whole.
 // Out of line (it runs at most twice per CTA and is register-hungry).  Returns false when the wait
 // ran out.
 template <int DH>
-__device__ __noinline__ bool finish_partial(uint32_t ob, Barriers* bar, Piece p, int pc, bool last_of_span, int row,
-                                            float m_used, float l, __nv_bfloat16* o, int L, int heads, Spans sp,
-                                            uint32_t* tickets, float* pieces, uint32_t* dev_status) {
+__device__ __noinline__ bool finish_partial(Row t, Barriers* bar, Piece p, int pc, bool last_of_span, float m_used, float l,
+                                            __nv_bfloat16* o, int L, int heads, Spans sp, uint32_t* tickets, float* pieces,
+                                            uint32_t* dev_status) {
   using C = AttCfg<DH>;
-  constexpr size_t kM = (size_t)kBM * DH, kL = (size_t)kBM * DH + kBM;
-  const int warp = row >> 5, lane = row & 31;
-  uint32_t* ticket = tickets + (size_t)p.u * 4 + warp;
+  constexpr size_t kM = (size_t)kUM * DH, kL = (size_t)kUM * DH + kUM;
+  const int row = t.row, lane = t.lane;
+  uint32_t* ticket = tickets + (size_t)p.u * 8 + t.warp;
   const int g_first = sp.owner(p.u * sp.nblk), g_last = sp.owner((p.u + 1) * sp.nblk - 1);
   bool own_first = false;  // this CTA is the lower of the two contributors
   const float* other = nullptr;
@@ -402,21 +447,27 @@ __device__ __noinline__ bool finish_partial(uint32_t ob, Barriers* bar, Piece p,
   float4 vo[16];
   // the publisher warp watches the tickets of the span's last unit; its answer carries the
   // acquire that orders the loads below after the other contributor's writes
-  const bool direct = last_of_span && g_last == g_first + 1 && ld_acquire_cta(&bar->others_done) == 1u;
-  if (last_of_span && row == 0) *(volatile uint32_t*)&bar->poll_stop = 1u;
+  uint32_t others = 0;
+  if (last_of_span && g_last == g_first + 1) {
+    if (lane == 0) others = ld_acquire_cta(&bar->others_done);
+    __syncwarp();
+    others = __shfl_sync(0xffffffffu, others, 0);
+  }
+  const bool direct = others == 1u;
+  if (last_of_span && (row & (kBM - 1)) == 0) *(volatile uint32_t*)&bar->poll_stop[t.q] = 1u;
   if (direct) {
     own_first = (int)blockIdx.x == g_first;
     other = slot_of<DH>(pieces, sp, own_first ? g_last : g_first, p.u);
     m_o = __ldcg(other + kM + row);
     l_o = __ldcg(other + kL + row);
 #pragma unroll
-    for (int q = 0; q < 16; ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)q * kBM + row);
+    for (int q = 0; q < 16; ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)q * kUM + row);
   }
-  if (!mbar_wait(&bar->o_done, pc & 1, dev_status, &bar->abort_flag)) return false;
+  if (!mbar_wait(&bar->o_done[t.q], pc & 1, dev_status, &bar->abort_flag)) return false;
   tc_fence_after();
   if (C::kSumMma) {
     uint32_t rs[16];
-    tmem_ld16(ob + DH, rs);
+    tmem_ld16(t.ob + DH, rs);
     tmem_wait_ld();
     l = __uint_as_float(rs[0]);
   }
@@ -432,12 +483,12 @@ __device__ __noinline__ bool finish_partial(uint32_t ob, Barriers* bar, Piece p,
 #pragma unroll
   for (int c = 0; c < DH / 32; ++c) {
     uint32_t r[32];
-    tmem_ld32(ob + c * 32, r);
+    tmem_ld32(t.ob + c * 32, r);
     tmem_wait_ld();
     if (direct) {
       if (c > 0 && (c & 1) == 0) {  // next 64 columns of the other piece
 #pragma unroll
-        for (int q = 0; q < 16; ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)(c * 8 + q) * kBM + row);
+        for (int q = 0; q < 16; ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)(c * 8 + q) * kUM + row);
       }
 #pragma unroll
       for (int q = 0; q < 8; ++q) {
@@ -453,13 +504,13 @@ __device__ __noinline__ bool finish_partial(uint32_t ob, Barriers* bar, Piece p,
     } else {
 #pragma unroll
       for (int e = 0; e < 32; e += 4)
-        reinterpret_cast<float4*>(slot)[(size_t)(c * 8 + (e >> 2)) * kBM + row] =
+        reinterpret_cast<float4*>(slot)[(size_t)(c * 8 + (e >> 2)) * kUM + row] =
             make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
     }
   }
   tc_fence_before();
   __syncwarp();
-  if (lane == 0) mbar_arrive(&bar->o_free);  // the next piece's first PV product may overwrite the accumulator
+  if (lane == 0) mbar_arrive(&bar->o_free[t.q]);  // the next piece's first PV product may overwrite the accumulator
   if (direct) return true;
   slot[kM + row] = m_used;
   slot[kL + row] = l;
@@ -477,16 +528,16 @@ __device__ __noinline__ bool finish_partial(uint32_t ob, Barriers* bar, Piece p,
 // contributors, which run that unit at the end of their spans, are normally later), add the
 // unit's pieces up now.
 template <int DH>
-__device__ __noinline__ void settle_first_piece(Barriers* bar, int it_begin, int it_end, int row, __nv_bfloat16* o, int L,
+__device__ __noinline__ void settle_first_piece(Barriers* bar, int it_begin, int it_end, Row t, __nv_bfloat16* o, int L,
                                                 int heads, Spans sp, const float* pieces, uint32_t* dev_status) {
   const int nblk = sp.nblk, u = it_begin / nblk;
   const bool first_partial = it_begin > u * nblk || it_end < (u + 1) * nblk;
   if (!first_partial || it_end <= (u + 1) * nblk) return;  // whole, or also the span's last piece: settled already
   const int g_first = sp.owner(u * nblk), g_last = sp.owner((u + 1) * nblk - 1);
   if (!mbar_wait(&bar->pub_done, 0, dev_status, &bar->abort_flag)) return;
-  if (bar->first_ticket[row >> 5] != (uint32_t)(g_last - g_first)) return;
+  if (bar->first_ticket[t.warp] != (uint32_t)(g_last - g_first)) return;
   __threadfence();
-  combine_rows<DH>(pieces, sp, u, g_first, g_last, row, out_row<DH>(o, u, row, L, heads));
+  combine_rows<DH>(pieces, sp, u, g_first, g_last, t.row, out_row<DH>(o, u, t.row, L, heads));
 }
 
 // The ragged last key tile of a sequence: out of line, so that the hot loop holds one copy of the
@@ -499,7 +550,7 @@ __device__ __noinline__ bool softmax_tile_ragged(uint32_t sb, uint32_t ob, float
 }
 
 template <int DH>
-__global__ void __launch_bounds__(256, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, int L, int heads,
                     float scale_log2, Spans sp, uint32_t* __restrict__ tickets, float* __restrict__ pieces,
@@ -508,35 +559,35 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = smem;
-  uint8_t* sK = sQ + C::kQBytes;
+  uint8_t* sK = sQ + C::kQBufs * C::kQBytes;
   uint8_t* sV = sK + C::kStages * C::kKvBytes;
   uint8_t* sOnes = sV + C::kStages * C::kKvBytes;
   Barriers* bar = reinterpret_cast<Barriers*>(sOnes + C::kOnesBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nblk = sp.nblk;
-  const int nq = (L + kBM - 1) / kBM;  // units per (batch, head)
+  const int nq = (L + kUM - 1) / kUM;  // units per (batch, head)
   const int it_begin = sp.bound(blockIdx.x), it_end = sp.bound(blockIdx.x + 1);
-  // Every role walks the same pieces; `n` counts this CTA's tiles across pieces (ring slots, S
-  // buffers and their barrier phases follow n), `pc` counts pieces (phases of the per-piece barriers).
 
   if (threadIdx.x == 0) {
-    mbar_init(&bar->q_full, 1);
-    mbar_init(&bar->q_empty, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&bar->q_full[s], 1);
+      mbar_init(&bar->q_empty[s], 1);
+      mbar_init(&bar->o_done[s], 1);
+      mbar_init(&bar->o_free[s], 4);  // one arrival per softmax warp of the group
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(&bar->s_full[s][b], 1);
+        mbar_init(&bar->p_full[s][b], 4);
+      }
+      bar->poll_stop[s] = 0;
+    }
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&bar->k_full[s], 1);
-      mbar_init(&bar->v_empty[s], 1);
+      mbar_init(&bar->kv_empty[s], 1);
     }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&bar->s_full[s], 1);
-      mbar_init(&bar->p_full[s], 4);  // one arrival per softmax warp
-    }
-    mbar_init(&bar->o_done, 1);
-    mbar_init(&bar->o_free, 4);
-    mbar_init(&bar->pub_ready, 4);
+    mbar_init(&bar->pub_ready, 8);
     mbar_init(&bar->pub_done, 1);
     bar->others_done = 0;
-    bar->poll_stop = 0;
     bar->abort_flag = 0;
     mbar_fence_init();
   }
@@ -544,154 +595,164 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     for (int e = threadIdx.x; e < C::kOnesBytes / 4; e += blockDim.x) reinterpret_cast<uint32_t*>(sOnes)[e] = 0x3F803F80u;
     fence_proxy_async();
   }
-  if (threadIdx.x == 128) {  // descriptor fetches overlap the previous kernel's tail
+  if (threadIdx.x == 256) {  // descriptor fetches overlap the previous kernel's tail
     prefetch_tmap(&tm_q);
     prefetch_tmap(&tm_k);
     prefetch_tmap(&tm_v);
   }
   dependency_wait();
   if (threadIdx.x == 0) release_dependents();
-  if (warp == 5) tmem_alloc(&bar->tmem_base, C::kTmemCols);
+  if (warp == 9) tmem_alloc(&bar->tmem_base, C::kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bar->tmem_base;
   volatile int* abort_flag = &bar->abort_flag;
 
-  if (warp == 4) {
+  if (warp == 8) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      bool ok = true;
-      int n = 0, pc = 0;
-      for (int it = it_begin; ok && it < it_end; ++pc) {
-        const Piece p = piece_at(it, it_end, nblk);
-        it += p.cnt;
-        const int bh = p.u / nq, q0 = (p.u - bh * nq) * kBM, b = bh / heads, h = bh - b * heads;
-        // Q's buffer is free once the S MMAs of the previous piece have read it
-        if (pc > 0 && !mbar_wait(&bar->q_empty, (pc - 1) & 1, dev_status, abort_flag)) break;
-        mbar_expect_tx(&bar->q_full, C::kQBytes);
-        for (int c = 0; c < C::kChunks; ++c) tma_load_3d(sQ + c * C::kQSlab, &tm_q, &bar->q_full, h * DH + c * 64, q0, b);
-        for (int j = 0; j < p.cnt; ++j, ++n) {
-          const int s = n % C::kStages;
-          const uint32_t par = ((n / C::kStages) - 1) & 1;
-          if (n >= C::kStages && !mbar_wait(&bar->v_empty[s], par, dev_status, abort_flag)) { ok = false; break; }
-          const int key0 = (p.k0 + j) * kBN;
-          mbar_expect_tx(&bar->k_full[s], 2 * C::kKvBytes);  // K and V of a tile arrive under one barrier
-          for (int c = 0; c < C::kChunks; ++c)
-            tma_load_3d(sK + s * C::kKvBytes + c * C::kKvSlab, &tm_k, &bar->k_full[s], h * DH + c * 64, key0, b);
-          for (int c = 0; c < C::kChunks; ++c)
-            tma_load_3d(sV + s * C::kKvBytes + c * C::kKvSlab, &tm_v, &bar->k_full[s], h * DH + c * 64, key0, b);
+    if (elect_one()) {
+      Cursor c;
+      for (c.init(it_begin, it_end, nblk); c.valid(); c.next()) {
+        if (c.j == 0) {
+          const int u = c.it / nblk;
+          const int bh = u / nq, q0 = (u - bh * nq) * kUM, b = bh / heads, h = bh - b * heads;
+          const int qb = c.pc % C::kQBufs;
+          // a Q buffer is free once the S MMAs of the piece that used it have read it
+          if (c.pc >= C::kQBufs && !mbar_wait(&bar->q_empty[qb], ((c.pc / C::kQBufs) - 1) & 1, dev_status, abort_flag)) break;
+          mbar_expect_tx(&bar->q_full[qb], C::kQBytes);
+          for (int t = 0; t < 2; ++t)
+            for (int ch = 0; ch < C::kChunks; ++ch)
+              tma_load_3d(sQ + qb * C::kQBytes + t * C::kQTile + ch * C::kQSlab, &tm_q, &bar->q_full[qb], h * DH + ch * 64,
+                          q0 + t * kBM, b);
         }
+        const int u = c.it / nblk, k0 = c.it - u * nblk;
+        const int bh = u / nq, b = bh / heads, h = bh - b * heads;
+        const int s = c.n % C::kStages;
+        if (c.n >= C::kStages && !mbar_wait(&bar->kv_empty[s], ((c.n / C::kStages) - 1) & 1, dev_status, abort_flag)) break;
+        const int key0 = (k0 + c.j) * kBN;
+        mbar_expect_tx(&bar->k_full[s], 2 * C::kKvBytes);  // K and V of a tile arrive under one barrier
+        for (int ch = 0; ch < C::kChunks; ++ch)
+          tma_load_3d(sK + s * C::kKvBytes + ch * C::kKvSlab, &tm_k, &bar->k_full[s], h * DH + ch * 64, key0, b);
+        for (int ch = 0; ch < C::kChunks; ++ch)
+          tma_load_3d(sV + s * C::kKvBytes + ch * C::kKvSlab, &tm_v, &bar->k_full[s], h * DH + ch * 64, key0, b);
       }
     }
-  } else if (warp == 5) {
-    // ------------------------------------------------------------------ MMA issuer for S = Q K^T
-    // The two issuers are separate warps so that their waits and commits (each a serial, ~100-cycle
-    // operation for a single thread) proceed in parallel.
-    if (lane == 0) {
+  } else if (warp == 9) {
+    // ------------------------------------------------------------------ MMA issuer
+    // One thread issues everything, so the tensor pipe executes in the order written here: the S
+    // product of tile n+2 goes into the buffer whose P the PV product of tile n, issued just
+    // before, still reads.
+    if (elect_one()) {
       constexpr uint32_t idesc_s = idesc_f16(kFmtBF16, kFmtBF16, false, false, kBM, kBN);
-      // Descriptors are built once and advanced by adding a constant to the 14-bit start-address
-      // field (no carry: all tiles live below 256 KB).
-      const uint64_t q_desc = smem_desc_sw128(smem_u32(sQ), 16, 1024);
-      const uint64_t k_desc0 = smem_desc_sw128(smem_u32(sK), 16, 1024);
-      bool ok = true;
-      int n = 0, pc = 0;
-      for (int it = it_begin; ok && it < it_end; ++pc) {
-        const Piece p = piece_at(it, it_end, nblk);
-        it += p.cnt;
-        if (!mbar_wait(&bar->q_full, pc & 1, dev_status, abort_flag)) break;
-        for (int j = 0; j < p.cnt; ++j, ++n) {
-          const int s = n % C::kStages;
-          if (!mbar_wait(&bar->k_full[s], (n / C::kStages) & 1, dev_status, abort_flag)) { ok = false; break; }
-          // S_n overwrites the buffer whose P_{n-2} the PV (and row-sum) MMAs of tile n-2 read as their
-          // A operand.  MMAs into different accumulators are not ordered among themselves, so that read
-          // has to be complete before the overwrite is issued.
-          if (n >= 2 && !mbar_wait(&bar->v_empty[(n - 2) % C::kStages], ((n - 2) / C::kStages) & 1, dev_status, abort_flag)) {
-            ok = false;
-            break;
-          }
-          tc_fence_after();
-          const uint64_t kb = k_desc0 + (uint64_t)((s * C::kKvBytes) >> 4);
-          const uint32_t t_s = tmem + C::kColS + (n & 1) * kBN;
-#pragma unroll
-          for (int kk = 0; kk < DH / 16; ++kk) {
-            const uint64_t qoff = (uint64_t)(((kk >> 2) * C::kQSlab + (kk & 3) * 32) >> 4);
-            const uint64_t koff = (uint64_t)(((kk >> 2) * C::kKvSlab + (kk & 3) * 32) >> 4);
-            mma_ss(t_s, q_desc + qoff, kb + koff, idesc_s, kk > 0);
-          }
-          mma_commit(&bar->s_full[n & 1]);
-        }
-        if (ok) mma_commit(&bar->q_empty);
-      }
-    }
-  } else if (warp == 6) {
-    // ------------------------------------------------------------------ MMA issuer for O += P V
-    if (lane == 0) {
       // With row sums on the tensor pipe the B operand is [V | ones]: N = DH + 16, the 16 extra
       // columns come from a constant slab of ones placed one "leading byte offset" after V's slab,
       // so one MMA per 16 keys updates O and the row sums (which sit right behind O in tensor memory).
       constexpr uint32_t idesc_o = idesc_f16(kFmtBF16, kFmtBF16, false, true, kBM, C::kSumMma ? DH + 16 : DH);
-      uint64_t v_desc[4];
-#pragma unroll
-      for (int st = 0; st < 4; ++st) {
-        const int ss = st < C::kStages ? st : 0;
-        const uint32_t va = smem_u32(sV + ss * C::kKvBytes);
-        v_desc[st] = smem_desc_sw128(va, C::kSumMma ? smem_u32(sOnes) - va : (uint32_t)C::kKvSlab, 1024);
-      }
-      const uint32_t t_o = tmem + C::kColO;
+      // Descriptors are built once and advanced by adding a constant to the 14-bit start-address
+      // field (no carry: all tiles live below 256 KB).
+      const uint64_t q_desc0 = smem_desc_sw128(smem_u32(sQ), 16, 1024);
+      const uint64_t k_desc0 = smem_desc_sw128(smem_u32(sK), 16, 1024);
+      const uint32_t v_addr0 = smem_u32(sV), ones_addr = smem_u32(sOnes);
+      Cursor cs, cp;  // the S products run two tiles ahead of the PV products
+      cs.init(it_begin, it_end, nblk);
+      cp.init(it_begin, it_end, nblk);
       bool ok = true;
-      int n = 0, pc = 0;
-      for (int it = it_begin; ok && it < it_end; ++pc) {
-        const Piece p = piece_at(it, it_end, nblk);
-        it += p.cnt;
-        for (int j = 0; j < p.cnt; ++j, ++n) {
-          const int s = n % C::kStages;
-          // P ready implies that the K/V tile has landed
-          if (!mbar_wait(&bar->p_full[n & 1], (n >> 1) & 1, dev_status, abort_flag)) { ok = false; break; }
-          // the first product of a piece overwrites the accumulator the previous epilogue reads
-          if (j == 0 && pc > 0 && !mbar_wait(&bar->o_free, (pc - 1) & 1, dev_status, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          const uint64_t vb = s == 0 ? v_desc[0] : s == 1 ? v_desc[1] : s == 2 ? v_desc[2] : v_desc[3];
-          const uint32_t t_p = tmem + C::kColS + (n & 1) * kBN;
+      // Q of the piece and K of the tile that `cs` points at have landed
+      auto s_inputs = [&]() -> bool {
+        if (cs.j == 0 && !mbar_wait(&bar->q_full[cs.pc % C::kQBufs], (cs.pc / C::kQBufs) & 1, dev_status, abort_flag)) return false;
+        return mbar_wait(&bar->k_full[cs.n % C::kStages], (cs.n / C::kStages) & 1, dev_status, abort_flag);
+      };
+      auto issue_s = [&](int q) {
+        const int s = cs.n % C::kStages, b = cs.n & 1, qb = cs.pc % C::kQBufs;
+        const uint64_t qd = q_desc0 + (uint64_t)((qb * C::kQBytes + q * C::kQTile) >> 4);
+        const uint64_t kd = k_desc0 + (uint64_t)((s * C::kKvBytes) >> 4);
+        const uint32_t t_s = tmem + C::kColS + (2 * q + b) * kBN;
 #pragma unroll
-          for (int kk = 0; kk < kBN / 16; ++kk) {  // 16 keys per MMA: 8 packed columns of P, 16 rows of V
-            mma_ts(t_o, t_p + kk * 8, vb + (uint64_t)((kk * 2048) >> 4), idesc_o, j > 0 || kk > 0);
-          }
-          mma_commit(&bar->v_empty[s]);  // frees the K/V slot and tells everyone that this PV has landed
+        for (int kk = 0; kk < DH / 16; ++kk) {
+          const uint64_t qoff = (uint64_t)(((kk >> 2) * C::kQSlab + (kk & 3) * 32) >> 4);
+          const uint64_t koff = (uint64_t)(((kk >> 2) * C::kKvSlab + (kk & 3) * 32) >> 4);
+          mma_ss(t_s, qd + qoff, kd + koff, idesc_s, kk > 0);
+        }
+        mma_commit(&bar->s_full[q][b]);
+      };
+      for (int pre = 0; pre < 2 && ok && cs.valid(); ++pre) {
+        ok = s_inputs();
+        if (!ok) break;
+        tc_fence_after();
+        issue_s(0);
+        issue_s(1);
+        if (cs.last_of_piece()) mma_commit(&bar->q_empty[cs.pc % C::kQBufs]);
+        cs.next();
+      }
+      while (ok && cp.valid()) {
+        const int s = cp.n % C::kStages, b = cp.n & 1;
+        const bool more = cs.valid();
+        const uint32_t va = v_addr0 + s * C::kKvBytes;
+        const uint64_t vd = smem_desc_sw128(va, C::kSumMma ? ones_addr - va : (uint32_t)C::kKvSlab, 1024);
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          // P ready implies that the K/V tile has landed
+          if (!mbar_wait(&bar->p_full[q][b], (cp.n >> 1) & 1, dev_status, abort_flag)) { ok = false; break; }
+          // the first product of a piece overwrites the accumulator the previous epilogue reads
+          if (cp.j == 0 && cp.pc > 0 && !mbar_wait(&bar->o_free[q], (cp.pc - 1) & 1, dev_status, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t t_o = tmem + C::kColO + q * C::kOStride;
+          const uint32_t t_p = tmem + C::kColS + (2 * q + b) * kBN;
+#pragma unroll
+          for (int kk = 0; kk < kBN / 16; ++kk)  // 16 keys per MMA: 8 packed columns of P, 16 rows of V
+            mma_ts(t_o, t_p + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o, cp.j > 0 || kk > 0);
           // One phase per piece: the next piece's products wait for o_free, which the epilogue gives
           // only after it has seen this phase, so a waiter is never two phases behind.
-          if (j + 1 == p.cnt) mma_commit(&bar->o_done);
+          if (cp.last_of_piece()) mma_commit(&bar->o_done[q]);
+          if (q == 1) mma_commit(&bar->kv_empty[s]);  // frees the K/V slot; also "PV of this tile has landed" for a rescale
+          if (more) {
+            if (q == 0) {
+              ok = s_inputs();
+              if (!ok) break;
+              tc_fence_after();
+            }
+            issue_s(q);
+          }
         }
+        if (!ok) break;
+        if (more) {
+          if (cs.last_of_piece()) mma_commit(&bar->q_empty[cs.pc % C::kQBufs]);
+          cs.next();
+        }
+        cp.next();
       }
     }
-  } else if (warp == 7) {
+  } else if (warp == 10) {
     // ------------------------------------------------------------------ publisher
     if (lane == 0) {
       // When the span's first piece is partial and more pieces follow, make that piece
-      // visible to the other CTAs and draw its four tickets here, off the softmax warps' path.
+      // visible to the other CTAs and draw its eight tickets here, off the softmax warps' path.
       const int u = it_begin / nblk;
       const bool early = (it_begin > u * nblk || it_end < (u + 1) * nblk) && it_end > (u + 1) * nblk;
       if (early && mbar_wait(&bar->pub_ready, 0, dev_status, abort_flag)) {
         __threadfence();
-        uint32_t t[4];
+        uint32_t t[8];
 #pragma unroll
-        for (int w = 0; w < 4; ++w) t[w] = atomicAdd(&tickets[(size_t)u * 4 + w], 1u);
+        for (int w = 0; w < 8; ++w) t[w] = atomicAdd(&tickets[(size_t)u * 8 + w], 1u);
 #pragma unroll
-        for (int w = 0; w < 4; ++w) bar->first_ticket[w] = t[w];
+        for (int w = 0; w < 8; ++w) bar->first_ticket[w] = t[w];
         mbar_arrive(&bar->pub_done);
       }
       // When the span ends inside a unit that one other CTA shares, that CTA ran its part at the
-      // start of its span and has normally published it long since.  Watch its four tickets (acquire)
+      // start of its span and has normally published it long since.  Watch its eight tickets (acquire)
       // and leave the answer in shared memory for the softmax warps: they add the two pieces up
       // straight from tensor memory if the answer is there when their last piece ends, and go
       // through scratch and tickets otherwise.  Polling keeps the ticket out of their registers.
       const int ul = (it_end - 1) / nblk;
       if (it_end < (ul + 1) * nblk && sp.owner((ul + 1) * nblk - 1) == sp.owner(ul * nblk) + 1) {
-        const uint32_t* tk = tickets + (size_t)ul * 4;
+        const uint32_t* tk = tickets + (size_t)ul * 8;
         for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-          if (*(volatile uint32_t*)&bar->poll_stop || *abort_flag) break;
-          if (ld_acquire_gpu(tk) == 1u && ld_acquire_gpu(tk + 1) == 1u && ld_acquire_gpu(tk + 2) == 1u &&
-              ld_acquire_gpu(tk + 3) == 1u) {
+          if ((*(volatile uint32_t*)&bar->poll_stop[0] && *(volatile uint32_t*)&bar->poll_stop[1]) || *abort_flag) break;
+          bool all = true;
+#pragma unroll
+          for (int w = 0; w < 8; ++w) all = all && ld_acquire_gpu(tk + w) == 1u;
+          if (all) {
             st_release_cta(&bar->others_done, 1u);
             break;
           }
@@ -699,11 +760,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
       }
     }
-  } else if (warp < 4) {
+  } else if (warp < 8) {
     // ------------------------------------------------------------------ softmax / correction / epilogue
-    const int row = warp * 32 + lane;  // query row inside the tile = tensor-memory lane
-    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-    const uint32_t ob = tmem + lane_addr + C::kColO;
+    Row t;
+    t.q = warp >> 2, t.warp = warp, t.lane = lane;
+    t.row = warp * 32 + lane;  // query row inside the unit; (warp & 3) * 32 + lane is its tensor-memory lane
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    t.ob = tmem + lane_addr + C::kColO + t.q * C::kOStride;
     bool ok = true;
     int n = 0, pc = 0;
     for (int it = it_begin; ok && it < it_end; ++pc) {
@@ -711,59 +774,52 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       it += p.cnt;
       float m_used = -INFINITY, l = 0.f;
       for (int j = 0; j < p.cnt; ++j, ++n) {
-        const uint32_t sb = tmem + lane_addr + C::kColS + (n & 1) * kBN;
-        if (!mbar_wait(&bar->s_full[n & 1], (n >> 1) & 1, dev_status, abort_flag)) { ok = false; break; }
+        const int b = n & 1;
+        const uint32_t sb = tmem + lane_addr + C::kColS + (2 * t.q + b) * kBN;
+        if (!mbar_wait(&bar->s_full[t.q][b], (n >> 1) & 1, dev_status, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const int valid = L - (p.k0 + j) * kBN;  // keys of this tile inside the sequence (>= 64: all)
-        uint64_t* pvb = &bar->v_empty[(n + C::kStages - 1) % C::kStages];  // barrier the previous tile's PV commits to
+        uint64_t* pvb = &bar->kv_empty[(n + C::kStages - 1) % C::kStages];  // barrier the previous tile's PV commits to
         const uint32_t pvp = (uint32_t)(((n - 1) / C::kStages) & 1);
-        if (valid >= kBN) ok = softmax_tile<DH, false>(sb, ob, scale_log2, kBN, j, m_used, l, pvb, pvp, dev_status, abort_flag);
-        else ok = softmax_tile_ragged<DH>(sb, ob, scale_log2, valid, j, m_used, l, pvb, pvp, dev_status, abort_flag);
+        if (valid >= kBN) ok = softmax_tile<DH, false>(sb, t.ob, scale_log2, kBN, j, m_used, l, pvb, pvp, dev_status, abort_flag);
+        else ok = softmax_tile_ragged<DH>(sb, t.ob, scale_log2, valid, j, m_used, l, pvb, pvp, dev_status, abort_flag);
         if (!ok) break;
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&bar->p_full[n & 1]);
+        if (lane == 0) mbar_arrive(&bar->p_full[t.q][b]);
       }
       if (!ok) break;
-      if (p.cnt == nblk) ok = finish_whole<DH>(ob, bar, p.u, pc, row, l, o, L, heads, dev_status);
-      else ok = finish_partial<DH>(ob, bar, p, pc, it >= it_end, row, m_used, l, o, L, heads, sp, tickets, pieces, dev_status);
+      if (p.cnt == nblk) ok = finish_whole<DH>(t, bar, p.u, pc, l, o, L, heads, dev_status);
+      else ok = finish_partial<DH>(t, bar, p, pc, it >= it_end, m_used, l, o, L, heads, sp, tickets, pieces, dev_status);
     }
-    if (ok) settle_first_piece<DH>(bar, it_begin, it_end, row, o, L, heads, sp, pieces, dev_status);
+    if (ok) settle_first_piece<DH>(bar, it_begin, it_end, t, o, L, heads, sp, pieces, dev_status);
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == 9) {
     tc_fence_after();
     tmem_dealloc(tmem, C::kTmemCols);
   }
 }
 
-constexpr int kMaxCtas = 320;  // scratch is sized for this many persistent CTAs
+constexpr int kMaxCtas = 160;  // scratch is sized for this many persistent CTAs
 
 size_t ticket_bytes(int B, int L, int heads) {
-  const size_t units = (size_t)B * heads * ((L + kBM - 1) / kBM);
-  return (units * 4 * sizeof(uint32_t) + 255) & ~(size_t)255;
+  const size_t units = (size_t)B * heads * ((L + kUM - 1) / kUM);
+  return (units * 8 * sizeof(uint32_t) + 255) & ~(size_t)255;
 }
 
 int max_ctas() {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v < 1)
-      v = 148;
-    sms = v;
-  }
-  int G = 2 * sms < kMaxCtas ? 2 * sms : kMaxCtas;
-  if (const char* e = getenv("TOMA_ATTENTION_CTAS")) {  // tuning aid
-    const int v = atoi(e);
-    if (v >= 1 && v <= kMaxCtas) G = v;
-  }
+  const int sms = sm_count();
+  int G = sms < kMaxCtas ? sms : kMaxCtas;
+  const int v = g_tune_attention_ctas.load(std::memory_order_relaxed);  // test-only override
+  if (v >= 1 && v <= kMaxCtas) G = v;
   return G;
 }
 
 // Key tiles a split costs a CTA, in units of one tile's time: writing, publishing and adding up the
 // partial results at the end of its span.
-constexpr int kSplitCostTiles = 5;
+constexpr int kSplitCostTiles = 4;
 
 // Whole units per CTA when that is at most kSplitCostTiles tiles slower than a perfectly even cut;
 // otherwise spans cut at single key tiles.
@@ -775,7 +831,8 @@ Spans plan_spans(int units, int nblk) {
   const int whole_tiles = ((units + gmax - 1) / gmax) * nblk;  // longest CTA with whole units
   const int even_tiles = (sp.T + gmax - 1) / gmax;             // longest CTA with an even cut
   int mode = whole_tiles <= even_tiles + kSplitCostTiles ? 0 : 1;
-  if (const char* e = getenv("TOMA_ATTENTION_SPLIT")) mode = atoi(e) != 0;  // tuning aid
+  const int forced = g_tune_attention_split.load(std::memory_order_relaxed);  // test-only override
+  if (forced == 0 || forced == 1) mode = forced;
   if (mode == 0) {
     sp.quantum = nblk;
     sp.G = units < gmax ? units : gmax;
@@ -800,25 +857,21 @@ cudaError_t launch(int B, int L, int heads, const void* q, const void* k, const 
   if (!encode_tmap_16bit(&tq, q, 3, dims, strides, box_q) || !encode_tmap_16bit(&tk, k, 3, dims, strides, box_kv) ||
       !encode_tmap_16bit(&tv, v, 3, dims, strides, box_kv))
     return cudaErrorInvalidValue;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
-  const long long units = (long long)B * heads * ((L + kBM - 1) / kBM);
+  static std::atomic<unsigned long long> smem_raised{0};
+  cudaError_t e = raise_dynamic_smem(attention_tc_kernel<DH>, C::kSmemBytes, smem_raised);
+  if (e != cudaSuccess) return e;
+  const long long units = (long long)B * heads * ((L + kUM - 1) / kUM);
   const int nblk = (L + kBN - 1) / kBN;
   if (units * nblk > 0x7fffffffLL) return cudaErrorInvalidValue;  // iteration indices are 32-bit
   const Spans sp = plan_spans((int)units, nblk);
   const size_t tb = ticket_bytes(B, L, heads);
   if (sp.quantum == 1 && !tickets_clean) {  // units are split: their tickets start at zero
-    cudaError_t e = cudaMemsetAsync(ws, 0, tb, s);
+    e = cudaMemsetAsync(ws, 0, tb, s);
     if (e != cudaSuccess) return e;
   }
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  cudaError_t e = launch_dependent(attention_tc_kernel<DH>, dim3(sp.G), dim3(256), (size_t)C::kSmemBytes, s, tq, tk, tv,
-                                   (__nv_bfloat16*)o, L, heads, scale_log2, sp, (uint32_t*)ws, (float*)((char*)ws + tb),
-                                   dev_status);
+  e = launch_dependent(attention_tc_kernel<DH>, dim3(sp.G), dim3(kThreads), (size_t)C::kSmemBytes, s, tq, tk, tv,
+                       (__nv_bfloat16*)o, L, heads, scale_log2, sp, (uint32_t*)ws, (float*)((char*)ws + tb), dev_status);
   if (e != cudaSuccess) return e;
   count_launch();
   return cudaGetLastError();
@@ -834,7 +887,7 @@ size_t attention_tc_workspace_bytes(int B, int L, int heads, int dh) {
 size_t attention_tc_ticket_bytes(int B, int L, int heads) { return ticket_bytes(B, L, heads); }
 
 int attention_tc_plan(int B, int L, int heads, int info[4], int* bounds, int* owner_first, int* owner_last, int capacity) {
-  const long long units = (long long)B * heads * ((L + kBM - 1) / kBM);
+  const long long units = (long long)B * heads * ((L + kUM - 1) / kUM);
   const int nblk = (L + kBN - 1) / kBN;
   if (units * nblk > 0x7fffffffLL) return 0;
   const Spans sp = plan_spans((int)units, nblk);

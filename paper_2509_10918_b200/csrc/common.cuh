@@ -45,6 +45,28 @@ Geom merge_geom(const Geom& g);
 extern std::atomic<unsigned long long> g_launches;
 inline void count_launch(int n = 1) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 
+// Test-only overrides of launch heuristics (set through toma_test_set_tuning; the product path never
+// writes them): attention work plan (-1 = heuristic, 0 = whole units, 1 = even cut), persistent CTA
+// count of the attention kernel (0 = heuristic), tile form of the projection kernel (0 = heuristic).
+extern std::atomic<int> g_tune_attention_split, g_tune_attention_ctas, g_tune_linear_tile;
+
+// Number of SMs of the current device (cached per device).
+int sm_count();
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize is a per-device attribute: `done` holds one bit per
+// device ordinal for which this kernel's limit has been raised (ordinals >= 64 are set every time).
+template <typename Kernel>
+cudaError_t raise_dynamic_smem(Kernel kernel, int bytes, std::atomic<unsigned long long>& done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 64 && ((done.load(std::memory_order_acquire) >> dev) & 1ull)) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  if (dev < 64) done.fetch_or(1ull << dev, std::memory_order_release);
+  return cudaSuccess;
+}
+
 // ---- launchers (each returns cudaGetLastError() of its launches) ----
 cudaError_t launch_quantise(const Geom& g, const void* x, __nv_bfloat16* y, cudaStream_t s);
 cudaError_t launch_gram_ffma(const Geom& g, const __nv_bfloat16* y, int16_t* sq, cudaStream_t s);

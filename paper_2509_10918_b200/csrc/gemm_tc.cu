@@ -185,8 +185,7 @@ cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* con
   // bytes per multiply-add (timed on eleven shapes from 4096 x 640 x 640 to 16384 x 8192 x 4096; the
   // model picks the faster form on each).  The 128 x 256 form keeps two CTAs per SM resident and is only
   // considered while its grid fits them.
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = sm_count();
   const int mb = (M + 127) / 128;
   const long long ctas320 = (long long)mb * ((N + 319) / 320) * n_mats, ctas256 = (long long)mb * ((N + 255) / 256) * n_mats;
   const long long ctas_pair = (long long)((M + 255) / 256) * ((N + 255) / 256) * n_mats;
@@ -195,10 +194,9 @@ cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* con
   const long long cost_pair = M > 128 ? ((ctas_pair + sms - 1) / sms) * (256 * 256) * 10 : cost320 + 1;
   int pair = cost_pair < cost320 && cost_pair < cost256;
   bool narrow = !pair && cost256 < cost320;
-  if (const char* e = getenv("TOMA_LINEAR_TILE")) {  // tuning aid: 256 x 256 (2), 128 x 320 (1) or 128 x 256 (0) tiles
-    const int v = atoi(e);
-    pair = v == 2 && M > 128;
-    narrow = v == 0;
+  if (const int v = g_tune_linear_tile.load(std::memory_order_relaxed)) {  // test-only override: 128 x 256 (1), 128 x 320 (2) or 256 x 256 (3) tiles
+    pair = v == 3 && M > 128;
+    narrow = v == 1;
   }
   const int cols = (narrow || pair) ? 256 : 320;
   const int slabs = ((N < cols ? N : cols) + 63) / 64;
@@ -208,13 +206,12 @@ cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* con
   const int nk = (K + kKC - 1) / kKC;
   if (stages > nk) stages = nk;
   const int smem = 1024 + stages * stage_bytes + 256;
-  static bool attr = false;
-  if (!attr) {
-    cudaError_t e = cudaFuncSetAttribute(linear_rows_kernel<320>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(linear_rows_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(linear_rows_kernel<256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  {
+    static std::atomic<unsigned long long> r320{0}, r256{0}, rpair{0};
+    cudaError_t e = raise_dynamic_smem(linear_rows_kernel<320>, 227 * 1024, r320);
+    if (e == cudaSuccess) e = raise_dynamic_smem(linear_rows_kernel<256>, 227 * 1024, r256);
+    if (e == cudaSuccess) e = raise_dynamic_smem(linear_rows_kernel<256, 2>, 227 * 1024, rpair);
     if (e != cudaSuccess) return e;
-    attr = true;
   }
   dim3 grid(pair ? (M + 255) / 256 : mb, (N + cols - 1) / cols, n_mats);
   cudaError_t e = pair ? launch_dependent(linear_rows_kernel<256, 2>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out,

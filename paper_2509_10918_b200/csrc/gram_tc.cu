@@ -141,12 +141,8 @@ cudaError_t launch_gram_tc(const Geom& g, const __nv_bfloat16* y, int16_t* sq, u
   if (!encode_tmap_16bit(&ta, y, 3, dims, strides, box_a) || !encode_tmap_16bit(&tb, y, 3, dims, strides, box_b))
     return cudaErrorInvalidValue;
   const int smem = 1024 + kStages * (128 * 128 + n_cols * 128) + 256;
-  static bool attr = false;
-  if (!attr) {
-    cudaError_t e = cudaFuncSetAttribute(gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e != cudaSuccess) return e;
-    attr = true;
-  }
+  static std::atomic<unsigned long long> smem_raised{0};
+  if (cudaError_t e = raise_dynamic_smem(gram_tc_kernel, 200 * 1024, smem_raised); e != cudaSuccess) return e;
   dim3 grid(g.B * g.P, (g.Nloc + 127) / 128, g.Nloc / n_cols);
   const cudaError_t le = launch_dependent(gram_tc_kernel, grid, dim3(192), (size_t)smem, s, ta, tb, sq, g.Nloc, g.d, n_cols, dev_status);
   count_launch();

@@ -399,13 +399,6 @@ bool encode_w(const Geom& g, const void* w, CUtensorMap* tm, uint32_t box_tokens
   return encode_tmap_16bit(tm, w, 3, dims, strides, box);
 }
 
-cudaError_t raise_smem_limit(const void* fn, bool* done) {
-  if (*done) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-  if (e == cudaSuccess) *done = true;
-  return e;
-}
-
 }  // namespace
 
 // Shapes the tensor-core merge / unmerge cover; everything else runs on the FFMA kernels.
@@ -433,8 +426,7 @@ cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* x
   // of 16 whose CTA count does not exceed the SM count (a few CTAs more would double the run time).
   p.dest_block = g.Dloc < kMaxCols ? g.Dloc : kMaxCols;
   if (g.Dloc > kMaxCols) {
-    int sms = 148, dev = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = sm_count();
     const int per_block = g.B * g.P * ((g.d + 127) / 128);  // CTAs per destination block
     for (int nb = (g.Dloc + kMaxCols - 1) / kMaxCols; nb * per_block <= sms; ++nb) {
       const int cand = (((g.Dloc + nb - 1) / nb) + 15) & ~15;
@@ -460,13 +452,13 @@ cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* x
   dim3 grid(g.B * g.P, (g.d + 127) / 128, (g.Dloc + p.dest_block - 1) / p.dest_block);
   cudaError_t e;
   if (g.Dloc > kMaxCols) {
-    static bool attr_b = false;
-    e = raise_smem_limit((const void*)merge_tc_kernel<true>, &attr_b);
+    static std::atomic<unsigned long long> raised_b{0};
+    e = raise_dynamic_smem(merge_tc_kernel<true>, 200 * 1024, raised_b);
     if (e != cudaSuccess) return e;
     e = launch_dependent(merge_tc_kernel<true>, grid, dim3(192), (size_t)smem, s, tx, tw, to, p, dev_status);
   } else {
-    static bool attr = false;
-    e = raise_smem_limit((const void*)merge_tc_kernel<false>, &attr);
+    static std::atomic<unsigned long long> raised{0};
+    e = raise_dynamic_smem(merge_tc_kernel<false>, 200 * 1024, raised);
     if (e != cudaSuccess) return e;
     e = launch_dependent(merge_tc_kernel<false>, grid, dim3(192), (size_t)smem, s, tx, tw, to, p, dev_status);
   }
@@ -486,8 +478,7 @@ cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void*
   LinParams p = make_params(g);
   // Tokens on M when a region has many destinations, and also when that form fits the SMs in one wave while
   // the channels-on-M grid would spill into a second one (64x64 tokens: 128 CTAs against 320 on 296 slots).
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = sm_count();
   const int rows_ctas = g.B * g.P * (g.Nloc / 128) * ((g.d + kRowsChBlock - 1) / kRowsChBlock);
   const int classic_ctas = g.B * g.P * ((g.d + 127) / 128) * (g.Nloc / n_tok);
   const bool one_wave = rows_ctas <= sms && classic_ctas > 2 * sms;
@@ -500,12 +491,8 @@ cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void*
     p.stages = p.stages > 4 ? 4 : p.stages < 2 ? 2 : p.stages;
     if (p.stages > (g.Dloc + kKC - 1) / kKC) p.stages = (g.Dloc + kKC - 1) / kKC;
     const int smem = 1024 + p.stages * stage_bytes + 256;
-    static bool attr_r = false;
-    if (!attr_r) {
-      cudaError_t e = cudaFuncSetAttribute(unmerge_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-      if (e != cudaSuccess) return e;
-      attr_r = true;
-    }
+    static std::atomic<unsigned long long> raised_r{0};
+    if (cudaError_t e = raise_dynamic_smem(unmerge_rows_kernel, 227 * 1024, raised_r); e != cudaSuccess) return e;
     dim3 grid(g.B * g.P * (g.Nloc / 128), (g.d + kRowsChBlock - 1) / kRowsChBlock);
     cudaError_t e = launch_dependent(unmerge_rows_kernel, grid, dim3(192), (size_t)smem, s, ty, tw128, (__nv_bfloat16*)out, p,
                                      dev_status);
@@ -522,8 +509,8 @@ cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void*
   p.stages = 2;
   if (p.stages > (g.Dloc + kKC - 1) / kKC) p.stages = (g.Dloc + kKC - 1) / kKC;
   const int smem = 1024 + p.stages * stage_bytes + 256;
-  static bool attr = false;
-  cudaError_t e = raise_smem_limit((const void*)unmerge_tc_kernel, &attr);
+  static std::atomic<unsigned long long> raised{0};
+  cudaError_t e = raise_dynamic_smem(unmerge_tc_kernel, 200 * 1024, raised);
   if (e != cudaSuccess) return e;
   dim3 grid(g.B * g.P, (g.d + 127) / 128, g.Nloc / n_tok);
   e = launch_dependent(unmerge_tc_kernel, grid, dim3(192), (size_t)smem, s, ty, tw, to, p, n_tok, dev_status);

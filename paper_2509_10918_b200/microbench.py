@@ -68,7 +68,7 @@ def main():
     idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     B, N, d = cfg.batch, cfg.n_tokens + cfg.n_extra, cfg.dim
-    Lm = cfg.n_merged + cfg.n_extra
+    Lm = (cfg.n_tiles * toma.toma_dest_per_tile(desc)) + cfg.n_extra
     xm = torch.empty((B, Lm, d), dtype=tdt, device="cuda")
     att = torch.empty_like(xm)
     toma.toma_select(desc, x, idx, ws, status)
@@ -112,10 +112,10 @@ def main():
         res.update(length=L, tflops_median=flops / med / 1e6, tflops_best=flops / mn / 1e6)
     elif args.stage in ("merge", "unmerge"):
         wbytes = 4 if cfg.dtype == "bf16" else 4
-        nbytes = B * (cfg.n_tokens * d * esz + cfg.n_merged * d * esz + cfg.n_tiles * cfg.n_loc * cfg.d_loc * wbytes)
+        nbytes = B * (cfg.n_tokens * d * esz + (cfg.n_tiles * toma.toma_dest_per_tile(desc)) * d * esz + cfg.n_tiles * cfg.n_loc * toma.toma_dest_per_tile(desc) * wbytes)
         res.update(algorithmic_bytes=nbytes, gbs_median=nbytes / med / 1e3, gbs_best=nbytes / mn / 1e3)
     elif args.stage == "select":
-        res.update(tiles=B * cfg.n_tiles, rounds=cfg.d_loc, us_per_round=med / cfg.d_loc)
+        res.update(tiles=B * cfg.n_tiles, rounds=toma.toma_dest_per_tile(desc), us_per_round=med / toma.toma_dest_per_tile(desc))
     print(json.dumps(res))
 
 

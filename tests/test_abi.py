@@ -108,17 +108,17 @@ def test_binding_refuses_cpu_tensors(toma):
 @pytest.mark.parametrize("split", ["0", "1", None])
 @pytest.mark.parametrize("shape", [(2, 2048, 10, 64), (1, 2560, 24, 128), (2, 1000, 3, 64), (1, 77, 2, 128),
                                    (4, 8192, 10, 64), (1, 300, 3, 64), (3, 4096, 7, 64)])
-def test_attention_work_plan_covers_every_key_tile_once(toma, monkeypatch, shape, split):
+def test_attention_work_plan_covers_every_key_tile_once(toma, shape, split):
     """Host logic of the attention kernel's work plan (no GPU needed): the spans tile the iteration space
     [0, units * tiles_per_unit) without gap or overlap, differ by at most one quantum, keep units whole
     when the plan says so, and the kernel's own owner arithmetic maps each span's ends back to its CTA."""
-    if split is None:
-        monkeypatch.delenv("TOMA_ATTENTION_SPLIT", raising=False)
-    else:
-        monkeypatch.setenv("TOMA_ATTENTION_SPLIT", split)
     B, L, h, dh = shape
-    plan = toma.toma_attention_plan(B, L, h, dh, "bf16")
-    units, nblk = B * h * ((L + 127) // 128), (L + 63) // 64
+    toma.toma_test_set_tuning(attention_split=-1 if split is None else int(split))
+    try:
+        plan = toma.toma_attention_plan(B, L, h, dh, "bf16")
+    finally:
+        toma.toma_test_set_tuning()
+    units, nblk = B * h * ((L + 255) // 256), (L + 63) // 64
     assert plan["units"] == units and plan["tiles_per_unit"] == nblk
     b = plan["bounds"]
     assert len(b) == plan["ctas"] + 1 and b[0] == 0 and b[-1] == units * nblk

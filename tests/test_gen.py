@@ -24,15 +24,13 @@ def test_normal_stream_is_counter_based_and_standard():
 
 
 def test_configs_shapes_and_locality():
-    expect = {"cfg1": (1, 1024, 640, 16, 64, 32), "cfg2": (2, 1024, 1280, 16, 64, 32),
-              "cfg3": (2, 4096, 640, 16, 256, 128), "cfg4": (1, 4096, 3072, 16, 256, 128),
-              "cfg5a": (4, 16384, 640, 64, 256, 128), "cfg5b": (4, 16384, 640, 16, 1024, 512)}
-    for name, (b, n, d, p, nl, dl) in expect.items():
+    expect = {"cfg1": (1, 1024, 640, 16, 64), "cfg2": (2, 1024, 1280, 16, 64),
+              "cfg3": (2, 4096, 640, 16, 256), "cfg4": (1, 4096, 3072, 16, 256),
+              "cfg5a": (4, 16384, 640, 64, 256), "cfg5b": (4, 16384, 640, 16, 1024)}
+    for name, (b, n, d, p, nl) in expect.items():
         c = gen.config(name)
-        assert (c.batch, c.n_tokens, c.dim, c.n_tiles, c.n_loc, c.d_loc) == (b, n, d, p, nl, dl)
+        assert (c.batch, c.n_tokens, c.dim, c.n_tiles, c.n_loc) == (b, n, d, p, nl)
         assert c.n_heads * c.head_dim == c.dim
-    c3 = gen.config("cfg3")
-    assert [c3.with_(merge_ratio=r).d_loc for r in (0.25, 0.5, 0.75)] == [192, 128, 64]
     c = gen.config("cfg2")
     x = gen.features(c)
     assert x.shape == (2, 1024, 1280) and x.dtype == np.float32

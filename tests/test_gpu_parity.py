@@ -22,6 +22,23 @@ def toma():
     return t
 
 
+@pytest.fixture
+def tuning(toma):
+    """Forces a launch configuration through the library's test-only setter; the heuristics come back afterwards."""
+    yield toma.toma_test_set_tuning
+    toma.toma_test_set_tuning()
+
+
+def od(cfg):
+    """Destinations per tile as the oracle counts them."""
+    return O.dest_count(cfg.n_loc, cfg.merge_ratio)
+
+
+def gd(toma, cfg):
+    """Destinations per tile as the library counts them (sizes of the device buffers)."""
+    return toma.toma_dest_per_tile(toma.desc_from_config(cfg))
+
+
 class Run:
     """Device buffers of one configuration plus the entry points bound to them."""
 
@@ -33,7 +50,8 @@ class Run:
         self.w = toma.alloc_weights(self.desc)
         self.ws = toma.alloc_workspace(self.desc)
         self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
-        self.lm = cfg.n_merged + cfg.n_extra
+        self.d_loc = toma.toma_dest_per_tile(self.desc)
+        self.lm = cfg.n_tiles * self.d_loc + cfg.n_extra
         self.xm = torch.empty((cfg.batch, self.lm, cfg.dim), dtype=self.x.dtype, device="cuda")
 
     def ok(self):
@@ -49,7 +67,7 @@ class Run:
         self.t.toma_merge_weights(self.desc, self.x, self.idx, self.w, self.ws, self.status)
         self.ok()
         c = self.cfg
-        dense = torch.empty((c.batch, c.n_tiles, c.d_loc, c.n_loc), dtype=torch.float32, device="cuda")
+        dense = torch.empty((c.batch, c.n_tiles, self.d_loc, c.n_loc), dtype=torch.float32, device="cuda")
         self.t.toma_weights_export(self.desc, self.w, dense)
         torch.cuda.synchronize()
         return dense.cpu().numpy().astype(np.float64)
@@ -108,7 +126,7 @@ def test_select_weights_merge_unmerge_parity(toma, name, over, n_check):
     y_dev = run.attend()
     unmerged = run.unmerge(y_dev)
     y_host = to_host64(y_dev)
-    D = cfg.n_merged
+    D = cfg.n_tiles * gd(toma, cfg)
     if cfg.n_extra:
         assert np.array_equal(merged[:, D:], x_host[:, cfg.n_tokens:].astype(np.float64))
         assert np.array_equal(unmerged[:, cfg.n_tokens:], y_host[:, D:])
@@ -118,15 +136,15 @@ def test_select_weights_merge_unmerge_parity(toma, name, over, n_check):
     got_m, want_m, got_u, want_u = [], [], [], []
     for b, p in sample_tiles(cfg, n_check):
         xt = tile_tokens(cfg, x_host, b, p)
-        want_idx, margin = O.select_tile(xt, cfg.d_loc)
+        want_idx, margin = O.select_tile(xt, od(cfg))
         assert margin > O.FRAGILE_MARGIN, "input sits on a quantisation boundary; choose another seed"
         assert np.array_equal(idx[b, p], want_idx), f"selection differs in tile ({b},{p})"
         w = O.merge_weights(xt, want_idx, cfg.tau)
         assert np.abs(dense[b, p] - w).max() <= w_abs, f"weights differ in tile ({b},{p})"
-        got_m.append(merged[b, p * cfg.d_loc:(p + 1) * cfg.d_loc])
+        got_m.append(merged[b, p * gd(toma, cfg):(p + 1) * gd(toma, cfg)])
         want_m.append(O.merge(w, xt))
         got_u.append(unmerged[b, ids[p]])
-        want_u.append(O.unmerge(w, y_host[b, p * cfg.d_loc:(p + 1) * cfg.d_loc]))
+        want_u.append(O.unmerge(w, y_host[b, p * gd(toma, cfg):(p + 1) * gd(toma, cfg)]))
     assert_close(np.stack(got_m), np.stack(want_m), cfg.dtype, "merge")
     assert_close(np.stack(got_u), np.stack(want_u), cfg.dtype, "unmerge")
 
@@ -169,11 +187,10 @@ def test_attention_parity(toma, dtype, B, L, h, dh, n_rows):
     ("0", "5", 1, 1000, 3, 64),     # whole units, several per CTA
     ("0", "320", 1, 300, 3, 128),   # whole units, fewer units than CTAs
 ])
-def test_attention_span_plans(toma, monkeypatch, split, ctas, B, L, h, dh):
-    """The tensor-core kernel under forced work plans (the tuning knobs TOMA_ATTENTION_SPLIT and
-    TOMA_ATTENTION_CTAS): every way a unit's keys can be cut across CTAs gives the same result."""
-    monkeypatch.setenv("TOMA_ATTENTION_SPLIT", split)
-    monkeypatch.setenv("TOMA_ATTENTION_CTAS", ctas)
+def test_attention_span_plans(toma, tuning, split, ctas, B, L, h, dh):
+    """The tensor-core kernel under forced work plans (toma_test_set_tuning): every way a unit's keys can
+    be cut across CTAs gives the same result."""
+    tuning(attention_split=int(split), attention_ctas=int(ctas))
     host = [gen.round_to_dtype(gen.normal(0, (78, L + dh, i), B * L * h * dh).reshape(B, L, h * dh).astype(np.float32),
                                "bf16") for i in range(3)]
     q, k, v = (to_dev(a, "bf16") for a in host)
@@ -313,7 +330,7 @@ def test_global_merge_parity(toma, over):
     x_host = gen.features(cfg)
     run = Run(toma, cfg, x_host, global_merge=True)
     idx = run.select()
-    N, D = cfg.n_tokens, cfg.n_merged
+    N, D = cfg.n_tokens, cfg.n_tiles * gd(toma, cfg)
     run.t.toma_merge_weights(run.desc, run.x, run.idx, run.w, run.ws, run.status)
     run.ok()
     dense = torch.empty((cfg.batch, 1, D, N), dtype=torch.float32, device="cuda")
@@ -328,7 +345,7 @@ def test_global_merge_parity(toma, over):
     w_abs = 2e-5 if cfg.dtype == "f32" else 6e-4
     for b in range(cfg.batch):
         for p in range(cfg.n_tiles):
-            want_idx, margin = O.select_tile(tile_tokens(cfg, x_host, b, p), cfg.d_loc)
+            want_idx, margin = O.select_tile(tile_tokens(cfg, x_host, b, p), od(cfg))
             assert margin > O.FRAGILE_MARGIN
             assert np.array_equal(idx[b, p], want_idx)
         x_img = x_host[b, :N].astype(np.float64)
@@ -385,8 +402,8 @@ def test_shares_unmerge_parity(toma, name, over, global_merge):
     assert toma.toma_weights_bytes(run.desc) == 2 * toma.toma_weights_bytes(ref.desc)
     idx = run.select()
     ref.idx.copy_(run.idx)
-    N, D = cfg.n_tokens, cfg.n_merged
-    shape = (cfg.batch, 1, D, N) if global_merge else (cfg.batch, cfg.n_tiles, cfg.d_loc, cfg.n_loc)
+    N, D = cfg.n_tokens, cfg.n_tiles * gd(toma, cfg)
+    shape = (cfg.batch, 1, D, N) if global_merge else (cfg.batch, cfg.n_tiles, gd(toma, cfg), cfg.n_loc)
     for r in (run, ref):
         r.t.toma_merge_weights(r.desc, r.x, r.idx, r.w, r.ws, r.status)
         r.ok()
@@ -425,7 +442,7 @@ def test_shares_unmerge_parity(toma, name, over, global_merge):
             want = O.softmax_shares(xt, idx[b, p], cfg.tau)
             assert np.abs(A[b, p] - want).max() <= w_abs, f"shares differ in tile ({b},{p})"
             got.append(unmerged[b, ids[p]])
-            want_u.append(O.unmerge(want, y_host[b, p * cfg.d_loc:(p + 1) * cfg.d_loc]))
+            want_u.append(O.unmerge(want, y_host[b, p * gd(toma, cfg):(p + 1) * gd(toma, cfg)]))
         assert_close(np.stack(got), np.stack(want_u), cfg.dtype, "shares unmerge")
     if cfg.n_extra:
         assert np.array_equal(unmerged[:, N:], y_host[:, D:])
@@ -474,11 +491,11 @@ def test_linear_parity(toma, dtype, m, n, k):
 
 @pytest.mark.parametrize("tile", [0, 1, 2], ids=["128x256", "128x320", "256x256"])
 @pytest.mark.parametrize("m,n,k", [(300, 328, 200), (129, 1920, 640), (1024, 72, 136), (640, 512, 64)])
-def test_linear_every_tile_form(toma, monkeypatch, tile, m, n, k):
+def test_linear_every_tile_form(toma, tuning, tile, m, n, k):
     """Each of the projection kernel's three tile forms, forced, on shapes with a ragged last row block (the
     second row block of a 256-row tile partly or wholly past the end), partial column blocks and a partial
     last k-step."""
-    monkeypatch.setenv("TOMA_LINEAR_TILE", str(tile))
+    tuning(linear_tile=tile + 1)
     a_host = gen.round_to_dtype(gen.normal(0, (191, m, k), m * k).reshape(m, k).astype(np.float32), "bf16")
     w_host = gen.round_to_dtype((gen.normal(0, (192, n, k), k * n).reshape(k, n) / np.sqrt(k)).astype(np.float32), "bf16")
     a, w = to_dev(a_host, "bf16"), to_dev(w_host, "bf16")
@@ -684,7 +701,7 @@ def test_block_long_sequence_schedule_and_sampled_parity(toma):
         cur = idx.cpu().numpy().astype(np.int64)
         if step % cfg.reuse_interval == 0:
             for b, p in tiles:
-                want, margin = O.select_tile(tile_tokens(cfg, x_host, b, p), cfg.d_loc)
+                want, margin = O.select_tile(tile_tokens(cfg, x_host, b, p), od(cfg))
                 assert margin > O.FRAGILE_MARGIN
                 assert np.array_equal(cur[b, p], want)
         else:
@@ -696,7 +713,7 @@ def test_block_long_sequence_schedule_and_sampled_parity(toma):
 def test_identity_weights_round_trip_is_bit_exact(toma):
     for dtype in ("bf16", "f32"):
         cfg = gen.config("cfg2", batch=1, grid_h=16, grid_w=16, dim=128, n_heads=2, merge_ratio=0.0, dtype=dtype)
-        assert cfg.d_loc == cfg.n_loc
+        assert gd(toma, cfg) == cfg.n_loc
         x_host = gen.features(cfg)
         run = Run(toma, cfg, x_host)
         eye = torch.eye(cfg.n_loc, dtype=torch.float32, device="cuda").repeat(cfg.batch, cfg.n_tiles, 1, 1).contiguous()
@@ -739,12 +756,12 @@ def test_edge_shapes(toma, over, dtype):
     for b in range(cfg.batch):
         for p in range(cfg.n_tiles):
             xt = tile_tokens(cfg, x_host, b, p)
-            want_idx, margin = O.select_tile(xt, cfg.d_loc)
+            want_idx, margin = O.select_tile(xt, od(cfg))
             assert margin > O.FRAGILE_MARGIN
             assert np.array_equal(idx[b, p], want_idx)
             w = O.merge_weights(xt, want_idx, cfg.tau)
             assert np.abs(dense[b, p] - w).max() <= (2e-5 if dtype == "f32" else 6e-4)
-            sl = slice(p * cfg.d_loc, (p + 1) * cfg.d_loc)
+            sl = slice(p * gd(toma, cfg), (p + 1) * gd(toma, cfg))
             assert_close(merged[b, sl], O.merge(w, xt), dtype, "merge")
             assert_close(unmerged[b, ids[p]], O.unmerge(w, y_host[b, sl]), dtype, "unmerge")
 
@@ -760,7 +777,7 @@ def test_degenerate_inputs_identical_and_zero_tokens(toma):
     idx = run.select()
     assert list(idx[0, 0]) == list(range(32))                              # ties resolve to the lowest index
     for p in range(2):
-        want, _ = O.select_tile(tile_tokens(cfg, x_host, 0, p), cfg.d_loc)
+        want, _ = O.select_tile(tile_tokens(cfg, x_host, 0, p), od(cfg))
         assert np.array_equal(idx[0, p], want)
 
 

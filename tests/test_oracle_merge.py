@@ -28,12 +28,12 @@ def test_weight_invariants_on_a_real_tile():
     c = gen.config("cfg2", batch=1)
     x = gen.features(c)[0]
     tile = O.split_regions(x, c.grid_h, c.grid_w, c.tile_h, c.tile_w)[7]
-    idx, _ = O.select_tile(tile, c.d_loc)
+    idx, _ = O.select_tile(tile, O.dest_count(c.n_loc, c.merge_ratio))
     w = O.merge_weights(tile, idx, c.tau)
-    assert w.shape == (c.d_loc, c.n_loc)
+    assert w.shape == (O.dest_count(c.n_loc, c.merge_ratio), c.n_loc)
     assert np.all(w >= 0)
     assert np.allclose(w.sum(axis=1), 1.0, atol=1e-12)          # merge rows sum to 1
-    Z = 1.0 / w[np.arange(c.d_loc), idx]                          # not used further; rows are positive
+    Z = 1.0 / w[np.arange(O.dest_count(c.n_loc, c.merge_ratio)), idx]                          # not used further; rows are positive
     assert np.all(np.isfinite(Z))
     # before row normalisation every source's shares sum to 1: recover A = w * Z_row
     xs = tile.astype(np.float64)
@@ -195,7 +195,7 @@ def test_softmax_shares_closed_form_and_relation_to_merge_weights():
     assert A[:, 0] == pytest.approx([e / (e + 1), 1 / (e + 1)])  # destination 0 against itself and against 1
     c = gen.config("cfg2", batch=1)
     tile = O.split_regions(gen.features(c)[0], c.grid_h, c.grid_w, c.tile_h, c.tile_w)[3]
-    idx, _ = O.select_tile(tile, c.d_loc)
+    idx, _ = O.select_tile(tile, O.dest_count(c.n_loc, c.merge_ratio))
     A = O.softmax_shares(tile, idx, c.tau)
     w = O.merge_weights(tile, idx, c.tau)
     assert np.all(A >= 0) and np.allclose(A.sum(axis=0), 1.0, atol=1e-12)
@@ -208,13 +208,13 @@ def test_shares_unmerge_is_a_partition_of_unity_and_beats_the_transpose_on_round
     range, and unmerge(merge(x)) is closer to x than with A~^T, whose columns sum to about D/N."""
     c = gen.config("cfg2", batch=1)
     tile = O.split_regions(gen.features(c)[0], c.grid_h, c.grid_w, c.tile_h, c.tile_w)[5].astype(np.float64)
-    idx, _ = O.select_tile(tile, c.d_loc)
+    idx, _ = O.select_tile(tile, O.dest_count(c.n_loc, c.merge_ratio))
     A = O.softmax_shares(tile, idx, c.tau)
     w = O.merge_weights(tile, idx, c.tau)
-    const = np.full((c.d_loc, 7), 2.5)
+    const = np.full((O.dest_count(c.n_loc, c.merge_ratio), 7), 2.5)
     assert np.allclose(O.unmerge(A, const), 2.5, atol=1e-12)
     assert not np.allclose(O.unmerge(w, const), 2.5, atol=0.1)   # the transpose attenuates
-    y = np.random.default_rng(3).normal(size=(c.d_loc, 5))
+    y = np.random.default_rng(3).normal(size=(O.dest_count(c.n_loc, c.merge_ratio), 5))
     un = O.unmerge(A, y)
     assert np.all(un <= y.max(axis=0) + 1e-12) and np.all(un >= y.min(axis=0) - 1e-12)
     merged = O.merge(w, tile)
@@ -223,7 +223,7 @@ def test_shares_unmerge_is_a_partition_of_unity_and_beats_the_transpose_on_round
     assert err_s < err_t
     # explicit loops: out_k = sum_i A_ik y_i
     k = 11
-    assert np.allclose(un[k], sum(A[i, k] * y[i] for i in range(c.d_loc)), atol=1e-12)
+    assert np.allclose(un[k], sum(A[i, k] * y[i] for i in range(O.dest_count(c.n_loc, c.merge_ratio))), atol=1e-12)
 
 
 def test_shares_unmerge_on_orthogonal_groups_copies_the_prototype_output():
@@ -251,7 +251,7 @@ def test_block_step_unmerge_modes_differ_only_in_the_unmerge():
     assert np.array_equal(merged_t, merged_s) and np.array_equal(att_t, att_s)
     assert np.array_equal(st_t.w, st_s.w) and np.array_equal(st_t.idx, st_s.idx)
     ids = O.tile_token_ids(16, 16, c.tile_h, c.tile_w)
-    d_loc = c.d_loc
+    d_loc = O.dest_count(c.n_loc, c.merge_ratio)
     p = 2
     want = st_s.u[0, p].T @ att_s[0, p * d_loc:(p + 1) * d_loc]
     assert np.allclose(out_s[0, ids[p]], want, atol=1e-12)

@@ -169,12 +169,12 @@ def test_fixed_point_selection_is_faithful_to_fp64_cosine_greedy():
     x = gen.features(c)[0]
     tiles = O.split_regions(x, c.grid_h, c.grid_w, c.tile_h, c.tile_w)
     for p in (0, 5, 10):
-        a, _ = O.select_tile(tiles[p], c.d_loc)
-        b = O.select_tile_definition(tiles[p], c.d_loc)
+        a, _ = O.select_tile(tiles[p], O.dest_count(c.n_loc, c.merge_ratio))
+        b = O.select_tile_definition(tiles[p], O.dest_count(c.n_loc, c.merge_ratio))
         cos = O.cosine_similarity(tiles[p])
         ratio = O.facility_location(cos, a) / O.facility_location(cos, b)
         assert ratio > 0.995
-        assert len(set(a) & set(b)) >= 0.8 * c.d_loc
+        assert len(set(a) & set(b)) >= 0.8 * O.dest_count(c.n_loc, c.merge_ratio)
 
 
 def test_region_split_tiles_and_stripes():
