@@ -82,7 +82,7 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
   volatile int* abort_flag = &bar->abort_flag;
 
   if (warp == 0) {
-    if (lane == 0) {
+    if (elect_one()) {
       for (int k = 0; k < nk; ++k) {
         const int s = k % stages;
         if (k >= stages && !mbar_wait(&bar->empty[s], ((k / stages) - 1) & 1, dev_status, abort_flag)) break;
@@ -94,7 +94,7 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (elect_one()) {
       const uint32_t idesc_a = idesc_f16(kFmtBF16, kFmtBF16, false, true, 128, n_a);
       const uint32_t idesc_b = idesc_f16(kFmtBF16, kFmtBF16, false, true, 128, n_b > 0 ? n_b : 64);
       bool ok = true;

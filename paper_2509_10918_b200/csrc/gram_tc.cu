@@ -57,7 +57,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   volatile int* abort_flag = &bar->abort_flag;
 
   if (warp == 0) {
-    if (lane == 0) {
+    if (elect_one()) {
       for (int k = 0; k < nk; ++k) {
         const int s = k % kStages;
         if (k >= kStages && !mbar_wait(&bar->empty[s], ((k / kStages) - 1) & 1, dev_status, abort_flag)) break;
@@ -68,7 +68,7 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (elect_one()) {
       const uint32_t idesc = idesc_f16(kFmtBF16, kFmtBF16, false, false, 128, n_cols);
       bool ok = true;
       for (int k = 0; k < nk; ++k) {

@@ -129,7 +129,7 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
   volatile int* abort_flag = &bar->abort_flag;
 
   if (warp == 0) {
-    if (lane == 0) {
+    if (elect_one()) {
       for (int k = 0; k < nk; ++k) {
         const int s = k % p.stages;
         if (k >= p.stages && !mbar_wait(&bar->empty[s], ((k / p.stages) - 1) & 1, dev_status, abort_flag)) break;
@@ -144,7 +144,7 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (elect_one()) {
       const uint32_t idesc = idesc_f16(kFmtBF16, kFmtBF16, true, true, 128, n_mma);
       bool ok = true;
       for (int k = 0; k < nk; ++k) {
@@ -214,7 +214,7 @@ unmerge_tc_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constan
   volatile int* abort_flag = &bar->abort_flag;
 
   if (warp == 0) {
-    if (lane == 0) {
+    if (elect_one()) {
       for (int k = 0; k < nk; ++k) {
         const int s = k % p.stages;
         if (k >= p.stages && !mbar_wait(&bar->empty[s], ((k / p.stages) - 1) & 1, dev_status, abort_flag)) break;
@@ -227,7 +227,7 @@ unmerge_tc_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constan
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (elect_one()) {
       const uint32_t idesc = idesc_f16(kFmtBF16, kFmtBF16, true, false, 128, n_tok);
       bool ok = true;
       for (int k = 0; k < nk; ++k) {
@@ -314,7 +314,7 @@ unmerge_rows_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_const
   volatile int* abort_flag = &bar->abort_flag;
 
   if (warp == 0) {
-    if (lane == 0) {
+    if (elect_one()) {
       for (int k = 0; k < nk; ++k) {
         const int s = k % p.stages;
         if (k >= p.stages && !mbar_wait(&bar->empty[s], ((k / p.stages) - 1) & 1, dev_status, abort_flag)) break;
@@ -327,7 +327,7 @@ unmerge_rows_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_const
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (elect_one()) {
       const uint32_t idesc_a = idesc_f16(kFmtBF16, kFmtBF16, false, true, 128, n_a);
       const uint32_t idesc_b = idesc_f16(kFmtBF16, kFmtBF16, false, true, 128, n_b > 0 ? n_b : 64);
       bool ok = true;

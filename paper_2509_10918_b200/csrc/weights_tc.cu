@@ -104,7 +104,7 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
   volatile int* abort_flag = &bar->abort_flag;
 
   if (warp == 0) {
-    if (lane == 0) {
+    if (elect_one()) {
       for (int k = 0; k < nk; ++k) {
         const int s = k % p.stages;
         if (k >= p.stages && !mbar_wait(&bar->empty[s], ((k / p.stages) - 1) & 1, dev_status, abort_flag)) break;
@@ -116,7 +116,7 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (elect_one()) {
       const uint32_t idesc0 = idesc_f16(kFmtBF16, kFmtBF16, false, false, 128, n0);
       const uint32_t idesc1 = idesc_f16(kFmtBF16, kFmtBF16, false, false, 128, n1 > 0 ? n1 : 16);
       bool ok = true;
