@@ -112,6 +112,13 @@ TOMA_API uint64_t toma_launch_counter(void);
  *   attention_ctas : > 0 = number of persistent CTAs (clamped to the scratch capacity), else heuristic
  *   linear_tile    : 1 = 128 x 256, 2 = 128 x 320, 3 = 256 x 256 tiles, else heuristic */
 TOMA_API void toma_test_set_tuning(int32_t attention_split, int32_t attention_ctas, int32_t linear_tile);
+/* TEST-ONLY (no counterpart in the paper): launches one CTA that waits, with the library's bounded wait and
+ * a limit of `polls` polls (1..100000), on a barrier that nobody signals.  The wait gives up, ORs
+ * TOMA_ERR_TIMEOUT's bit (bit 0) into *dev_status (device, may be NULL), writes 2 to *outcome (device, may be
+ * NULL; 1 would mean the wait completed) and the kernel returns: nothing traps, faults or spins without
+ * limit, and the context stays usable.  This is the path every device-side wait of the library takes when
+ * its producer never comes. */
+TOMA_API toma_status toma_test_wait_timeout(uint32_t polls, uint32_t* dev_status, uint32_t* outcome, void* stream);
 
 /* Destination selection (Sec. 4.1, Algorithm 2) inside every tile.
  *   x   [batch][N + n_extra][dim]  in
@@ -131,14 +138,17 @@ TOMA_API toma_status toma_select(const toma_desc* desc, const void* x, int32_t* 
  * synchronises the device, is illegal during stream capture and sidesteps the host's memory pool.
  * Same inputs, outputs and results as toma_select; the scratch is a static device array of
  * TOMA_STATIC_SCRATCH_BYTES inside the library, so:
- *   - it occupies that much memory on every GPU that loads the library, until process exit;
+ *   - a GPU holds that much memory from the moment the library's device code is loaded on it (with the
+ *     CUDA runtime's default lazy loading: from the first toma_select_static call on that GPU) until
+ *     process exit;
  *   - a problem whose scratch, batch*P*N_loc*(dim + N_loc)*2 bytes plus padding, exceeds it is
  *     refused with TOMA_ERR_SCRATCH_LIMIT before any launch;
  *   - all calls on a device share it and it keeps the previous call's contents (nothing needs
  *     zeroing: every byte read is written earlier in the same call); calls that can overlap on
  *     the GPU race on it, so the caller must serialise them;
- *   - the first call on each device resolves the array's device address; make that call before
- *     starting any stream capture.
+ *   - the first call on each device resolves the array's device address, which is also where the
+ *     memory is reserved: it returns TOMA_ERR_CUDA (nothing launched, no sticky error left) if the
+ *     device has none left; make that call before starting any stream capture.
  * The call never allocates or frees memory. */
 TOMA_API toma_status toma_select_static(const toma_desc* desc, const void* x, int32_t* idx, uint32_t* dev_status,
                                         void* stream);

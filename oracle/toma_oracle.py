@@ -127,6 +127,16 @@ def quantise_tokens(x: np.ndarray) -> Tuple[np.ndarray, float]:
     return _round_to_8_significant_bits(k), margin
 
 
+def round_gram(K: np.ndarray) -> np.ndarray:
+    """rint(K / 4096) with ties to even, in integer arithmetic: the step that turns the exact integer
+    Gram entries K_ij (units of 2^-24) into the similarities S_q (units of 2^-12)."""
+    K = np.asarray(K, dtype=np.int64)
+    q = K >> 12            # floor(K / 4096)
+    rem = K - (q << 12)    # in [0, 4096)
+    up = (rem > 2048) | ((rem == 2048) & ((q & 1) == 1))
+    return (q + up).astype(np.int32)
+
+
 def pinned_similarity(x: np.ndarray) -> Tuple[np.ndarray, float]:
     """int32 [n, n] fixed-point cosine similarity S_q (units of 2^-12) of one
     region, plus the quantisation margin (see quantise_tokens)."""
@@ -134,10 +144,7 @@ def pinned_similarity(x: np.ndarray) -> Tuple[np.ndarray, float]:
     K = k @ k.T  # exact in int64
     if np.abs(K).max(initial=0) >= (1 << 24):
         raise ValueError("Gram entry does not fit 24 bits; input outside the supported range")
-    q = K >> 12            # floor(K / 4096)
-    rem = K - (q << 12)    # in [0, 4096)
-    up = (rem > 2048) | ((rem == 2048) & ((q & 1) == 1))
-    S = (q + up).astype(np.int32)
+    S = round_gram(K)
     np.fill_diagonal(S, DIAG_Q)
     return S, margin
 

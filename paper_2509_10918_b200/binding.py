@@ -19,7 +19,7 @@ TOMA_BF16, TOMA_F32 = 0, 1
 STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_RATIO", "ERR_TAU", "ERR_WORKSPACE",
                 "ERR_UNSUPPORTED", "ERR_CUDA", "ERR_TIMEOUT", "ERR_SCRATCH_LIMIT"]
 
-EXPORTS = ["toma_select_static", "toma_launch_counter", "toma_test_set_tuning", "toma_workspace_bytes", "toma_weights_bytes", "toma_dest_per_tile", "toma_validate", "toma_status_str",
+EXPORTS = ["toma_select_static", "toma_launch_counter", "toma_test_set_tuning", "toma_test_wait_timeout", "toma_workspace_bytes", "toma_weights_bytes", "toma_dest_per_tile", "toma_validate", "toma_status_str",
            "toma_select", "toma_merge_weights", "toma_merge", "toma_attention_workspace_bytes", "toma_attention_plan", "toma_attention",
            "toma_unmerge", "toma_block", "toma_block_host", "toma_linear", "toma_block_proj", "toma_attention_proj_workspace_bytes",
            "toma_attention_proj", "toma_block_mlp", "toma_mlp_workspace_bytes", "toma_mlp",
@@ -63,6 +63,8 @@ def _load() -> ctypes.CDLL:
     lib.toma_launch_counter.argtypes = []
     lib.toma_test_set_tuning.restype = None
     lib.toma_test_set_tuning.argtypes = [c_int32, c_int32, c_int32]
+    lib.toma_test_wait_timeout.restype = c_int32
+    lib.toma_test_wait_timeout.argtypes = [ctypes.c_uint32, c_void_p, c_void_p, c_void_p]
     lib.toma_validate.restype = c_int32
     lib.toma_validate.argtypes = [P]
     lib.toma_status_str.restype = c_char_p
@@ -172,6 +174,11 @@ def toma_weights_bytes(desc: TomaDesc) -> int:
 def toma_test_set_tuning(attention_split: int = -1, attention_ctas: int = 0, linear_tile: int = 0) -> None:
     """Test-only: force the attention work plan / the projection tile form (defaults restore the heuristics)."""
     lib.toma_test_set_tuning(attention_split, attention_ctas, linear_tile)
+
+
+def toma_test_wait_timeout(polls, dev_status, outcome) -> None:
+    """Test-only: one CTA waits `polls` polls on a barrier nobody signals, reports through dev_status and returns."""
+    _check(lib.toma_test_wait_timeout(polls, _ptr(dev_status), _ptr(outcome), _stream()), "toma_test_wait_timeout")
 
 
 def toma_dest_per_tile(desc: TomaDesc) -> int:

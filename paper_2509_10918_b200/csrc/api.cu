@@ -298,13 +298,10 @@ toma_status toma_linear(int32_t m, int32_t n, int32_t k, int32_t dtype, const vo
   return cuda_ok(do_linear(m, n, k, dtype == TOMA_F32, a, ws, cs, 1, kActNone, dev_status, (cudaStream_t)stream));
 }
 
-// The wrapped module F: attention over the merged tokens with Q = K = V = X_m, or, with projection weights
-// (proj = {wq, wk, wv, wo}, each [dim][dim], row-major [in][out]), the whole attention module
-// (X_m wq, X_m wk, X_m wv -> attention -> wo); or, with mlp = {w1 [dim][hidden], w2 [hidden][dim]}, the MLP
-// GELU(X_m w1) w2.
-static toma_status block_impl(const toma_desc* desc, int32_t step, const void* x, const void* const* proj,
-                              const void* const* mlp, int hidden, void* out, int32_t* idx_state, void* w_state, void* ws,
-                              size_t ws_bytes, uint32_t* dev_status, void* stream) {
+// Every host-detectable error of a block call, checked before anything is enqueued.
+static toma_status block_check(const toma_desc* desc, int32_t step, const void* x, const void* const* proj,
+                               const void* const* mlp, int hidden, const void* out, const int32_t* idx_state,
+                               const void* w_state, const void* ws, size_t ws_bytes, Geom* geom) {
   Geom g;
   toma_status st = make_geom(desc, &g);
   if (st != TOMA_OK) return st;
@@ -324,6 +321,20 @@ static toma_status block_impl(const toma_desc* desc, int32_t step, const void* x
   if (misaligned(x) || misaligned(out) || misaligned(w_state)) return TOMA_ERR_SHAPE;
   if (!attention_supported_simt(g.dh)) return TOMA_ERR_UNSUPPORTED;
   if ((st = check_ws(g, ws, ws_bytes)) != TOMA_OK) return st;
+  *geom = g;
+  return TOMA_OK;
+}
+
+// The wrapped module F: attention over the merged tokens with Q = K = V = X_m, or, with projection weights
+// (proj = {wq, wk, wv, wo}, each [dim][dim], row-major [in][out]), the whole attention module
+// (X_m wq, X_m wk, X_m wv -> attention -> wo); or, with mlp = {w1 [dim][hidden], w2 [hidden][dim]}, the MLP
+// GELU(X_m w1) w2.
+static toma_status block_impl(const toma_desc* desc, int32_t step, const void* x, const void* const* proj,
+                              const void* const* mlp, int hidden, void* out, int32_t* idx_state, void* w_state, void* ws,
+                              size_t ws_bytes, uint32_t* dev_status, void* stream) {
+  Geom g;
+  toma_status st = block_check(desc, step, x, proj, mlp, hidden, out, idx_state, w_state, ws, ws_bytes, &g);
+  if (st != TOMA_OK) return st;
   cudaStream_t s = (cudaStream_t)stream;
   char* wsb = (char*)ws;
   const WsLayout l = ws_layout(g);
@@ -445,10 +456,10 @@ toma_status toma_block_host(const toma_desc* desc, int32_t step, const void* x_h
                             void* out_dev, int32_t* idx_state, void* w_state, void* ws, size_t ws_bytes,
                             uint32_t* dev_status, void* stream, void* copy_in_stream, void* copy_out_stream,
                             void* copied_in_event, void* computed_event) {
-  Geom g;
-  toma_status st = make_geom(desc, &g);
+  if (!x_host || !out_host) return TOMA_ERR_NULL;
+  Geom g;  // the same checks toma_block makes, before the first copy is enqueued
+  toma_status st = block_check(desc, step, x_dev, nullptr, nullptr, 0, out_dev, idx_state, w_state, ws, ws_bytes, &g);
   if (st != TOMA_OK) return st;
-  if (!x_host || !out_host || !x_dev || !out_dev) return TOMA_ERR_NULL;
   cudaStream_t s = (cudaStream_t)stream;
   cudaStream_t s_in = copy_in_stream ? (cudaStream_t)copy_in_stream : s;
   cudaStream_t s_out = copy_out_stream ? (cudaStream_t)copy_out_stream : s;

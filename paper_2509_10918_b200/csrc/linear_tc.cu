@@ -405,7 +405,9 @@ bool encode_w(const Geom& g, const void* w, CUtensorMap* tm, uint32_t box_tokens
 bool linear_tc_supported(const Geom& g) {
   if (g.f32) return false;
   if (g.tw > 64 || (64 % g.tw) != 0 || (g.th % (64 / g.tw)) != 0) return false;  // 64 tokens = whole tile rows
-  if (g.Nloc % 64 != 0 || g.Dloc % 8 != 0) return false;
+  // The unmerge multiplies destinations 16 at a time out of rows addressed as one (rows, channels)
+  // sheet of the merged tensor: with D_loc a multiple of 16 a step never touches a row of the next tile.
+  if (g.Nloc % 64 != 0 || g.Dloc % 16 != 0) return false;
   if (g.Nloc > kUnmergeTok && g.Nloc % kUnmergeTok != 0) return false;  // unmerge token blocks
   return true;
 }

@@ -9,8 +9,12 @@
 // library instead.
 //
 // Consequences the caller has to know:
-//   * Every GPU that loads the library carries the array (TOMA_STATIC_SCRATCH_BYTES) until the
-//     process exits, used or not.
+//   * The array (TOMA_STATIC_SCRATCH_BYTES) belongs to this library's device code.  With the CUDA
+//     runtime's default lazy loading, a device reserves it when that code is first loaded there,
+//     which is the first toma_select_static call on that device, and keeps it until the process
+//     exits; with eager loading every device that initialises the library holds it from then on.
+//     Either way that first call is where the reservation can fail (no free memory left on the
+//     device): it then returns TOMA_ERR_CUDA, launches nothing, and leaves no sticky error behind.
 //   * Problems whose scratch (quantised tokens + int16 similarity matrices) does not fit are
 //     rejected with TOMA_ERR_SCRATCH_LIMIT before anything is launched.
 //   * All calls on one device share the one array and it keeps whatever the previous call left.
@@ -18,7 +22,8 @@
 //     calls that may overlap on the GPU (different streams, no dependency) race on it; callers
 //     must order them.
 //   * The first call on each device looks the array's device address up (cudaGetSymbolAddress with
-//     that device current).  Make that first call outside any stream capture.
+//     that device current; this is what loads the code and reserves the array, see above).  Make
+//     that first call outside any stream capture.
 // Nothing here calls cudaMalloc, cudaFree or any allocating routine.
 #include <mutex>
 
@@ -46,7 +51,10 @@ cudaError_t scratch_for_current_device(void** out) {
   if (!g_scratch_addr[dev]) {
     void* p = nullptr;
     e = cudaGetSymbolAddress(&p, g_select_scratch);
-    if (e != cudaSuccess) return e;
+    if (e != cudaSuccess) {
+      (void)cudaGetLastError();  // the failed lookup must not surface again in the caller's next CUDA call
+      return e;
+    }
     if (!p) return cudaErrorInvalidSymbol;
     g_scratch_addr[dev] = p;
   }

@@ -13,7 +13,7 @@ namespace toma {
 namespace tc {
 
 constexpr uint32_t kStatusTimeout = 1u;  // bit OR-ed into *dev_status when a bounded wait runs out
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSpinLimit = 1u << 20;  // polls before a wait gives up (each poll suspends the thread for up to about a microsecond)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -50,7 +50,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false (and records the timeout) if the phase never completes;
 // callers then skip their remaining work and fall through to the kernel's teardown.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* dev_status, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* dev_status, volatile int* abort_flag,
+                                          uint32_t limit = kSpinLimit) {
   {  // a phase that is already complete (the common case on a pipelined path) is cheaper to test than to wait for
     uint32_t done;
     asm volatile(
@@ -62,7 +63,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32
         : "memory");
     if (done) return true;
   }
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 1023u) == 1023u && *abort_flag) return false;
   }

@@ -97,6 +97,17 @@ def test_null_and_workspace_errors_are_returned_before_any_launch(toma):
                                None, None, None) == NULL
 
 
+def test_destinations_per_tile_agree_with_the_oracle_on_every_config(toma):
+    """The library's D_loc (toma_dest_per_tile) and the oracle's (dest_count) are computed independently; the
+    buffers of the GPU tests are sized from the former, the expected values from the latter."""
+    import gen
+    from oracle import toma_oracle as O
+    for name in ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5a", "cfg5b"):
+        for ratio in (None, 0.25, 0.75, 0.3, 0.99, 0.0):
+            cfg = gen.config(name) if ratio is None else gen.config(name, merge_ratio=ratio)
+            assert toma.toma_dest_per_tile(toma.desc_from_config(cfg)) == O.dest_count(cfg.n_loc, cfg.merge_ratio)
+
+
 def test_binding_refuses_cpu_tensors(toma):
     import torch
     d = _desc(toma)

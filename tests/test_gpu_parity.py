@@ -234,6 +234,25 @@ def test_attention_growing_logits_exercise_the_rescale_path(toma, dh, L):
     assert_close(to_host64(o)[0], want, "bf16", "attention with growing logits")
 
 
+def test_a_wait_that_nobody_ends_gives_up_and_reports(toma):
+    """The bounded wait every tensor-core kernel uses, made to run out on purpose in the accepted way: a
+    barrier that nobody signals and a limit of a thousand polls.  The kernel must return, the status word
+    must carry the timeout bit, and the next ordinary call on the same context must work."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    outcome = torch.zeros(1, dtype=torch.int32, device="cuda")
+    toma.toma_test_wait_timeout(1000, status, outcome)
+    torch.cuda.synchronize()
+    assert int(outcome.item()) == 2, "the wait on an unsignalled barrier did not give up"
+    assert int(status.item()) & 1 == 1, "TOMA_ERR_TIMEOUT's bit is missing from the status word"
+    # the context is intact: a normal call afterwards succeeds with a clean status word
+    cfg = gen.config("cfg2", batch=1, grid_h=16, grid_w=16)
+    run = Run(toma, cfg, gen.features(cfg))
+    want, _ = O.select_tile(tile_tokens(cfg, gen.features(cfg), 0, 0), od(cfg))
+    assert np.array_equal(run.select()[0, 0], want)
+    run.weights()
+    run.merge()
+
+
 BLOCK_CASES = [
     ("cfg1", {}, None),
     ("cfg2", {}, None),
@@ -527,17 +546,19 @@ def _storage_rounding(dtype):
                          ids=["cfg2", "cfg3", "cfg1-f32", "extra-tokens"])
 def test_block_with_projections_parity(toma, name, over):
     """toma_block_proj: the wrapped module is the whole attention module (Q/K/V projections, attention, output
-    projection) on the merged tokens.  The oracle mirrors the storage rounding between stages."""
+    projection) on the merged tokens.  Primary assertion: the plain fp64 chain of the oracle, no rounding
+    anywhere.  Secondary (labelled) assertion: the oracle with the storage rounding of the kernels mirrored
+    between stages, which isolates arithmetic differences from the six bf16 roundings on the way."""
     cfg = gen.config(name, steps=2, reuse_interval=2, **over)
     desc = toma.desc_from_config(cfg)
     w_host = _proj_weights(cfg)
     w_dev = [to_dev(w, cfg.dtype) for w in w_host]
     idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    st = O.BlockState()
+    st, st_mirror = O.BlockState(), O.BlockState()
     kw = dict(grid_h=cfg.grid_h, grid_w=cfg.grid_w, tile_h=cfg.tile_h, tile_w=cfg.tile_w, merge_ratio=cfg.merge_ratio,
               tau=cfg.tau, n_heads=cfg.n_heads, reuse_interval=2, n_extra=cfg.n_extra,
-              proj=[x.astype(np.float64) for x in w_host], round_fn=_storage_rounding(cfg.dtype))
+              proj=[x.astype(np.float64) for x in w_host])
     for step, x_host in enumerate(gen.feature_sequence(cfg)):
         x = to_dev(x_host, cfg.dtype)
         out = torch.empty_like(x)
@@ -546,7 +567,10 @@ def test_block_with_projections_parity(toma, name, over):
         assert int(status.item()) == 0
         want, _, _ = O.block_step(x_host, step, st, **kw)
         assert np.array_equal(idx.cpu().numpy().astype(np.int64), st.idx)
-        assert_close(to_host64(out), want, cfg.dtype, f"block with projections, step {step}")
+        err = assert_close(to_host64(out), want, cfg.dtype, f"block with projections vs the plain fp64 oracle, step {step}")
+        mirrored, _, _ = O.block_step(x_host, step, st_mirror, round_fn=_storage_rounding(cfg.dtype), **kw)
+        err_m = assert_close(to_host64(out), mirrored, cfg.dtype, f"[secondary: storage rounding mirrored] step {step}")
+        print(f"block_proj {name} step {step}: plain max-abs {err[0]:.3g} rel-fro {err[1]:.3g}; mirrored {err_m[0]:.3g} {err_m[1]:.3g}")
 
 
 @pytest.mark.parametrize("dtype,B,L,h,dh", [("bf16", 2, 1024, 10, 64), ("bf16", 1, 600, 3, 128), ("f32", 1, 200, 2, 64)])
@@ -566,9 +590,11 @@ def test_attention_module_with_projections_parity(toma, dtype, B, L, h, dh):
     rnd = _storage_rounding(dtype)
     got = to_host64(out)
     for b in range(B):
+        q, k, v = (O.linear(x_host[b], w) for w in w_host[:3])
+        assert_close(got[b], O.linear(O.attention(q, k, v, h), w_host[3]), dtype, f"attention module vs the plain fp64 chain, b={b}")
         q, k, v = (rnd(O.linear(x_host[b], w)) for w in w_host[:3])
         want = O.linear(rnd(O.attention(q, k, v, h)), w_host[3])
-        assert_close(got[b], want, dtype, f"attention module b={b}")
+        assert_close(got[b], want, dtype, f"[secondary: storage rounding mirrored] attention module b={b}")
 
 
 def _mlp_weights(cfg, hidden, seed=97):
@@ -595,8 +621,9 @@ def test_mlp_parity(toma, dtype, rows, d, f):
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     pick = np.unique(np.concatenate([[0, rows - 1], np.random.default_rng(rows).choice(rows, size=min(rows, 160), replace=False)]))
+    assert_close(to_host64(out)[pick], O.mlp(x_host[pick], w_host[0], w_host[1]), dtype, "mlp vs the plain fp64 chain")
     want = O.mlp(x_host[pick], w_host[0], w_host[1], _storage_rounding(dtype))
-    assert_close(to_host64(out)[pick], want, dtype, "mlp")
+    assert_close(to_host64(out)[pick], want, dtype, "[secondary: storage rounding mirrored] mlp")
     # the hidden tensor itself: GELU of the first projection, in storage dtype
     hid = ws[: rows * f * (4 if dtype == "f32" else 2)].view(torch.float32 if dtype == "f32" else torch.bfloat16).reshape(rows, f)
     assert_close(to_host64(hid)[pick], O.gelu(O.linear(x_host[pick], w_host[0])), dtype, "mlp hidden")
@@ -606,17 +633,18 @@ def test_mlp_parity(toma, dtype, rows, d, f):
                                               ("cfg2", dict(batch=1, grid_h=16, grid_w=16, n_extra=9), 1288)],
                          ids=["cfg2", "cfg3", "cfg1-f32", "extra-tokens"])
 def test_block_with_mlp_parity(toma, name, over, hidden):
-    """toma_block_mlp: the wrapped module is the MLP on the merged tokens; a refresh step and a reuse step."""
+    """toma_block_mlp: the wrapped module is the MLP on the merged tokens; a refresh step and a reuse step.
+    Primary assertion: the plain fp64 chain; secondary (labelled): storage rounding mirrored between stages."""
     cfg = gen.config(name, steps=2, reuse_interval=2, **over)
     desc = toma.desc_from_config(cfg)
     w_host = _mlp_weights(cfg, hidden)
     w1, w2 = (to_dev(w, cfg.dtype) for w in w_host)
     idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    st = O.BlockState()
+    st, st_mirror = O.BlockState(), O.BlockState()
     kw = dict(grid_h=cfg.grid_h, grid_w=cfg.grid_w, tile_h=cfg.tile_h, tile_w=cfg.tile_w, merge_ratio=cfg.merge_ratio,
               tau=cfg.tau, n_heads=cfg.n_heads, reuse_interval=2, n_extra=cfg.n_extra,
-              mlp_weights=[x.astype(np.float64) for x in w_host], round_fn=_storage_rounding(cfg.dtype))
+              mlp_weights=[x.astype(np.float64) for x in w_host])
     for step, x_host in enumerate(gen.feature_sequence(cfg)):
         x = to_dev(x_host, cfg.dtype)
         out = torch.empty_like(x)
@@ -625,7 +653,10 @@ def test_block_with_mlp_parity(toma, name, over, hidden):
         assert int(status.item()) == 0
         want, _, _ = O.block_step(x_host, step, st, **kw)
         assert np.array_equal(idx.cpu().numpy().astype(np.int64), st.idx)
-        assert_close(to_host64(out), want, cfg.dtype, f"block with MLP, step {step}")
+        err = assert_close(to_host64(out), want, cfg.dtype, f"block with MLP vs the plain fp64 oracle, step {step}")
+        mirrored, _, _ = O.block_step(x_host, step, st_mirror, round_fn=_storage_rounding(cfg.dtype), **kw)
+        err_m = assert_close(to_host64(out), mirrored, cfg.dtype, f"[secondary: storage rounding mirrored] step {step}")
+        print(f"block_mlp {name} step {step}: plain max-abs {err[0]:.3g} rel-fro {err[1]:.3g}; mirrored {err_m[0]:.3g} {err_m[1]:.3g}")
     # a hidden width beyond four times the model width does not fit the block's workspace
     wide = torch.zeros((cfg.dim, 4 * cfg.dim + 8), dtype=x.dtype, device="cuda")
     with pytest.raises(toma.TomaError):
@@ -708,6 +739,68 @@ def test_block_long_sequence_schedule_and_sampled_parity(toma):
             assert np.array_equal(cur, prev), "selection changed on a reuse step"
         prev = cur
         assert torch.isfinite(out.float()).all()
+
+
+@pytest.mark.parametrize("name", ["cfg5a", "cfg5b"])
+def test_block_output_sampled_parity_at_the_largest_sizes(toma, name):
+    """The whole chain merge -> attention over 8192 merged tokens -> unmerge at the stress sizes, element by
+    element on sampled tiles, for a refresh step and the reuse step after it.  The oracle cannot run the whole
+    batch in reasonable time, so: the destinations of the sampled tiles are checked against the oracle bit for
+    bit; weights and merged tokens of every tile of the sampled batch items are computed by the oracle from the
+    destinations; the attention is evaluated at the merged rows of the sampled tiles only (all keys); those rows
+    are unmerged and compared with the library's output for the tile's tokens."""
+    cfg = gen.config(name, steps=2)
+    desc = toma.desc_from_config(cfg)
+    idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ids = O.tile_token_ids(cfg.grid_h, cfg.grid_w, cfg.tile_h, cfg.tile_w)
+    d_loc = od(cfg)
+    assert d_loc == gd(toma, cfg)
+    sampled = {0: [0, cfg.n_tiles // 2 + 1], cfg.batch - 1: [cfg.n_tiles - 1]}
+    weights = {}
+    for step, x_host in enumerate(gen.feature_sequence(cfg)):
+        x = to_dev(x_host, cfg.dtype)
+        out = torch.empty_like(x)
+        toma.toma_block(desc, step, x, out, idx, w, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        got_idx = idx.cpu().numpy().astype(np.int64)
+        got = to_host64(out)
+        for b, tiles in sampled.items():
+            xb = x_host[b].astype(np.float64)
+            if step == 0:
+                for p in tiles:
+                    want_idx, margin = O.select_tile(xb[ids[p]], d_loc)
+                    assert margin > O.FRAGILE_MARGIN
+                    assert np.array_equal(got_idx[b, p], want_idx), f"{name}: selection of tile {p} differs"
+                weights[b] = [O.merge_weights(xb[ids[p]], got_idx[b, p], cfg.tau) for p in range(cfg.n_tiles)]
+            merged = np.concatenate([O.merge(weights[b][p], xb[ids[p]]) for p in range(cfg.n_tiles)])
+            for p in tiles:
+                rows = np.arange(p * d_loc, (p + 1) * d_loc)
+                att = O.attention(merged, merged, merged, cfg.n_heads, query_rows=rows)
+                assert_close(got[b][ids[p]], O.unmerge(weights[b][p], att), cfg.dtype, f"{name} step {step} b={b} tile {p}")
+
+
+def test_unmerge_does_not_read_the_next_tile(toma):
+    """D_loc = 24 (a multiple of 8 but not of 16, the tensor cores' step along destinations) and a NaN planted
+    in every tile's successor rows of the unmerge input: a tile's output may depend on its own D_loc rows only."""
+    cfg = gen.config("cfg2", batch=1, grid_h=16, grid_w=16, dim=128, n_heads=2, merge_ratio=0.625)
+    assert gd(toma, cfg) == 24 and od(cfg) == 24
+    x_host = gen.features(cfg)
+    run = Run(toma, cfg, x_host)
+    idx = run.select()
+    wts = run.weights()
+    y_host = gen.round_to_dtype(0.25 * gen.normal(0, (41, 24), cfg.n_tiles * 24 * cfg.dim).reshape(1, -1, cfg.dim).astype(np.float32), "bf16")
+    ids = O.tile_token_ids(cfg.grid_h, cfg.grid_w, cfg.tile_h, cfg.tile_w)
+    for p in range(cfg.n_tiles - 1):
+        y = y_host.copy()
+        y[0, (p + 1) * 24:(p + 1) * 24 + 8] = np.nan    # the rows a 16-wide step would read past tile p
+        got = run.unmerge(to_dev(y, cfg.dtype))
+        want = O.unmerge(O.merge_weights(x_host[0][ids[p]], idx[0, p], cfg.tau), y_host[0, p * 24:(p + 1) * 24])
+        assert np.isfinite(got[0][ids[p]]).all(), f"tile {p} picked up a value of tile {p + 1}"
+        assert_close(got[0][ids[p]], want, cfg.dtype, f"unmerge tile {p}")
+        if p >= 2:
+            break
 
 
 def test_identity_weights_round_trip_is_bit_exact(toma):

@@ -184,6 +184,109 @@ def test_global_merge_reduces_to_tile_merge_for_one_tile_and_sees_across_tiles()
     assert np.argmax(w2[:, other] * w2.shape[1]) == 0 or np.argmax(w2[:, other]) == 0
 
 
+def test_global_destinations_hand_written_two_by_two_tiles():
+    """4x4 grid cut into four 2x2 tiles, written out by hand: tile p holds tokens
+    p0: 0 1 4 5 | p1: 2 3 6 7 | p2: 8 9 12 13 | p3: 10 11 14 15 (local slot = row-major inside the tile),
+    so the tile-local picks below map to these image tokens, tile-major, pick order inside a tile."""
+    ids = O.tile_token_ids(4, 4, 2, 2)
+    assert ids.tolist() == [[0, 1, 4, 5], [2, 3, 6, 7], [8, 9, 12, 13], [10, 11, 14, 15]]
+    idx_tiles = np.array([[3, 0], [1, 2], [0, 3], [2, 1]])
+    assert O.global_destinations(idx_tiles, ids).tolist() == [5, 0, 3, 6, 8, 13, 14, 11]
+    # a permutation of the picks permutes the result the same way (any fixed one-to-one map would not)
+    assert O.global_destinations(idx_tiles[:, ::-1], ids).tolist() == [0, 5, 6, 3, 13, 8, 11, 14]
+    # the global-merge block puts exactly these tokens' rows first in their softmax columns: token 5 is
+    # destination 0, so A[0, 5] is the largest share of column 5 when tau is cold
+    rng = np.random.default_rng(5)
+    x = rng.normal(size=(16, 8)) * 3.0
+    A = O.softmax_shares(x, O.global_destinations(idx_tiles, ids), 0.01)
+    for row, tok in enumerate([5, 0, 3, 6, 8, 13, 14, 11]):
+        assert np.argmax(A[:, tok]) == row
+
+
+def test_block_step_with_projections_is_the_hand_composed_chain():
+    """block_step(proj=(wq, wk, wv, wo)) against the chain written out here from the pinned pieces: merge with
+    the block's own weights, X_m wq / X_m wk / X_m wv, attention, wo, transpose unmerge.  Distinct random
+    matrices: swapping any two of wq, wk, wv, wo in block_step changes the result."""
+    c = gen.config("cfg3", batch=2, grid_h=8, grid_w=8, tile_h=4, tile_w=4, dim=16, n_heads=2, head_dim=8, steps=1, n_extra=3)
+    x = gen.features(c).astype(np.float64)
+    rng = np.random.default_rng(11)
+    wq, wk, wv, wo = (rng.normal(size=(16, 16)) / 4.0 for _ in range(4))
+    kw = dict(grid_h=8, grid_w=8, tile_h=4, tile_w=4, merge_ratio=0.5, tau=c.tau, n_heads=2, reuse_interval=1, n_extra=3)
+    st = O.BlockState()
+    out, merged, attended = O.block_step(x, 0, st, proj=(wq, wk, wv, wo), **kw)
+    ids = O.tile_token_ids(8, 8, 4, 4)
+    d_loc = O.dest_count(16, 0.5)
+    for b in range(2):
+        xm = np.concatenate([O.merge(st.w[b, p], x[b, ids[p]]) for p in range(4)] + [x[b, 64:]])
+        assert np.allclose(merged[b], xm, atol=1e-12)
+        att = O.attention(O.linear(xm, wq), O.linear(xm, wk), O.linear(xm, wv), 2)
+        y = O.linear(att, wo)
+        assert np.allclose(attended[b], y, atol=1e-12)
+        for p in range(4):
+            assert np.allclose(out[b, ids[p]], O.unmerge(st.w[b, p], y[p * d_loc:(p + 1) * d_loc]), atol=1e-12)
+        assert np.allclose(out[b, 64:], y[4 * d_loc:], atol=1e-12)
+        for perm in ((wk, wq, wv, wo), (wq, wv, wk, wo), (wq, wk, wo, wv), (wo, wk, wv, wq)):
+            other = O.block_step(x, 0, O.BlockState(), proj=perm, **kw)[0]
+            assert not np.allclose(other[b], out[b], atol=1e-3)
+
+
+def _quarter(t):
+    return np.round(np.asarray(t, dtype=np.float64) * 4.0) / 4.0
+
+
+def test_block_step_round_fn_placement_with_projections_and_mlp():
+    """Where block_step applies round_fn: to the merged tokens, to q, k, v, to the attention output and to the
+    projected output (projections); to the merged tokens, the hidden tensor and the MLP output (MLP); to the
+    merged and the attended tokens (plain attention).  A coarse rounding (multiples of 1/4) makes every
+    placement visible; the chain is written out by hand."""
+    c = gen.config("cfg3", batch=1, grid_h=8, grid_w=8, tile_h=4, tile_w=4, dim=16, n_heads=2, head_dim=8, steps=1)
+    x = gen.features(c).astype(np.float64)
+    rng = np.random.default_rng(12)
+    wq, wk, wv, wo = (rng.normal(size=(16, 16)) / 2.0 for _ in range(4))
+    w1, w2 = rng.normal(size=(16, 16)) / 2.0, rng.normal(size=(16, 16)) / 2.0   # square: a swapped pair would still run
+    kw = dict(grid_h=8, grid_w=8, tile_h=4, tile_w=4, merge_ratio=0.5, tau=c.tau, n_heads=2, reuse_interval=1)
+    ids = O.tile_token_ids(8, 8, 4, 4)
+    d_loc = O.dest_count(16, 0.5)
+    calls = []
+
+    def rnd(t):
+        calls.append(np.shape(t))
+        return _quarter(t)
+
+    def unmerged(st, y):
+        out = np.empty((64, 16))
+        for p in range(4):
+            out[ids[p]] = O.unmerge(st.w[0, p], y[p * d_loc:(p + 1) * d_loc])
+        return out
+
+    # projections
+    st = O.BlockState()
+    out = O.block_step(x, 0, st, proj=(wq, wk, wv, wo), round_fn=rnd, **kw)[0]
+    xm = _quarter(np.concatenate([O.merge(st.w[0, p], x[0, ids[p]]) for p in range(4)]))
+    q, k, v = (_quarter(O.linear(xm, w)) for w in (wq, wk, wv))
+    y = _quarter(O.linear(_quarter(O.attention(q, k, v, 2)), wo))
+    assert np.allclose(out[0], unmerged(st, y), atol=1e-12)
+    assert len(calls) == 6          # merged; q, k, v; attention output; projected output
+    assert not np.allclose(out[0], O.block_step(x, 0, O.BlockState(), proj=(wq, wk, wv, wo), **kw)[0][0], atol=1e-3)
+    # MLP
+    calls.clear()
+    st = O.BlockState()
+    out = O.block_step(x, 0, st, mlp_weights=(w1, w2), round_fn=rnd, **kw)[0]
+    hid = _quarter(O.gelu(O.linear(xm, w1)))
+    assert np.allclose(out[0], unmerged(st, _quarter(O.linear(hid, w2))), atol=1e-12)
+    assert len(calls) == 3          # merged; hidden; MLP output
+    plain = O.block_step(x, 0, O.BlockState(), mlp_weights=(w1, w2), **kw)[0]
+    xm_plain = np.concatenate([O.merge(st.w[0, p], x[0, ids[p]]) for p in range(4)])
+    assert np.allclose(plain[0], unmerged(st, O.linear(O.gelu(O.linear(xm_plain, w1)), w2)), atol=1e-12)
+    assert not np.allclose(plain[0], O.block_step(x, 0, O.BlockState(), mlp_weights=(w2, w1), **kw)[0][0], atol=1e-3)
+    # plain attention: merged and attended, once each
+    calls.clear()
+    st = O.BlockState()
+    out = O.block_step(x, 0, st, round_fn=rnd, **kw)[0]
+    assert np.allclose(out[0], unmerged(st, _quarter(O.attention(xm, xm, xm, 2))), atol=1e-12)
+    assert len(calls) == 2
+
+
 def test_softmax_shares_closed_form_and_relation_to_merge_weights():
     """The matrix of the "shares" unmerge: columns sum to 1 (a token's shares over the destinations),
     A~ is A with its rows rescaled, and the closed form of the two-destination case."""

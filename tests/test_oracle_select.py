@@ -155,6 +155,20 @@ def test_pinned_similarity_properties():
         assert np.array_equal(acc.astype(np.float64) * 2.0 ** 24, K[:8, :8].astype(np.float64))
 
 
+def test_gram_rounding_is_ties_to_even_by_hand():
+    """S_q = rint(K / 4096), halves to the even neighbour (the reading taken where Sec. 4.1 gives no precision).
+    Hand-computed: 2048/4096 = 0.5 -> 0, 6144/4096 = 1.5 -> 2, 2049/4096 -> 1, 2047/4096 -> 0, 10240/4096 = 2.5 -> 2,
+    and the same on the negative side (floor, half-up and ties-to-even differ on these)."""
+    K = np.array([2048, 6144, 2049, 2047, 10240, 4096, 0, -2048, -6144, -2049, -2047, -10240, -4096])
+    want = np.array([0, 2, 1, 0, 2, 1, 0, 0, -2, -1, 0, -2, -1])
+    assert np.array_equal(O.round_gram(K), want)
+    # ... and pinned_similarity goes through exactly this step: two tokens at 60 degrees, d = 2
+    x = np.array([[1.0, 0.0], [0.5, np.sqrt(0.75)]])
+    k, _ = O.quantise_tokens(x)
+    S, _ = O.pinned_similarity(x)
+    assert S[0, 1] == O.round_gram(np.array([int(k[0] @ k[1])]))[0] and abs(S[0, 1] - 0.99 ** 2 * 0.5 * 4096) <= 8
+
+
 def test_zero_norm_token_is_harmless():
     rng = np.random.default_rng(7)
     x = rng.normal(size=(8, 32))
