@@ -82,19 +82,30 @@ struct Barriers {
 };
 static_assert(sizeof(Barriers) <= 512, "barrier block outgrew its reservation");
 
-// The iterations [0, T) are cut into G spans at multiples of `quantum`: with T / quantum = q * G + r,
-// the first r spans hold q + 1 quanta and the others q.
-// quantum = 1 balances the spans to within one key tile and splits units; quantum = nblk keeps
-// units whole (no scratch traffic), which wins when the unit count happens to fill the CTAs evenly.
+constexpr int kMaxCtas = 160;  // scratch and the span table are sized for this many persistent CTAs
+
+// The iterations [0, T) are cut into G contiguous spans, CTA g running [bounds[g], bounds[g + 1]).
+// With whole units every bound is a multiple of nblk (no scratch traffic), which wins when the unit
+// count happens to fill the CTAs evenly; otherwise the spans are cut at single key tiles, equal to
+// within one tile, and then every bound that falls within kSnapTiles of a unit boundary is moved
+// onto it: a piece of one or two tiles costs its CTA a whole pipeline drain and epilogue, more than
+// the tiles it moves are worth.
 struct Spans {
-  int T, G, nblk, quantum, q, r;
-  __host__ __device__ int bound(int g) const { return (g * q + (g < r ? g : r)) * quantum; }
-  // the CTA whose span holds iteration `it` (quantum 1 only)
+  int T, G, nblk, split;
+  int bounds[kMaxCtas + 1];
+  __host__ __device__ int bound(int g) const { return bounds[g]; }
+  // the CTA whose span holds iteration `it`
   __host__ __device__ int owner(int it) const {
-    const int big = r * (q + 1);
-    return it < big ? it / (q + 1) : r + (it - big) / q;
+    int lo = 0, hi = G - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (bounds[mid] <= it) lo = mid;
+      else hi = mid - 1;
+    }
+    return lo;
   }
 };
+constexpr int kSnapTiles = 2;
 
 // One piece = the part of a span inside one unit: key tiles [k0, k0 + cnt) of unit u.
 struct Piece {
@@ -303,7 +314,7 @@ __device__ __forceinline__ const float* slot_of(const float* pieces, const Spans
 // ascending CTA order with one fused multiply-add each, starting from zero: finish_piece's direct
 // path follows the same order, so the result does not depend on which path a launch takes.  Loads bypass L1: the pieces were written by other SMs during this launch.
 template <int DH>
-__device__ __noinline__ void combine_rows(const float* pieces, Spans sp, int u, int g_first, int g_last, int row,
+__device__ __noinline__ void combine_rows(const float* pieces, const Spans& sp, int u, int g_first, int g_last, int row,
                                           __nv_bfloat16* dst) {
   constexpr size_t kM = (size_t)kUM * DH, kL = (size_t)kUM * DH + kUM;
   float M = -INFINITY;
@@ -434,7 +445,7 @@ __device__ __forceinline__ bool finish_whole(const Row& t, Barriers* bar, int un
 // ran out.
 template <int DH>
 __device__ __noinline__ bool finish_partial(Row t, Barriers* bar, Piece p, int pc, bool last_of_span, float m_used, float l,
-                                            __nv_bfloat16* o, int L, int heads, Spans sp, uint32_t* tickets, float* pieces,
+                                            __nv_bfloat16* o, int L, int heads, const Spans& sp, uint32_t* tickets, float* pieces,
                                             uint32_t* dev_status) {
   using C = AttCfg<DH>;
   constexpr size_t kM = (size_t)kUM * DH, kL = (size_t)kUM * DH + kUM;
@@ -529,7 +540,7 @@ __device__ __noinline__ bool finish_partial(Row t, Barriers* bar, Piece p, int p
 // unit's pieces up now.
 template <int DH>
 __device__ __noinline__ void settle_first_piece(Barriers* bar, int it_begin, int it_end, Row t, __nv_bfloat16* o, int L,
-                                                int heads, Spans sp, const float* pieces, uint32_t* dev_status) {
+                                                int heads, const Spans& sp, const float* pieces, uint32_t* dev_status) {
   const int nblk = sp.nblk, u = it_begin / nblk;
   const bool first_partial = it_begin > u * nblk || it_end < (u + 1) * nblk;
   if (!first_partial || it_end <= (u + 1) * nblk) return;  // whole, or also the span's last piece: settled already
@@ -553,7 +564,7 @@ template <int DH>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, int L, int heads,
-                    float scale_log2, Spans sp, uint32_t* __restrict__ tickets, float* __restrict__ pieces,
+                    float scale_log2, const __grid_constant__ Spans sp, uint32_t* __restrict__ tickets, float* __restrict__ pieces,
                     uint32_t* dev_status) {
   using C = AttCfg<DH>;
   extern __shared__ uint8_t smem_raw[];
@@ -802,8 +813,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   }
 }
 
-constexpr int kMaxCtas = 160;  // scratch is sized for this many persistent CTAs
-
 size_t ticket_bytes(int B, int L, int heads) {
   const size_t units = (size_t)B * heads * ((L + kUM - 1) / kUM);
   return (units * 8 * sizeof(uint32_t) + 255) & ~(size_t)255;
@@ -822,7 +831,7 @@ int max_ctas() {
 constexpr int kSplitCostTiles = 4;
 
 // Whole units per CTA when that is at most kSplitCostTiles tiles slower than a perfectly even cut;
-// otherwise spans cut at single key tiles.
+// otherwise spans cut at single key tiles (see Spans).
 Spans plan_spans(int units, int nblk) {
   Spans sp;
   sp.nblk = nblk;
@@ -833,15 +842,19 @@ Spans plan_spans(int units, int nblk) {
   int mode = whole_tiles <= even_tiles + kSplitCostTiles ? 0 : 1;
   const int forced = g_tune_attention_split.load(std::memory_order_relaxed);  // test-only override
   if (forced == 0 || forced == 1) mode = forced;
-  if (mode == 0) {
-    sp.quantum = nblk;
-    sp.G = units < gmax ? units : gmax;
-  } else {
-    sp.quantum = 1;
-    sp.G = sp.T < gmax ? sp.T : gmax;
+  sp.split = mode;
+  const int quantum = mode == 0 ? nblk : 1;
+  const int quanta = sp.T / quantum;
+  sp.G = quanta < gmax ? quanta : gmax;
+  const int q = quanta / sp.G, r = quanta - q * sp.G;  // the first r spans hold q + 1 quanta, the others q
+  for (int g = 0; g <= sp.G; ++g) sp.bounds[g] = (g * q + (g < r ? g : r)) * quantum;
+  if (mode == 1 && q >= 8 * kSnapTiles) {
+    for (int g = 1; g < sp.G; ++g) {
+      const int unit_edge = (sp.bounds[g] + nblk / 2) / nblk * nblk;
+      const int off = sp.bounds[g] - unit_edge;
+      if (off != 0 && off >= -kSnapTiles && off <= kSnapTiles) sp.bounds[g] = unit_edge;
+    }
   }
-  sp.q = sp.T / sp.quantum / sp.G;
-  sp.r = sp.T / sp.quantum - sp.q * sp.G;
   return sp;
 }
 
@@ -865,7 +878,7 @@ cudaError_t launch(int B, int L, int heads, const void* q, const void* k, const 
   if (units * nblk > 0x7fffffffLL) return cudaErrorInvalidValue;  // iteration indices are 32-bit
   const Spans sp = plan_spans((int)units, nblk);
   const size_t tb = ticket_bytes(B, L, heads);
-  if (sp.quantum == 1 && !tickets_clean) {  // units are split: their tickets start at zero
+  if (sp.split && !tickets_clean) {  // units are split: their tickets start at zero
     e = cudaMemsetAsync(ws, 0, tb, s);
     if (e != cudaSuccess) return e;
   }
@@ -892,12 +905,12 @@ int attention_tc_plan(int B, int L, int heads, int info[4], int* bounds, int* ow
   if (units * nblk > 0x7fffffffLL) return 0;
   const Spans sp = plan_spans((int)units, nblk);
   info[0] = sp.G;
-  info[1] = sp.quantum == 1 ? 1 : 0;
+  info[1] = sp.split;
   info[2] = (int)units;
   info[3] = nblk;
   for (int g = 0; g <= sp.G && g < capacity; ++g) {
     if (bounds) bounds[g] = sp.bound(g);
-    if (g < sp.G && sp.quantum == 1) {
+    if (g < sp.G && sp.split) {
       if (owner_first) owner_first[g] = sp.owner(sp.bound(g));
       if (owner_last) owner_last[g] = sp.owner(sp.bound(g + 1) - 1);
     }
