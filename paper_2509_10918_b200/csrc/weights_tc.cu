@@ -9,6 +9,8 @@
 //      block, the partial row sums sum_k A_ik.
 //   3. weights_normalise_kernel: A~_ik = A_ik / sum_k' A_ik' with the partial sums added in a
 //      fixed order, stored as A~^T [N_loc][D_loc] split into a hi and a lo bf16 plane.
+// Tiles of at most 256 tokens and 256 destinations take weights_fused_kernel instead of 2 and 3: one
+// CTA per tile, the row normalisation applied in the epilogue of the logits contraction.
 #include "common.cuh"
 #include "tc.cuh"
 
@@ -227,6 +229,201 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// The whole of Sec. 4.2.1 for one tile in one CTA (tiles of at most 256 tokens and 256
+// destinations): logits on the tensor cores for both 128-source blocks of the tile (one
+// accumulator each), softmax over the destinations in registers, the destinations' row sums added
+// up across the tile through shared memory, and the row normalisation 1/Z_i applied as the
+// accumulators are read a last time: A~^T leaves the kernel as its hi and lo bf16 planes, and the
+// fp32 shares never exist in memory.
+//   kMB: 128-source blocks per tile (1 or 2).  Warp 0 TMA, warp 1 MMA, then four epilogue warps
+//   per source block (thread = source token = tensor-memory lane).
+// ------------------------------------------------------------------------------------------------
+template <int kMB>
+__global__ void __launch_bounds__(64 + 128 * kMB, 1)
+weights_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_d,
+                     __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wu, const WParams p, uint32_t* dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int Dl = p.Dloc;
+  const int n_mma = (Dl + 15) & ~15;  // MMA N: destinations padded to 16
+  const int a_bytes = 128 * 128;      // one source block of a stage (only m_tok rows are loaded)
+  const int b_bytes = ((((Dl + 7) & ~7) * 128 + 1023) / 1024) * 1024;
+  const int stage_bytes = kMB * a_bytes + b_bytes;
+  WBars* bar = reinterpret_cast<WBars*>(smem + p.stages * stage_bytes);
+  float* zw = reinterpret_cast<float*>(bar + 1);  // [4 kMB warps][D_loc] partial row sums
+  float* zinv = zw + 4 * kMB * Dl;                // [D_loc] reciprocal row sums of the tile
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int batch = blockIdx.x;
+  const int b = batch / p.P, tile = batch - b * p.P;
+  const int ty = tile / p.tiles_x, tx = tile - ty * p.tiles_x;
+  const int rows_per_box = p.m_tok / p.tw;
+  const int nk = (p.d + kKC - 1) / kKC;
+  const uint32_t ncols_mb = n_mma > 128 ? 256u : n_mma > 64 ? 128u : n_mma > 32 ? 64u : 32u;
+  const uint32_t ncols = kMB * ncols_mb;  // a power of two again (kMB is 1 or 2)
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&bar->full[s], 1);
+      mbar_init(&bar->empty[s], 1);
+    }
+    mbar_init(&bar->done, 1);
+    bar->abort_flag = 0;
+    mbar_fence_init();
+    prefetch_tmap(&tm_x);
+    prefetch_tmap(&tm_d);
+  }
+  dependency_wait();  // before tensor memory is held and before any global access
+  if (threadIdx.x == 0) release_dependents();
+  if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bar->tmem_base;
+  volatile int* abort_flag = &bar->abort_flag;
+
+  if (warp == 0) {
+    if (elect_one()) {
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % p.stages;
+        if (k >= p.stages && !mbar_wait(&bar->empty[s], ((k / p.stages) - 1) & 1, dev_status, abort_flag)) break;
+        uint8_t* sa = smem + s * stage_bytes;
+        mbar_expect_tx(&bar->full[s], kMB * p.m_tok * 128 + Dl * 128);
+        for (int mb = 0; mb < kMB; ++mb)
+          tma_load_4d(sa + mb * a_bytes, &tm_x, &bar->full[s], k * kKC, tx * p.tw, ty * p.th + mb * rows_per_box, b);
+        tma_load_3d(sa + kMB * a_bytes, &tm_d, &bar->full[s], k * kKC, 0, batch);
+      }
+    }
+  } else if (warp == 1) {
+    if (elect_one()) {
+      const uint32_t idesc = idesc_f16(kFmtBF16, kFmtBF16, false, false, 128, n_mma);
+      bool ok = true;
+      for (int k = 0; k < nk; ++k) {
+        const int s = k % p.stages;
+        if (!mbar_wait(&bar->full[s], (k / p.stages) & 1, dev_status, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t aa = smem_u32(smem + s * stage_bytes), ba = aa + kMB * a_bytes;
+#pragma unroll
+        for (int mb = 0; mb < kMB; ++mb)
+#pragma unroll
+          for (int kk = 0; kk < kKC / 16; ++kk)
+            mma_ss(tmem + mb * ncols_mb, smem_desc_sw128(aa + mb * a_bytes + kk * 32, 16, 1024),
+                   smem_desc_sw128(ba + kk * 32, 16, 1024), idesc, k > 0 || kk > 0);
+        mma_commit(&bar->empty[s]);
+      }
+      if (ok) mma_commit(&bar->done);
+    }
+  } else {
+    const int mb = (warp - 2) >> 2, quarter = warp & 3;
+    const int k_loc = quarter * 32 + lane;  // source row inside its block = tensor-memory lane
+    const bool valid = k_loc < p.m_tok;
+    const uint32_t taddr = tmem + mb * ncols_mb + ((uint32_t)(quarter * 32) << 16);
+    float* zrow = zw + (mb * 4 + quarter) * Dl;
+    float neg_m = 0.f, inv = 0.f;
+    const bool ok = mbar_wait(&bar->done, 0, dev_status, abort_flag);
+    if (ok) {
+      tc_fence_after();
+      // pass 1: maximum logit over the destinations
+      float mx = -INFINITY;
+      for (int i0 = 0; i0 < Dl; i0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + i0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if (i0 + e < Dl) mx = fmaxf(mx, __uint_as_float(r[e]));
+      }
+      neg_m = -mx * p.scale_log2;
+      // pass 2: denominator of the token's softmax
+      float sum = 0.f;
+      for (int i0 = 0; i0 < Dl; i0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + i0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if (i0 + e < Dl) sum += fast_exp2(fmaf(__uint_as_float(r[e]), p.scale_log2, neg_m));
+      }
+      inv = valid ? 1.f / sum : 0.f;
+      // pass 3: the shares' sums over this warp's 32 source tokens, per destination
+      for (int i0 = 0; i0 < Dl; i0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + i0, r);
+        tmem_wait_ld();
+        float a[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const float v = fast_exp2(fmaf(__uint_as_float(r[e]), p.scale_log2, neg_m)) * inv;
+          a[e] = (valid && i0 + e < Dl) ? v : 0.f;
+        }
+        // transpose-reduce: afterwards lane c holds the sum over the warp's 32 rows of column i0 + c
+#pragma unroll
+        for (int off = 16, n = 32; off >= 1; off >>= 1, n >>= 1) {
+          const bool upper = (lane & off) != 0;
+#pragma unroll
+          for (int c = 0; c < n / 2; ++c) {
+            const float send = upper ? a[c] : a[c + n / 2];
+            const float keep = upper ? a[c + n / 2] : a[c];
+            a[c] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+          }
+        }
+        if (i0 + lane < Dl) zrow[i0 + lane] = a[0];
+      }
+    }
+    // the tile's row sums: warps of a block pairwise, then the blocks in order (a fixed order: the
+    // result does not depend on scheduling); a row sum that underflowed to 0 gives a zero row
+    asm volatile("bar.sync 1, %0;" ::"n"(128 * kMB) : "memory");
+    for (int i = threadIdx.x - 64; i < Dl; i += 128 * kMB) {
+      float z = 0.f;
+#pragma unroll
+      for (int m = 0; m < kMB; ++m) {
+        const float* q = zw + m * 4 * Dl + i;
+        z += (q[0] + q[Dl]) + (q[2 * Dl] + q[3 * Dl]);
+      }
+      zinv[i] = z > 0.f ? 1.f / z : 0.f;
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(128 * kMB) : "memory");
+    if (ok && valid) {
+      // pass 4: A~_ik = A_ik / Z_i, written as row k of A~^T [N_loc][D_loc], hi plane then lo plane
+      const size_t plane = (size_t)p.Nloc * Dl;
+      const size_t row = (size_t)(mb * p.m_tok + k_loc) * Dl;
+      __nv_bfloat16* t_hi = w + (size_t)batch * 2 * plane + row;
+      __nv_bfloat16* u_hi = wu ? wu + (size_t)batch * 2 * plane + row : nullptr;
+      for (int i0 = 0; i0 < Dl; i0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + i0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e0 = 0; e0 < 32; e0 += 8) {
+          if (i0 + e0 >= Dl) break;  // D_loc is a multiple of 8
+          __align__(16) __nv_bfloat16 hi[8], lo[8], uh[8], ul[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const float a = fast_exp2(fmaf(__uint_as_float(r[e0 + e]), p.scale_log2, neg_m)) * inv;
+            const float v = a * zinv[i0 + e0 + e];
+            hi[e] = __float2bfloat16_rn(v);
+            lo[e] = __float2bfloat16_rn(v - __bfloat162float(hi[e]));
+            uh[e] = __float2bfloat16_rn(a);
+            ul[e] = __float2bfloat16_rn(a - __bfloat162float(uh[e]));
+          }
+          *reinterpret_cast<uint4*>(t_hi + i0 + e0) = *reinterpret_cast<const uint4*>(hi);
+          *reinterpret_cast<uint4*>(t_hi + plane + i0 + e0) = *reinterpret_cast<const uint4*>(lo);
+          if (u_hi) {
+            *reinterpret_cast<uint4*>(u_hi + i0 + e0) = *reinterpret_cast<const uint4*>(uh);
+            *reinterpret_cast<uint4*>(u_hi + plane + i0 + e0) = *reinterpret_cast<const uint4*>(ul);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, ncols);
+  }
+}
+
 __global__ void __launch_bounds__(256)
 weights_normalise_kernel(const float* __restrict__ shares, const float* __restrict__ zpart, __nv_bfloat16* __restrict__ w,
                          __nv_bfloat16* __restrict__ wu, int Nloc, int Dloc, int mblocks) {
@@ -378,6 +575,11 @@ cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, 
   if (le != cudaSuccess) return le;
 
   CUtensorMap tx, td;
+  // One CTA per tile, no fp32 shares in memory.  With two source blocks per tile the fused form halves the
+  // CTA count, and a CTA takes in its operands at a few tens of bytes per clock whatever else it does: it
+  // wins once there are enough tiles to occupy the SMs anyway (measured: 77 against 91 us on 256 tiles, 30
+  // against 26 us on 32 tiles); with one source block per tile it only saves the second kernel.
+  const bool fused = g.Dloc <= 256 && g.Dloc % 8 == 0 && (mblocks == 1 || (mblocks == 2 && (int)tiles >= sm_count() / 2));
   const uint64_t xdims[4] = {(uint64_t)g.d, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.B};
   const uint64_t xstr[3] = {(uint64_t)g.d * 2, (uint64_t)g.W * g.d * 2, (uint64_t)g.tokens_all() * g.d * 2};
   const uint32_t xbox[4] = {64, (uint32_t)g.tw, (uint32_t)(p.m_tok / g.tw), 1};
@@ -387,9 +589,29 @@ cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, 
   if (!encode_tmap_16bit(&tx, x, 4, xdims, xstr, xbox) || !encode_tmap_16bit(&td, dg, 3, ddims, dstr, dbox))
     return cudaErrorInvalidValue;
   const int b_rows = g.Dloc > 256 ? 512 : ((g.Dloc + 7) & ~7);
+  const int nk = (g.d + kKC - 1) / kKC;
+  if (fused) {
+    const int stage_bytes = mblocks * 128 * 128 + ((b_rows * 128 + 1023) / 1024) * 1024;
+    p.stages = (200 * 1024) / stage_bytes;
+    p.stages = p.stages > 4 ? 4 : p.stages;
+    if (p.stages > nk) p.stages = nk;
+    const int smem = 1024 + p.stages * stage_bytes + (int)sizeof(WBars) + (4 * mblocks + 1) * g.Dloc * 4 + 64;
+    if (mblocks == 2) {
+      static std::atomic<unsigned long long> raised2{0};
+      if (cudaError_t e = raise_dynamic_smem(weights_fused_kernel<2>, 227 * 1024, raised2); e != cudaSuccess) return e;
+      le = launch_dependent(weights_fused_kernel<2>, dim3((unsigned)tiles), dim3(320), (size_t)smem, s, tx, td,
+                            (__nv_bfloat16*)w, (__nv_bfloat16*)wu, p, dev_status);
+    } else {
+      static std::atomic<unsigned long long> raised1{0};
+      if (cudaError_t e = raise_dynamic_smem(weights_fused_kernel<1>, 227 * 1024, raised1); e != cudaSuccess) return e;
+      le = launch_dependent(weights_fused_kernel<1>, dim3((unsigned)tiles), dim3(192), (size_t)smem, s, tx, td,
+                            (__nv_bfloat16*)w, (__nv_bfloat16*)wu, p, dev_status);
+    }
+    count_launch();
+    return le != cudaSuccess ? le : cudaGetLastError();
+  }
   const int stage_bytes = 128 * 128 + ((b_rows * 128 + 1023) / 1024) * 1024;
   p.stages = stage_bytes <= 48 * 1024 ? 4 : 2;
-  const int nk = (g.d + kKC - 1) / kKC;
   if (p.stages > nk) p.stages = nk;
   const int smem = 1024 + p.stages * stage_bytes + (int)sizeof(WBars) + 4 * p.d_block * 4 + 64;
   static std::atomic<unsigned long long> smem_raised{0};
