@@ -110,8 +110,11 @@ TOMA_API uint64_t toma_launch_counter(void);
  * on these settings, only the launch configuration does.  Process-wide; not for concurrent use.
  *   attention_split: 0 = whole work units per CTA, 1 = spans cut at single key tiles, other = heuristic
  *   attention_ctas : > 0 = number of persistent CTAs (clamped to the scratch capacity), else heuristic
- *   linear_tile    : 1 = 128 x 256, 2 = 128 x 320, 3 = 256 x 256 tiles, else heuristic */
-TOMA_API void toma_test_set_tuning(int32_t attention_split, int32_t attention_ctas, int32_t linear_tile);
+ *   linear_tile    : 1 = 128 x 256, 2 = 128 x 320, 3 = 256 x 256 tiles, else heuristic
+ *   block_unfused  : 1 = toma_block runs merge, attention and unmerge as three kernels even for the shapes its
+ *                    one-kernel reuse step covers (so that both paths can be compared), else the library chooses */
+TOMA_API void toma_test_set_tuning(int32_t attention_split, int32_t attention_ctas, int32_t linear_tile,
+                                   int32_t block_unfused);
 /* TEST-ONLY (no counterpart in the paper): launches one CTA that waits, with the library's bounded wait and
  * a limit of `polls` polls (1..100000), on a barrier that nobody signals.  The wait gives up, ORs
  * TOMA_ERR_TIMEOUT's bit (bit 0) into *dev_status (device, may be NULL), writes 2 to *outcome (device, may be

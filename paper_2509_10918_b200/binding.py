@@ -62,7 +62,7 @@ def _load() -> ctypes.CDLL:
     lib.toma_launch_counter.restype = ctypes.c_uint64
     lib.toma_launch_counter.argtypes = []
     lib.toma_test_set_tuning.restype = None
-    lib.toma_test_set_tuning.argtypes = [c_int32, c_int32, c_int32]
+    lib.toma_test_set_tuning.argtypes = [c_int32, c_int32, c_int32, c_int32]
     lib.toma_test_wait_timeout.restype = c_int32
     lib.toma_test_wait_timeout.argtypes = [ctypes.c_uint32, c_void_p, c_void_p, c_void_p]
     lib.toma_validate.restype = c_int32
@@ -171,9 +171,10 @@ def toma_weights_bytes(desc: TomaDesc) -> int:
     return lib.toma_weights_bytes(ctypes.byref(desc))
 
 
-def toma_test_set_tuning(attention_split: int = -1, attention_ctas: int = 0, linear_tile: int = 0) -> None:
-    """Test-only: force the attention work plan / the projection tile form (defaults restore the heuristics)."""
-    lib.toma_test_set_tuning(attention_split, attention_ctas, linear_tile)
+def toma_test_set_tuning(attention_split: int = -1, attention_ctas: int = 0, linear_tile: int = 0, block_unfused: int = 0) -> None:
+    """Test-only: force the attention work plan / the projection tile form / the three-kernel block path
+    (defaults restore the library's own choices)."""
+    lib.toma_test_set_tuning(attention_split, attention_ctas, linear_tile, block_unfused)
 
 
 def toma_test_wait_timeout(polls, dev_status, outcome) -> None:

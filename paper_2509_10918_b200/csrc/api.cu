@@ -344,6 +344,11 @@ static toma_status block_impl(const toma_desc* desc, int32_t step, const void* x
   cudaError_t e = cudaSuccess;
   if (refresh_sel) e = do_select(g, x, idx_state, wsb, dev_status, s);
   if (e == cudaSuccess && refresh_w) e = do_weights(g, x, idx_state, w_state, wsb, dev_status, s);
+  // merge, attention and unmerge as one kernel where the shape allows (small tiles, few merged tokens)
+  if (!proj && !mlp && block_fused_supported(g) && !g_tune_block_unfused.load(std::memory_order_relaxed)) {
+    if (e == cudaSuccess) e = launch_block_fused(g, w_state, x, out, dev_status, s);
+    return cuda_ok(e);
+  }
   void* xm = wsb + l.xm_off;
   void* att = wsb + l.att_off;
   // the merge kernel clears the attention kernel's tickets on the side (saves a memset between them)
@@ -510,7 +515,7 @@ toma_status toma_unmerge_weights_export(const toma_desc* desc, const void* w, fl
 
 namespace toma {
 std::atomic<unsigned long long> g_launches{0};
-std::atomic<int> g_tune_attention_split{-1}, g_tune_attention_ctas{0}, g_tune_linear_tile{0};
+std::atomic<int> g_tune_attention_split{-1}, g_tune_attention_ctas{0}, g_tune_linear_tile{0}, g_tune_block_unfused{0};
 
 int sm_count() {
   static std::atomic<int> cached[64];
@@ -524,7 +529,8 @@ int sm_count() {
 }
 extern "C" uint64_t toma_launch_counter(void) { return (uint64_t)toma::g_launches.load(); }
 
-extern "C" void toma_test_set_tuning(int32_t attention_split, int32_t attention_ctas, int32_t linear_tile) {
+extern "C" void toma_test_set_tuning(int32_t attention_split, int32_t attention_ctas, int32_t linear_tile, int32_t block_unfused) {
+  toma::g_tune_block_unfused.store(block_unfused == 1 ? 1 : 0);
   toma::g_tune_attention_split.store(attention_split == 0 || attention_split == 1 ? attention_split : -1);
   toma::g_tune_attention_ctas.store(attention_ctas > 0 ? attention_ctas : 0);
   toma::g_tune_linear_tile.store(linear_tile >= 1 && linear_tile <= 3 ? linear_tile : 0);

@@ -34,20 +34,19 @@
 // registers for both the maximum and the exponentials.
 // Keys past the sequence end are zero-filled by TMA and masked out; query rows past the end are
 // computed on zeros and not written.
+#include "attention_core.cuh"
 #include "common.cuh"
 #include "tc.cuh"
 
 namespace toma {
 
 using namespace tc;
+using namespace attn;
 
 namespace {
 
-constexpr int kBM = 128;      // rows of one query tile = threads of one softmax warp group
 constexpr int kUM = 2 * kBM;  // queries per work unit
-constexpr int kBN = 64;       // keys per tile
 constexpr int kThreads = 384;
-constexpr float kRescaleThreshold = 8.0f;
 
 template <int DH>
 struct AttCfg {
@@ -147,149 +146,6 @@ struct Cursor {
 // Scratch of one piece: O as [DH / 4][256 rows] float4, then m[256], l[256].
 template <int DH>
 __host__ __device__ constexpr size_t piece_floats() { return (size_t)kUM * DH + 2 * kUM; }
-
-__device__ __forceinline__ float ex2_mufu(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-// 2^x for x <= ~9 on the FMA pipe: round to nearest integer with the 1.5*2^23 trick, degree-3
-// near-minimax polynomial for 2^f on [-0.5, 0.5], exponent patched in with an integer add.
-__device__ __forceinline__ float ex2_poly(float x) {
-  x = fmaxf(x, -126.f);
-  const float t = x + 12582912.f;
-  const float f = x - (t - 12582912.f);
-  float p = fmaf(0.0551716648f, f, 0.2426111251f);
-  p = fmaf(p, f, 0.6932609677f);
-  p = fmaf(p, f, 0.9999280572f);
-  return __int_as_float(__float_as_int(p) + (int)((unsigned)__float_as_int(t) << 23));
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-  float d;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
-__device__ __forceinline__ uint32_t pack_bf16_rn(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-__device__ __forceinline__ uint32_t pack_bf16_trunc(float lo, float hi) {  // upper halves of both words
-  return __byte_perm(__float_as_uint(lo), __float_as_uint(hi), 0x7632);
-}
-
-// View of 32 consecutive registers of a larger per-thread array (all indices are compile-time).
-template <int kOff, int kN>
-__device__ __forceinline__ uint32_t (&sub32(uint32_t (&r)[kN]))[32] {
-  return *reinterpret_cast<uint32_t(*)[32]>(&r[kOff]);
-}
-
-// Maximum of 32 tensor-memory words (columns first .. first+31 of this row; columns >= valid ignored).
-template <bool kMask>
-__device__ __forceinline__ float chunk_max(const uint32_t (&r)[32], float mx, int first, int valid) {
-  if (kMask) {
-#pragma unroll
-    for (int e = 0; e < 32; ++e) mx = fmaxf(mx, (first + e < valid) ? __uint_as_float(r[e]) : -INFINITY);
-  } else {
-#pragma unroll
-    for (int e = 0; e < 32; e += 2) mx = max3(mx, __uint_as_float(r[e]), __uint_as_float(r[e + 1]));
-  }
-  return mx;
-}
-
-// P for 32 columns as packed bf16 pairs in pk[16]; returns their fp32 sum when sums stay in registers.
-template <bool kMask, bool kRegSum>
-__device__ __forceinline__ float chunk_exp(const uint32_t (&r)[32], uint32_t (&pk)[16], float scale, float neg_m,
-                                           int first, int valid) {
-  float l = 0.f;
-#pragma unroll
-  for (int e = 0; e < 32; e += 2) {
-    const float x0 = fmaf(__uint_as_float(r[e]), scale, neg_m);
-    const float x1 = fmaf(__uint_as_float(r[e + 1]), scale, neg_m);
-    float p0 = ex2_mufu(x0);
-    float p1 = (e & 2) ? ex2_poly(x1) : ex2_mufu(x1);  // every fourth exponential on the FMA pipe
-    if (kMask) {
-      if (first + e >= valid) p0 = 0.f;
-      if (first + e + 1 >= valid) p1 = 0.f;
-    }
-    if (kRegSum) {
-      l += p0 + p1;
-      pk[e >> 1] = pack_bf16_rn(p0, p1);
-    } else {
-      pk[e >> 1] = pack_bf16_trunc(p0, p1);
-    }
-  }
-  return l;
-}
-
-// One 64-key tile of the online softmax for one query row.
-template <int DH, bool kMask>
-__device__ __forceinline__ bool softmax_tile(uint32_t sb, uint32_t ob, float scale_log2, int valid, int j, float& m_used,
-                                             float& l, uint64_t* pv_done, uint32_t pv_parity, uint32_t* dev_status, volatile int* abort_flag) {
-  using C = AttCfg<DH>;
-  uint32_t sr[64];
-  tmem_ld32(sb, sub32<0>(sr));
-  tmem_ld32(sb + 32, sub32<32>(sr));
-  tmem_wait_ld();
-  float mx = -INFINITY;
-  mx = chunk_max<kMask>(sub32<0>(sr), mx, 0, valid);
-  mx = chunk_max<kMask>(sub32<32>(sr), mx, 32, valid);
-  mx *= scale_log2;
-  float factor = 1.f;
-  bool rescale = false;
-  if (j == 0) {
-    m_used = mx;
-  } else if (mx > m_used + kRescaleThreshold) {
-    factor = ex2_mufu(m_used - mx);
-    m_used = mx;
-    rescale = true;
-  }
-  if (__any_sync(0xffffffffu, rescale)) {
-    // O holds every PV product issued so far; the last one (tile j-1) must have landed
-    if (!mbar_wait(pv_done, pv_parity, dev_status, abort_flag)) return false;
-    tc_fence_after();
-    l *= factor;
-#pragma unroll
-    for (int c = 0; c < DH / 32; ++c) {
-      uint32_t t[32];
-      tmem_ld32(ob + c * 32, t);
-      tmem_wait_ld();
-#pragma unroll
-      for (int e = 0; e < 32; ++e) t[e] = __float_as_uint(__uint_as_float(t[e]) * factor);
-      tmem_st32(ob + c * 32, t);
-    }
-    if (C::kSumMma) {
-      uint32_t rs[16];
-      tmem_ld16(ob + DH, rs);
-      tmem_wait_ld();
-#pragma unroll
-      for (int e = 0; e < 16; ++e) rs[e] = __float_as_uint(__uint_as_float(rs[e]) * factor);
-      tmem_st16(ob + DH, rs);
-    }
-  }
-  // P = 2^(S*c - m) as packed bf16 over the first 32 columns of this S buffer
-  const float neg_m = -m_used;
-  constexpr bool kRegSum = !C::kSumMma;
-  uint32_t pk[16];
-  l += chunk_exp<kMask, kRegSum>(sub32<0>(sr), pk, scale_log2, neg_m, 0, valid);
-  tmem_st16(sb, pk);
-  l += chunk_exp<kMask, kRegSum>(sub32<32>(sr), pk, scale_log2, neg_m, 32, valid);
-  tmem_st16(sb + 16, pk);
-  tmem_wait_st();
-  return true;
-}
-
-// 32 accumulator columns of one row, scaled and rounded to bf16: 64 contiguous bytes.
-__device__ __forceinline__ void store_row32(__nv_bfloat16* dst, const uint32_t (&r)[32], float inv) {
-#pragma unroll
-  for (int e = 0; e < 32; e += 8) {
-    uint4 v;
-    v.x = pack_bf16_rn(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
-    v.y = pack_bf16_rn(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-    v.z = pack_bf16_rn(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-    v.w = pack_bf16_rn(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
-    *reinterpret_cast<uint4*>(dst + e) = v;
-  }
-}
 
 // Where the output rows of unit u start for query row `row` (0..255) of the unit (nullptr past the sequence end).
 template <int DH>
@@ -557,7 +413,7 @@ template <int DH>
 __device__ __noinline__ bool softmax_tile_ragged(uint32_t sb, uint32_t ob, float scale_log2, int valid, int j, float& m_used,
                                                  float& l, uint64_t* pv_done, uint32_t pv_parity, uint32_t* dev_status,
                                                  volatile int* abort_flag) {
-  return softmax_tile<DH, true>(sb, ob, scale_log2, valid, j, m_used, l, pv_done, pv_parity, dev_status, abort_flag);
+  return softmax_tile<DH, AttCfg<DH>::kSumMma, true>(sb, ob, scale_log2, valid, j, m_used, l, pv_done, pv_parity, dev_status, abort_flag);
 }
 
 template <int DH>
@@ -792,7 +648,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const int valid = L - (p.k0 + j) * kBN;  // keys of this tile inside the sequence (>= 64: all)
         uint64_t* pvb = &bar->kv_empty[(n + C::kStages - 1) % C::kStages];  // barrier the previous tile's PV commits to
         const uint32_t pvp = (uint32_t)(((n - 1) / C::kStages) & 1);
-        if (valid >= kBN) ok = softmax_tile<DH, false>(sb, t.ob, scale_log2, kBN, j, m_used, l, pvb, pvp, dev_status, abort_flag);
+        if (valid >= kBN) ok = softmax_tile<DH, C::kSumMma, false>(sb, t.ob, scale_log2, kBN, j, m_used, l, pvb, pvp, dev_status, abort_flag);
         else ok = softmax_tile_ragged<DH>(sb, t.ob, scale_log2, valid, j, m_used, l, pvb, pvp, dev_status, abort_flag);
         if (!ok) break;
         tc_fence_before();

@@ -284,6 +284,41 @@ def test_block_sequence_parity(toma, name, over, _):
         assert_close(to_host64(out), want, cfg.dtype, f"block step {step}")
 
 
+@pytest.mark.parametrize("over", [dict(), dict(batch=1, grid_h=32, grid_w=16, dim=128, n_heads=2),
+                                  dict(batch=3, grid_h=16, grid_w=32, tile_h=4, tile_w=16, dim=640, n_heads=10)],
+                         ids=["cfg2", "256-merged-tokens", "4x16-tiles"])
+def test_block_one_kernel_reuse_step_parity(toma, tuning, over):
+    """Shapes with 64-token tiles, 32 destinations and at most 512 merged tokens run merge, attention and unmerge of
+    a step as ONE kernel.  Both forms of the step (one kernel; three kernels, forced through the test-only
+    setter) must match the oracle on a refresh step and on the reuse step after it, and each other closely."""
+    cfg = gen.config("cfg2", steps=2, reuse_interval=2, **over)
+    desc = toma.desc_from_config(cfg)
+    kw = dict(grid_h=cfg.grid_h, grid_w=cfg.grid_w, tile_h=cfg.tile_h, tile_w=cfg.tile_w, merge_ratio=cfg.merge_ratio,
+              tau=cfg.tau, n_heads=cfg.n_heads, reuse_interval=2)
+    outs = {}
+    for unfused in (0, 1):
+        tuning(block_unfused=unfused)
+        idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        st = O.BlockState()
+        launches = []
+        for step, x_host in enumerate(gen.feature_sequence(cfg)):
+            x = to_dev(x_host, cfg.dtype)
+            out = torch.full_like(x, float("nan"))
+            n0 = toma.toma_launch_counter()
+            toma.toma_block(desc, step, x, out, idx, w, ws, status)
+            torch.cuda.synchronize()
+            launches.append(toma.toma_launch_counter() - n0)
+            assert int(status.item()) == 0
+            want, _, _ = O.block_step(x_host, step, st, **kw)
+            assert np.array_equal(idx.cpu().numpy().astype(np.int64), st.idx)
+            assert_close(to_host64(out), want, cfg.dtype, f"block step {step}, {'three kernels' if unfused else 'one kernel'}")
+            outs[(unfused, step)] = to_host64(out)
+        assert launches[1] == (3 if unfused else 1), f"reuse step launched {launches[1]} kernels"
+    for step in (0, 1):
+        assert np.abs(outs[(0, step)] - outs[(1, step)]).max() <= 2 ** -6, "the two forms of the step disagree"
+
+
 def test_block_separate_weight_schedule_parity(toma):
     """Destinations every 4 steps, weights every 2 (the paper refreshes weights more often than
     destinations): indices stay put at step 2 while the weights follow the drifted features."""
