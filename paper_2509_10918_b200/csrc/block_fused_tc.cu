@@ -6,14 +6,16 @@
 //
 // Merge is linear per channel and local to a tile, and a head's attention needs the merged tokens of
 // all tiles but only the head's 64 channels.  So one CTA = (batch, head, 256 merged queries = 8 tiles):
-//   A  merges the head's 64 channels of ALL tiles of the image into a [D][64] bf16 matrix in shared
-//      memory (the other CTAs of the head recompute it: a few MFLOP each) - this is K and V;
+//   A  merges the head's 64 channels of its own 8 tiles into its 256 rows of a [D][64] bf16 matrix in
+//      shared memory - K and V of the head.  With 512 merged tokens the head's two CTAs form a cluster,
+//      and each sends its rows to the other's copy of the matrix (bulk copies between the shared memories);
 //   B  runs the attention of its 256 merged queries (two 128-row query tiles, rows of the same matrix)
 //      over the D keys exactly as attention_tc.cu does (S double-buffered in tensor memory, P written
 //      over S, [V | 1] operand for the row sums, lazy rescale), except that nothing is loaded: K and V
 //      are resident;
 //   C  unmerges its 8 tiles' 512 tokens x 64 channels from the normalised accumulators (written to
-//      shared memory as bf16, the B operand of the unmerge) and stores them in spatial order.
+//      shared memory as bf16, the B operand of the unmerge) and stores them in spatial order (rows staged
+//      where K and V were, one TMA store per warp's half tile).
 // Both contractions with the weights run on the tensor cores with 128 rows on M by pairing tiles: the
 // operand of a pair is block diagonal, a [128 tokens][64 destinations] slab whose row k holds token k's
 // 32 weights in the half that belongs to its tile and zeros in the other.  Read MN-major it is the A
@@ -25,7 +27,7 @@
 //
 // Warps 0..3 / 4..7: softmax of query tile 0 / 1; in A warps 0..3 build slabs and warps 4..7 move
 // merged rows from tensor memory to shared memory; in C each group builds and stores its own pairs.
-// Warp 8: TMA producer of the token tiles (A only).  Warp 9: one elected thread issues every MMA.
+// Warp 8: TMA producer of the token tiles (A only; the four pairs have a stage each).  Warp 9: one elected thread issues every MMA.
 #include "attention_core.cuh"
 #include "common.cuh"
 #include "tc.cuh"
@@ -45,11 +47,12 @@ constexpr int kOnesBytes = kBN * 128;
 constexpr int kMaxD = 512;                    // merged tokens per image the shared-memory matrix holds
 
 struct FBars {
-  uint64_t x_full[4], x_empty[4];        // token tiles of a pair landed (TMA) / its MMAs are done with them
+  uint64_t x_full[4];                    // token tiles of a pair landed (TMA)
   uint64_t slab_full[2], slab_empty[2];  // slab of a pair built (4 warps) / its MMAs are done with it
   uint64_t slab2_full;                   // the extra slab of the unmerge's third pair
-  uint64_t acc_full[2], acc_empty[2];  // merge: a group of four tiles accumulated / moved to shared memory
-  uint64_t kv_ready;       // the merged matrix is complete in shared memory
+  uint64_t acc_full[2];    // merge: a group of four tiles accumulated
+  uint64_t kv_ready;       // the merged matrix is complete in shared memory (both CTAs' rows)
+  uint64_t kv_sent;        // the peer has received this CTA's rows (they may be overwritten)
   uint64_t s_full[2][2], p_full[2][2];
   uint64_t pv_done[4];     // per key tile: its PV products (both query tiles) have landed
   uint64_t o_done[2];
@@ -60,9 +63,8 @@ struct FBars {
 };
 
 struct FParams {
-  int P, tiles_x, th, tw, W, d, n_all, heads, D, units;  // units = D / 256 per (batch, head)
+  int tiles_x, th, tw, heads, D, units;  // units = D / 256 per (batch, head)
   const __nv_bfloat16* w;  // A~^T planes: [tile][hi, lo][64 tokens][32 destinations]
-  __nv_bfloat16* out;      // [batch][tokens][d]
   float scale_log2;
 };
 
@@ -72,7 +74,7 @@ struct SlabRow {
 };
 __device__ __forceinline__ SlabRow load_slab_row(const FParams& p, int b, int ta, int r /*0..127*/) {
   const int tile = r < kTileTok ? ta : ta + 1, k = r & (kTileTok - 1);
-  const size_t row = ((size_t)(2 * (b * p.P + tile)) * kTileTok + k) * kTileDest;
+  const size_t row = ((size_t)(2 * (b * (p.D / kTileDest) + tile)) * kTileTok + k) * kTileDest;
   SlabRow w;
 #pragma unroll
   for (int pl = 0; pl < 2; ++pl) {
@@ -97,6 +99,51 @@ __device__ __forceinline__ void store_slab_row(uint8_t* slab, const SlabRow& w, 
   }
 }
 
+// ---- the two CTAs of a head as a cluster
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Every thread of both CTAs arrives; nobody passes before all have (shared memory and barriers of the peer exist).
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// The address of the peer CTA's copy of a shared-memory location of this CTA.
+__device__ __forceinline__ uint32_t peer_addr(uint32_t local, uint32_t peer) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(peer));
+  return r;
+}
+// Bulk copy of `bytes` of this CTA's shared memory to the peer's (same layout); the bytes count on the peer's barrier.
+__device__ __forceinline__ void copy_to_peer(uint32_t peer_dst, const void* src, uint32_t bytes, uint32_t peer_bar) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(peer_dst),
+               "r"(smem_u32(src)), "r"(bytes), "r"(peer_bar)
+               : "memory");
+}
+// One arrival on a barrier of the peer.
+__device__ __forceinline__ void mbar_arrive_peer(uint32_t addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(addr) : "memory");
+}
+// mbar_wait() whose acquire spans the cluster: the barrier also counts bytes the peer CTA sends.
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, uint32_t* dev_status, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    if (done) return true;
+    if ((it & 1023u) == 1023u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  if (dev_status) atomicOr(dev_status, kStatusTimeout);
+  return false;
+}
+
 // 64 fp32 of a tensor-memory row -> one 128-byte bf16 row of a swizzled shared-memory tile, scaled.
 __device__ __forceinline__ void row_to_smem(uint32_t taddr, uint8_t* tile, int row, float scale) {
 #pragma unroll
@@ -117,7 +164,7 @@ __device__ __forceinline__ void row_to_smem(uint32_t taddr, uint8_t* tile, int r
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-block_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const FParams p, uint32_t* dev_status) {
+block_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_out, const FParams p, uint32_t* dev_status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sKV = smem;                           // [D][128 B]: merged tokens of the head, K-major rows
@@ -130,21 +177,19 @@ block_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const FParams p, ui
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int unit = blockIdx.x % p.units, bh = blockIdx.x / p.units, h = bh % p.heads, b = bh / p.heads;
-  const int n_pairs = p.P / 2;          // pairs of tiles merged in phase A
+  constexpr int n_pairs = 4;            // pairs of tiles this CTA merges (its unit's 8 tiles) and unmerges
   const int nblk = p.D / kBN;           // key tiles
   const int tiles_x = p.tiles_x;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < 4; ++s) {
       mbar_init(&bar->x_full[s], 1);
-      mbar_init(&bar->x_empty[s], 1);
     }
     mbar_init(&bar->slab2_full, 4);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bar->slab_full[s], 4);
       mbar_init(&bar->slab_empty[s], 1);
       mbar_init(&bar->acc_full[s], 1);
-      mbar_init(&bar->acc_empty[s], 4);
       mbar_init(&bar->o_done[s], 1);
       mbar_init(&bar->os_full[s], 4);
       for (int t = 0; t < 2; ++t) {
@@ -154,10 +199,13 @@ block_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const FParams p, ui
       }
     }
     for (int s = 0; s < 4; ++s) mbar_init(&bar->pv_done[s], 1);
-    mbar_init(&bar->kv_ready, 4);
+    mbar_init(&bar->kv_ready, p.units == 2 ? 5 : 4);  // own warps; the peer's rows arrive as bytes
     bar->abort_flag = 0;
     mbar_fence_init();
+    mbar_init(&bar->kv_sent, 1);
+    if (p.units == 2) mbar_expect_tx(&bar->kv_ready, 2 * kPairBytes);
     prefetch_tmap(&tm_x);
+    prefetch_tmap(&tm_out);
   }
   for (int e = threadIdx.x; e < kOnesBytes / 4; e += blockDim.x) reinterpret_cast<uint32_t*>(sOnes)[e] = 0x3F803F80u;
   for (int e = threadIdx.x; e < kZeroBytes / 4; e += blockDim.x) {
@@ -171,6 +219,7 @@ block_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const FParams p, ui
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (p.units == 2) cluster_sync();  // the peer's barriers are initialised before anything is sent to it
   const uint32_t tmem = bar->tmem_base;
   volatile int* abort_flag = &bar->abort_flag;
   // tensor memory: columns 0..255 the four S buffers (the merge accumulators before, the unmerge accumulators
@@ -181,11 +230,10 @@ block_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const FParams p, ui
     // ------------------------------------------------------------------ A: token tiles of every pair
     if (elect_one()) {
       for (int i = 0; i < n_pairs; ++i) {
-        const int s = i & 3;
-        if (i >= 4 && !mbar_wait(&bar->x_empty[s], ((i >> 2) - 1) & 1, dev_status, abort_flag)) break;
+        const int s = i;
         mbar_expect_tx(&bar->x_full[s], kPairBytes);
         for (int t = 0; t < 2; ++t) {
-          const int tile = 2 * i + t, ty = tile / tiles_x, tx = tile - ty * tiles_x;
+          const int tile = unit * 8 + 2 * i + t, ty = tile / tiles_x, tx = tile - ty * tiles_x;
           tma_load_4d(sX + s * kPairBytes + t * (kPairBytes / 2), &tm_x, &bar->x_full[s], h * 64, tx * p.tw, ty * p.th, b);
         }
       }
@@ -197,13 +245,12 @@ block_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const FParams p, ui
       // ---- A: X_m rows of four tiles = (pair 0 | zeros) and (zeros | pair 1) times the tokens of the pairs
       constexpr uint32_t idesc_m = idesc_f16(kFmtBF16, kFmtBF16, true, true, 128, 64);
       for (int i = 0; ok && i < n_pairs; ++i) {
-        const int s = i & 1, xs = i & 3, g = i >> 1;  // slab stage; token stage; group of four tiles
-        if ((i & 1) == 0 && g >= 2 && !mbar_wait(&bar->acc_empty[g & 1], ((g >> 1) - 1) & 1, dev_status, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(&bar->x_full[xs], (i >> 2) & 1, dev_status, abort_flag) ||
+        const int s = i & 1, xs = i, g = i >> 1;  // slab stage; token stage; group of four tiles
+        if (!mbar_wait(&bar->x_full[xs], 0, dev_status, abort_flag) ||
             !mbar_wait(&bar->slab_full[s], (i >> 1) & 1, dev_status, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t xa = smem_u32(sX + xs * kPairBytes);
-        const uint32_t t_acc = tmem + (g & 1) * 64;
+        const uint32_t t_acc = tmem + g * 64;
 #pragma unroll
         for (int pl = 0; pl < 2; ++pl) {
           const uint32_t sa = smem_u32(sA + (2 * s + pl) * kPairBytes);
@@ -216,13 +263,13 @@ block_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const FParams p, ui
             mma_ss(t_acc, ad, smem_desc_sw128(xa + kk * 2048, 16, 1024), idesc_m, (i & 1) != 0 || pl > 0 || kk > 0);
           }
         }
-        mma_commit(&bar->x_empty[xs]);
         mma_commit(&bar->slab_empty[s]);
-        if (i & 1) mma_commit(&bar->acc_full[g & 1]);
+        if (i & 1) mma_commit(&bar->acc_full[g]);
       }
       // ---- B: attention of the unit's two query tiles over all D keys of the resident matrix
-      if (ok) ok = mbar_wait(&bar->kv_ready, 0, dev_status, abort_flag);
+      if (ok) ok = mbar_wait_cluster(&bar->kv_ready, 0, dev_status, abort_flag);
       if (ok) {
+        if (p.units == 2) mbar_arrive_peer(peer_addr(smem_u32(&bar->kv_sent), (uint32_t)(unit ^ 1)));
         tc_fence_after();
         constexpr uint32_t idesc_s = idesc_f16(kFmtBF16, kFmtBF16, false, false, kBM, kBN);
         constexpr uint32_t idesc_o = idesc_f16(kFmtBF16, kFmtBF16, false, true, kBM, 64 + 16);
@@ -291,12 +338,14 @@ block_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const FParams p, ui
     if (q == 0) {
       // slabs of all pairs, then (same stages, same barriers) of the first two pairs of the unmerge; a pair's
       // weights are requested before the wait for its stage, so that their latency passes under it
-      const int n_build = n_pairs + 2;
-      SlabRow w = load_slab_row(p, b, 0, r);
+      constexpr int n_build = n_pairs + 2;
+      SlabRow w0 = load_slab_row(p, b, unit * 8, r), w1 = load_slab_row(p, b, unit * 8 + 2, r);
+#pragma unroll
       for (int i = 0; i < n_build; ++i) {
         const int s = i & 1;
-        const SlabRow cur = w;
-        if (i + 1 < n_build) w = load_slab_row(p, b, i + 1 < n_pairs ? 2 * (i + 1) : unit * 8 + 2 * (i + 1 - n_pairs), r);
+        const SlabRow cur = w0;
+        w0 = w1;
+        if (i + 2 < n_build) w1 = load_slab_row(p, b, unit * 8 + 2 * ((i + 2) % n_pairs), r);
         if (i >= 2 && !mbar_wait(&bar->slab_empty[s], ((i >> 1) - 1) & 1, dev_status, abort_flag)) { ok = false; break; }
         store_slab_row(sA + 2 * s * kPairBytes, cur, r);
         fence_proxy_async();
@@ -305,17 +354,17 @@ block_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const FParams p, ui
       }
     } else {
       // merged rows of every group of four tiles: tensor memory -> bf16 rows of the shared matrix
-      const int n_groups = n_pairs / 2;
-      for (int g = 0; g < n_groups; ++g) {
-        if (!mbar_wait(&bar->acc_full[g & 1], (g >> 1) & 1, dev_status, abort_flag)) { ok = false; break; }
+      const uint32_t peer = (uint32_t)(unit ^ 1);
+      for (int g = 0; g < n_pairs / 2; ++g) {
+        if (!mbar_wait(&bar->acc_full[g], 0, dev_status, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        row_to_smem(tmem + lane_addr + (g & 1) * 64, sKV + g * kPairBytes, r, 1.f);
-        tc_fence_before();
+        uint8_t* rows = sKV + (unit * 2 + g) * kPairBytes + quarter * 4096;  // this warp's 32 rows
+        row_to_smem(tmem + lane_addr + g * 64, sKV + (unit * 2 + g) * kPairBytes, r, 1.f);
+        fence_proxy_async();  // read by the tensor cores and by the copy
         __syncwarp();
-        if (lane == 0) mbar_arrive(&bar->acc_empty[g & 1]);
+        if (p.units == 2 && lane == 0) copy_to_peer(peer_addr(smem_u32(rows), peer), rows, 4096, peer_addr(smem_u32(&bar->kv_ready), peer));
       }
-      fence_proxy_async();  // the matrix is read by the tensor cores
-      __syncwarp();
+      tc_fence_before();
       if (lane == 0) mbar_arrive(&bar->kv_ready);
       // the unmerge's third pair, into the token stages 2 and 3: every merge MMA has completed (the last group's
       // accumulator was complete), so nothing reads them any more
@@ -342,6 +391,8 @@ block_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const FParams p, ui
       if (lane == 0) mbar_arrive(&bar->p_full[q][bb]);
     }
     // normalised accumulator -> bf16 rows in shared memory (the unmerge's B operand)
+    SlabRow w3;
+    if (q == 1) w3 = load_slab_row(p, b, unit * 8 + 6, r);  // the unmerge's fourth pair; needed after the next wait
     if (ok) ok = mbar_wait(&bar->o_done[q], 0, dev_status, abort_flag);
     if (ok) {
       tc_fence_after();
@@ -357,30 +408,30 @@ block_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const FParams p, ui
     // ------------------------------------------------------------------ C
     if (ok && q == 1) {  // the fourth pair's slab takes the stage of the first once its MMAs are done
       const int gi = n_pairs + 2, s = gi & 1;
-      const SlabRow w = load_slab_row(p, b, unit * 8 + 6, r);
       ok = mbar_wait(&bar->slab_empty[s], ((gi >> 1) - 1) & 1, dev_status, abort_flag);
       if (ok) {
-        store_slab_row(sA + 2 * s * kPairBytes, w, r);
+        store_slab_row(sA + 2 * s * kPairBytes, w3, r);
         fence_proxy_async();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bar->slab_full[s]);
       }
     }
+    // the rows of K and V become the staging area of the output; the peer must have received its copy of them
+    if (ok && p.units == 2) ok = mbar_wait_cluster(&bar->kv_sent, 0, dev_status, abort_flag);
     for (int c = 2 * q; ok && c < 2 * q + 2; ++c) {
       if (!mbar_wait(&bar->c_full[q][c & 1], 0, dev_status, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const int tile = unit * 8 + 2 * c + (r >> 6);
-      const int tok = tile_token(tile, r & 63, tiles_x, p.th, p.tw, p.W);
-      __nv_bfloat16* dst = p.out + ((size_t)b * p.n_all + tok) * p.d + h * 64;
-      const uint32_t t_c = tmem + lane_addr + (2 * q + (c & 1)) * kBN;
-#pragma unroll
-      for (int cc = 0; cc < 2; ++cc) {
-        uint32_t v[32];
-        tmem_ld32(t_c + cc * 32, v);
-        tmem_wait_ld();
-        store_row32(dst + cc * 32, v, 1.f);
+      uint8_t* stage = sKV + c * kPairBytes;  // K and V are no longer read: every MMA before this accumulator's has completed
+      row_to_smem(tmem + lane_addr + (2 * q + (c & 1)) * kBN, stage, r, 1.f);
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) {  // the warp's 32 tokens are the upper or lower half of a tile
+        const int tile = unit * 8 + 2 * c + (quarter >> 1), ty = tile / tiles_x, tx = tile - ty * tiles_x;
+        tma_store_4d(&tm_out, stage + quarter * 4096, h * 64, tx * p.tw, ty * p.th + (quarter & 1) * (p.th / 2), b);
+        tma_store_commit();
       }
     }
+    if (lane == 0) tma_store_wait_read();  // shared memory must outlive the engine's reads
   }
   tc_fence_before();
   __syncthreads();
@@ -388,6 +439,7 @@ block_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const FParams p, ui
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }
+  if (p.units == 2) cluster_sync();  // neither CTA's shared memory goes away while the other could still write to it
 }
 
 constexpr int kFusedSmem = 1024 + kMaxD * 128 + 4 * kPairBytes + 2 * kZeroBytes + 4 * kPairBytes + kOnesBytes + 512;
@@ -398,28 +450,28 @@ constexpr int kFusedSmem = 1024 + kMaxD * 128 + 4 * kPairBytes + 2 * kZeroBytes 
 bool block_fused_supported(const Geom& g) {
   if (g.f32 || g.global_merge || g.n_extra != 0 || g.unmerge_mode != TOMA_UNMERGE_TRANSPOSE) return false;
   if (g.dh != 64 || g.Nloc != kTileTok || g.Dloc != kTileDest) return false;
-  if (g.tw > 64 || 64 % g.tw != 0 || g.th != 64 / g.tw) return false;  // a tile is one 4-D TMA box of 64 tokens
+  if (g.tw > 32 || 64 % g.tw != 0 || g.th != 64 / g.tw) return false;  // a tile is one 4-D TMA box of 64 tokens, half a tile a box too
   if (g.D > kMaxD || g.D % 256 != 0 || g.P % 4 != 0) return false;     // whole 256-query units, whole groups of four tiles
   return true;
 }
 
 cudaError_t launch_block_fused(const Geom& g, const void* w, const void* x, void* out, uint32_t* dev_status, cudaStream_t s) {
   static_assert(sizeof(FBars) <= 512, "barrier block outgrew its reservation");
-  CUtensorMap tx;
+  CUtensorMap tx, to;
   const uint64_t dims[4] = {(uint64_t)g.d, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.B};
   const uint64_t strides[3] = {(uint64_t)g.d * 2, (uint64_t)g.W * g.d * 2, (uint64_t)g.tokens_all() * g.d * 2};
   const uint32_t box[4] = {64, (uint32_t)g.tw, (uint32_t)g.th, 1};
-  if (!encode_tmap_16bit(&tx, x, 4, dims, strides, box)) return cudaErrorInvalidValue;
+  const uint32_t box_out[4] = {64, (uint32_t)g.tw, (uint32_t)g.th / 2, 1};  // a warp stores half a tile
+  if (!encode_tmap_16bit(&tx, x, 4, dims, strides, box) || !encode_tmap_16bit(&to, out, 4, dims, strides, box_out)) return cudaErrorInvalidValue;
   FParams p;
-  p.P = g.P; p.tiles_x = g.tiles_x; p.th = g.th; p.tw = g.tw; p.W = g.W; p.d = g.d; p.n_all = (int)g.tokens_all();
+  p.tiles_x = g.tiles_x; p.th = g.th; p.tw = g.tw;
   p.heads = g.heads; p.D = g.D; p.units = g.D / 256;
   p.w = (const __nv_bfloat16*)w;
-  p.out = (__nv_bfloat16*)out;
   p.scale_log2 = 1.4426950408889634f / 8.0f;  // log2(e) / sqrt(64)
   static std::atomic<unsigned long long> raised{0};
   cudaError_t e = raise_dynamic_smem(block_fused_kernel, kFusedSmem, raised);
   if (e != cudaSuccess) return e;
-  e = launch_dependent(block_fused_kernel, dim3(g.B * g.heads * p.units), dim3(kThreads), (size_t)kFusedSmem, s, tx, p, dev_status);
+  e = launch_dependent_cluster(block_fused_kernel, dim3(g.B * g.heads * p.units), dim3(kThreads), (size_t)kFusedSmem, p.units, s, tx, to, p, dev_status);
   if (e != cudaSuccess) return e;
   count_launch();
   return cudaGetLastError();
