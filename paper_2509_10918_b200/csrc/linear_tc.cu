@@ -274,14 +274,15 @@ unmerge_tc_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constan
 // as they are, the attended rows an MN-major B operand (two MMAs along N: at most 192 + 128 channels).
 // Against channels on M (128 x 128 tiles) a k-step moves 72 KB for 10.5 MFLOP instead of 48 KB for
 // 4.2 MFLOP, the weights are read twice instead of five times, and the 128 CTAs of the 64x64-token
-// case fit the SMs in one wave with a three-stage pipeline; each thread then owns a token row and
-// writes its channels as one contiguous run.
+// case fit the SMs in one wave with a three-stage pipeline; each thread then owns a token row, which it
+// stages in shared memory (the pipeline's stages, free by then) as 64-channel slabs in the layout of the
+// output tensor map's box: the CTA's 128 tokens are whole tile rows, one TMA store per slab.
 // ------------------------------------------------------------------------------------------------
 constexpr int kRowsChBlock = 320;  // channels per CTA (five 64-channel slabs)
 
 __global__ void __launch_bounds__(192, 1)
 unmerge_rows_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_w,
-                    __nv_bfloat16* __restrict__ out, const LinParams p, uint32_t* dev_status) {
+                    const __grid_constant__ CUtensorMap tm_o, const LinParams p, uint32_t* dev_status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -303,6 +304,7 @@ unmerge_rows_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_const
     pipe_init(bar, p.stages);
     prefetch_tmap(&tm_y);
     prefetch_tmap(&tm_w);
+    prefetch_tmap(&tm_o);
   }
   dependency_wait();
   if (threadIdx.x == 0) release_dependents();
@@ -356,12 +358,12 @@ unmerge_rows_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_const
     const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16);
     if (mbar_wait(&bar->done, 0, dev_status, abort_flag)) {
       tc_fence_after();
-      const size_t tok = (size_t)tile_token(tile, t0 + row, p.tiles_x, p.th, p.tw, p.W);
-      __nv_bfloat16* dst = out + ((size_t)b * p.n_all + tok) * p.d + c0;
+      // every load has been consumed: slab c of the output, [128 tokens][128 B] swizzled, goes to smem + c * 16 KB
       for (int c = 0; c < n_ch; c += 32) {  // accumulator column = channel (the second accumulator starts at 192)
         uint32_t r[32];
         tmem_ld32(taddr + c, r);
         tmem_wait_ld();
+        uint8_t* slab = smem + (c >> 6) * (128 * 128);
 #pragma unroll
         for (int e = 0; e < 32; e += 8) {
           if (c + e < n_ch) {
@@ -369,9 +371,19 @@ unmerge_rows_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_const
 #pragma unroll
             for (int u = 0; u < 4; ++u)
               q[u] = __floats2bfloat162_rn(__uint_as_float(r[e + 2 * u]), __uint_as_float(r[e + 2 * u + 1]));
-            *reinterpret_cast<uint4*>(dst + c + e) = *reinterpret_cast<const uint4*>(q);
+            *reinterpret_cast<uint4*>(slab + sw128_offset(row, ((c & 63) + e) >> 3)) = *reinterpret_cast<const uint4*>(q);
           }
         }
+      }
+      fence_proxy_async();  // the staged rows are read by the TMA engine
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar->epi);
+      if (row == 0 && mbar_wait(&bar->epi, 0, dev_status, abort_flag)) {
+        const int ty = tile / p.tiles_x, tx = tile - ty * p.tiles_x;
+        for (int c = 0; c < slabs; ++c)  // a slab cut short by the channel count is clipped by the store
+          tma_store_4d(&tm_o, smem + c * (128 * 128), c0 + c * 64, tx * p.tw, ty * p.th + t0 / p.tw, b);
+        tma_store_commit();
+        tma_store_wait_read();  // shared memory must outlive the engine's reads
       }
     }
   }
@@ -491,13 +503,19 @@ cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void*
     const int stage_bytes = 2 * 128 * 128 + slabs * kSlab;
     p.stages = (224 * 1024) / stage_bytes;
     p.stages = p.stages > 4 ? 4 : p.stages < 2 ? 2 : p.stages;
-    if (p.stages > (g.Dloc + kKC - 1) / kKC) p.stages = (g.Dloc + kKC - 1) / kKC;
+    // never fewer than two: the stages double as the staging area of the output (slabs x 16 KB <= 2 stages)
+    if (p.stages > (g.Dloc + kKC - 1) / kKC) p.stages = (g.Dloc + kKC - 1) / kKC < 2 ? 2 : (g.Dloc + kKC - 1) / kKC;
     const int smem = 1024 + p.stages * stage_bytes + 256;
     static std::atomic<unsigned long long> raised_r{0};
     if (cudaError_t e = raise_dynamic_smem(unmerge_rows_kernel, 227 * 1024, raised_r); e != cudaSuccess) return e;
+    // output tokens as (channel, x, y, batch): a CTA's 128 tokens are 128 / tile_w whole tile rows
+    CUtensorMap to;
+    const uint64_t odims[4] = {(uint64_t)g.d, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.B};
+    const uint64_t ostrides[3] = {(uint64_t)g.d * 2, (uint64_t)g.W * g.d * 2, (uint64_t)g.tokens_all() * g.d * 2};
+    const uint32_t obox[4] = {64, (uint32_t)g.tw, (uint32_t)(128 / g.tw), 1};
+    if (!encode_tmap_16bit(&to, out, 4, odims, ostrides, obox)) return cudaErrorInvalidValue;
     dim3 grid(g.B * g.P * (g.Nloc / 128), (g.d + kRowsChBlock - 1) / kRowsChBlock);
-    cudaError_t e = launch_dependent(unmerge_rows_kernel, grid, dim3(192), (size_t)smem, s, ty, tw128, (__nv_bfloat16*)out, p,
-                                     dev_status);
+    cudaError_t e = launch_dependent(unmerge_rows_kernel, grid, dim3(192), (size_t)smem, s, ty, tw128, to, p, dev_status);
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
   }
