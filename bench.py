@@ -282,7 +282,7 @@ class Workload:
     def block(self, step):
         self.toma.toma_block(self.desc, step, self.x, self.out, self.idx, self.w, self.ws, self.status)
 
-    # algorithmic bytes / flops per launch ("Kernels and what bounds them")
+    # algorithmic bytes / flops per launch
     def esz(self):
         return 2 if self.cfg.dtype == "bf16" else 4
 

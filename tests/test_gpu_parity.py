@@ -285,8 +285,10 @@ def test_block_sequence_parity(toma, name, over, _):
 
 
 @pytest.mark.parametrize("over", [dict(), dict(batch=1, grid_h=32, grid_w=16, dim=128, n_heads=2),
-                                  dict(batch=3, grid_h=16, grid_w=32, tile_h=4, tile_w=16, dim=640, n_heads=10)],
-                         ids=["cfg2", "256-merged-tokens", "4x16-tiles"])
+                                  dict(batch=3, grid_h=16, grid_w=32, tile_h=4, tile_w=16, dim=640, n_heads=10),
+                                  dict(batch=1, grid_h=32, grid_w=16, tile_h=16, tile_w=4, dim=128, n_heads=2),
+                                  dict(batch=2, grid_h=16, grid_w=64, tile_h=2, tile_w=32, dim=256, n_heads=4)],
+                         ids=["cfg2", "256-merged-tokens", "4x16-tiles", "16x4-tiles", "2x32-tiles"])
 def test_block_one_kernel_reuse_step_parity(toma, tuning, over):
     """Shapes with 64-token tiles, 32 destinations and at most 512 merged tokens run merge, attention and unmerge of
     a step as ONE kernel.  Both forms of the step (one kernel; three kernels, forced through the test-only
