@@ -345,7 +345,7 @@ static toma_status block_impl(const toma_desc* desc, int32_t step, const void* x
   if (refresh_sel) e = do_select(g, x, idx_state, wsb, dev_status, s);
   if (e == cudaSuccess && refresh_w) e = do_weights(g, x, idx_state, w_state, wsb, dev_status, s);
   // merge, attention and unmerge as one kernel where the shape allows (small tiles, few merged tokens)
-  if (!proj && !mlp && block_fused_supported(g) && !g_tune_block_unfused.load(std::memory_order_relaxed)) {
+  if (!proj && !mlp && block_fused_supported(g) && !g_tune_block_unfused.load(std::memory_order_relaxed) && block_fused_launchable(g)) {
     if (e == cudaSuccess) e = launch_block_fused(g, w_state, x, out, dev_status, s);
     return cuda_ok(e);
   }

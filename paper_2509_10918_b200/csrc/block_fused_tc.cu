@@ -455,6 +455,38 @@ bool block_fused_supported(const Geom& g) {
   return true;
 }
 
+// Whether this device can hold the kernel's launch at all: the shared memory of one CTA and, for 512 merged
+// tokens, two such CTAs as a cluster.  Asked once per device (a host-side occupancy query, nothing is launched);
+// toma_block takes the three-kernel form where the answer is no.
+bool block_fused_launchable(const Geom& g) {
+  static std::atomic<unsigned long long> raised{0};
+  static std::atomic<int> answer[64][2];  // per device and cluster size - 1: 0 unknown, 1 yes, 2 no
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+  const int units = g.D / 256;
+  const int known = answer[dev][units - 1].load(std::memory_order_relaxed);
+  if (known) return known == 1;
+  bool ok = raise_dynamic_smem(block_fused_kernel, kFusedSmem, raised) == cudaSuccess;
+  if (ok) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * units);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kFusedSmem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)units;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    ok = cudaOccupancyMaxActiveClusters(&clusters, block_fused_kernel, &cfg) == cudaSuccess && clusters >= 1;
+  }
+  if (!ok) (void)cudaGetLastError();  // a failed query is an answer, not an error of the caller's stream
+  answer[dev][units - 1].store(ok ? 1 : 2, std::memory_order_relaxed);
+  return ok;
+}
+
 cudaError_t launch_block_fused(const Geom& g, const void* w, const void* x, void* out, uint32_t* dev_status, cudaStream_t s) {
   static_assert(sizeof(FBars) <= 512, "barrier block outgrew its reservation");
   CUtensorMap tx, to;

@@ -104,6 +104,7 @@ cudaError_t launch_attention_tc(int B, int L, int heads, int dh, const void* q, 
                                 void* ws, bool tickets_clean, uint32_t* dev_status, cudaStream_t s);
 // The reuse step (merge, attention over the merged tokens, unmerge) as one kernel, for the shapes it is written for.
 bool block_fused_supported(const Geom& g);
+bool block_fused_launchable(const Geom& g);  // this device holds its launch (host-side query, cached per device)
 cudaError_t launch_block_fused(const Geom& g, const void* w, const void* x, void* out, uint32_t* dev_status, cudaStream_t s);
 // Image-level destination ids [batch][D] (tile-major, pick order) from the tile-local picks.
 cudaError_t launch_global_idx(const Geom& g, const int32_t* idx, int32_t* gidx, cudaStream_t s);
