@@ -519,16 +519,36 @@ softmax_rows_kernel(float* __restrict__ shares, float* __restrict__ zblk, int Nl
   }
 }
 
-// z[batch][i] = sum over the row blocks of zblk, in block order.
+// z[batch][i] = sum over the row blocks of zblk.  A CTA takes 32 destinations; its eight warps each add an eighth
+// of the blocks in block order (four loads in flight at a time), and the eight partial sums are added in warp
+// order: a fixed association, so the result does not depend on scheduling, and the chain of dependent loads is
+// an eighth as long as one thread per destination would make it.
 __global__ void __launch_bounds__(256) z_reduce_kernel(const float* __restrict__ zblk, float* __restrict__ z, int nblk, int Dloc) {
+  __shared__ float part[8][32];
   dependency_wait();
   if (threadIdx.x == 0) release_dependents();
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= Dloc) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int i = blockIdx.x * 32 + lane;
   const size_t batch = blockIdx.y;
+  const int per = (nblk + 7) / 8, b0 = warp * per, b1 = min(nblk, b0 + per);
   float acc = 0.f;
-  for (int b = 0; b < nblk; ++b) acc += zblk[(batch * nblk + b) * Dloc + i];
-  z[batch * Dloc + i] = acc;
+  if (i < Dloc) {
+    const float* src = zblk + batch * nblk * Dloc + i;
+    int b = b0;
+    for (; b + 4 <= b1; b += 4) {
+      const float v0 = src[(size_t)b * Dloc], v1 = src[(size_t)(b + 1) * Dloc], v2 = src[(size_t)(b + 2) * Dloc], v3 = src[(size_t)(b + 3) * Dloc];
+      acc = (((acc + v0) + v1) + v2) + v3;
+    }
+    for (; b < b1; ++b) acc += src[(size_t)b * Dloc];
+  }
+  part[warp][lane] = acc;
+  __syncthreads();
+  if (warp == 0 && i < Dloc) {
+    float t = part[0][lane];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) t += part[w][lane];
+    z[batch * Dloc + i] = t;
+  }
 }
 
 }  // namespace
@@ -630,7 +650,7 @@ cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, 
                           zblk, g.Nloc, g.Dloc);
     count_launch();
     if (le != cudaSuccess) return le;
-    le = launch_dependent(z_reduce_kernel, dim3((unsigned)((g.Dloc + 255) / 256), (unsigned)tiles), dim3(256), 0, s,
+    le = launch_dependent(z_reduce_kernel, dim3((unsigned)((g.Dloc + 31) / 32), (unsigned)tiles), dim3(256), 0, s,
                           (const float*)zblk, z, nrb, g.Dloc);
     count_launch();
     if (le != cudaSuccess) return le;
