@@ -188,13 +188,16 @@ template <bool kSmemS>
 __global__ void __launch_bounds__(1024) greedy_kernel(const int16_t* __restrict__ sq, int32_t* __restrict__ idx,
                                                       int Nloc, int Dloc) {
   extern __shared__ __align__(16) uint8_t greedy_smem[];
-  __shared__ int2 changed[2][kMaxNloc];  // (column j, new << 16 | old & 0xffff) of columns whose cached maximum improved
+  // (column j, new << 16 | old & 0xffff) of columns whose cached maximum improved; cleared at the start and padded,
+  // so that the entries behind a list's end are readable and name a valid column
+  __shared__ int2 changed[2][kMaxNloc + 4];
   __shared__ ArgMax red[2][32];
   __shared__ __align__(16) int keys[2][8];  // warp keys of block_argmax_packed (unused slots stay -1)
   __shared__ int n_changed[2];
   const int16_t* Sg = sq + (size_t)blockIdx.x * Nloc * Nloc;
   const int16_t* S = Sg;
   if (threadIdx.x == 0) n_changed[0] = n_changed[1] = 0;
+  for (int e = threadIdx.x; e < 2 * (kMaxNloc + 4); e += blockDim.x) (&changed[0][0])[e] = make_int2(0, 0);
   if (threadIdx.x < 16) keys[threadIdx.x >> 3][threadIdx.x & 7] = -1;
   tc::dependency_wait();  // launched with programmatic stream serialisation
   if (threadIdx.x == 0) tc::release_dependents();
@@ -239,10 +242,10 @@ __global__ void __launch_bounds__(1024) greedy_kernel(const int16_t* __restrict_
       selected = true;
       out[r] = pick.i;
     }
-    // columns whose cached maximum improves, compacted into a list (one shared-memory atomic per warp)
     const int s_new = live ? (int)S[(size_t)pick.i * Nloc + i] : 0;
     const bool ch = live && s_new > m_own;
     const unsigned mask = __ballot_sync(0xffffffffu, ch);
+    // columns whose cached maximum improves, compacted into a list (one shared-memory atomic per warp)
     if (mask) {
       int base = 0;
       if (lane == 0) base = atomicAdd(&n_changed[pb], __popc(mask));
@@ -269,10 +272,16 @@ __global__ void __launch_bounds__(1024) greedy_kernel(const int16_t* __restrict_
 #pragma unroll
         for (int u = 0; u < 4; ++u) gain += max(sv[u] - (c[u].y >> 16), 0) - max(sv[u] - (int)(short)(c[u].y & 0xFFFF), 0);
       }
-      for (; e < n; ++e) {
-        const int2 c = changed[pb][e];
-        const int sv = S[(size_t)c.x * Nloc + i];
-        gain += max(sv - (c.y >> 16), 0) - max(sv - (int)(short)(c.y & 0xFFFF), 0);
+      if (e < n) {  // up to three left: fetched together whether they exist or not, counted only if they do
+        int2 c[3];
+        int sv[3];
+#pragma unroll
+        for (int u = 0; u < 3; ++u) c[u] = changed[pb][e + u];
+#pragma unroll
+        for (int u = 0; u < 3; ++u) sv[u] = S[(size_t)c[u].x * Nloc + i];
+#pragma unroll
+        for (int u = 0; u < 3; ++u)
+          gain += (e + u < n) ? max(sv[u] - (c[u].y >> 16), 0) - max(sv[u] - (int)(short)(c[u].y & 0xFFFF), 0) : 0;
       }
     }
   }
