@@ -342,10 +342,18 @@ static toma_status block_impl(const toma_desc* desc, int32_t step, const void* x
   const bool refresh_sel = step % desc->reuse_interval == 0;
   const bool refresh_w = refresh_sel || step % kw == 0;
   cudaError_t e = cudaSuccess;
-  if (refresh_sel) e = do_select(g, x, idx_state, wsb, dev_status, s);
-  if (e == cudaSuccess && refresh_w) e = do_weights(g, x, idx_state, w_state, wsb, dev_status, s);
+  const bool unfused = g_tune_block_unfused.load(std::memory_order_relaxed) != 0;
+  if (refresh_sel && refresh_w && refresh_fused_supported(g) && !unfused) {
+    // small tiles: Gram, greedy rounds and weights of a tile in one kernel behind the quantisation
+    __nv_bfloat16* y = (__nv_bfloat16*)(wsb + l.y_off);
+    e = launch_quantise(g, x, y, s);
+    if (e == cudaSuccess) e = launch_refresh_fused(g, y, x, idx_state, w_state, dev_status, s);
+  } else {
+    if (refresh_sel) e = do_select(g, x, idx_state, wsb, dev_status, s);
+    if (e == cudaSuccess && refresh_w) e = do_weights(g, x, idx_state, w_state, wsb, dev_status, s);
+  }
   // merge, attention and unmerge as one kernel where the shape allows (small tiles, few merged tokens)
-  if (!proj && !mlp && block_fused_supported(g) && !g_tune_block_unfused.load(std::memory_order_relaxed) && block_fused_launchable(g)) {
+  if (!proj && !mlp && block_fused_supported(g) && !unfused && block_fused_launchable(g)) {
     if (e == cudaSuccess) e = launch_block_fused(g, w_state, x, out, dev_status, s);
     return cuda_ok(e);
   }

@@ -48,7 +48,8 @@ inline void count_launch(int n = 1) { g_launches.fetch_add((unsigned long long)n
 // Test-only overrides of launch heuristics (set through toma_test_set_tuning; the product path never
 // writes them): attention work plan (-1 = heuristic, 0 = whole units, 1 = even cut), persistent CTA
 // count of the attention kernel (0 = heuristic), tile form of the projection kernel (0 = heuristic), 1 = toma_block
-// takes the three-kernel path even where the fused reuse-step kernel applies.
+// takes the three-kernel path even where the fused reuse-step kernel applies, and the separate selection and
+// weights kernels where the one-kernel refresh of small tiles applies.
 extern std::atomic<int> g_tune_attention_split, g_tune_attention_ctas, g_tune_linear_tile, g_tune_block_unfused;
 
 // Number of SMs of the current device (cached per device).
@@ -104,7 +105,12 @@ cudaError_t launch_attention_tc(int B, int L, int heads, int dh, const void* q, 
                                 void* ws, bool tickets_clean, uint32_t* dev_status, cudaStream_t s);
 // The reuse step (merge, attention over the merged tokens, unmerge) as one kernel, for the shapes it is written for.
 bool block_fused_supported(const Geom& g);
-bool block_fused_launchable(const Geom& g);  // this device holds its launch (host-side query, cached per device)
+bool block_fused_launchable(const Geom& g);
+// Selection and merge weights of 64-token tiles in one kernel (after launch_quantise), for the shapes it is written for.
+bool refresh_fused_supported(const Geom& g);
+cudaError_t launch_refresh_fused(const Geom& g, const __nv_bfloat16* y, const void* x, int32_t* idx, void* w, uint32_t* dev_status,
+                                 cudaStream_t s);
+//  // this device holds its launch (host-side query, cached per device)
 cudaError_t launch_block_fused(const Geom& g, const void* w, const void* x, void* out, uint32_t* dev_status, cudaStream_t s);
 // Image-level destination ids [batch][D] (tile-major, pick order) from the tile-local picks.
 cudaError_t launch_global_idx(const Geom& g, const int32_t* idx, int32_t* gidx, cudaStream_t s);

@@ -316,9 +316,63 @@ def test_block_one_kernel_reuse_step_parity(toma, tuning, over):
             assert np.array_equal(idx.cpu().numpy().astype(np.int64), st.idx)
             assert_close(to_host64(out), want, cfg.dtype, f"block step {step}, {'three kernels' if unfused else 'one kernel'}")
             outs[(unfused, step)] = to_host64(out)
+            if step == 0:
+                # the refresh step's weights themselves (one kernel does Gram, greedy rounds and weights of a tile
+                # when the step is not forced onto the separate kernels): every tile against Sec. 4.2.1
+                dense = torch.empty((cfg.batch, cfg.n_tiles, gd(toma, cfg), cfg.n_loc), dtype=torch.float32, device="cuda")
+                toma.toma_weights_export(desc, w, dense)
+                torch.cuda.synchronize()
+                dense = dense.cpu().numpy().astype(np.float64)
+                ids = O.tile_token_ids(cfg.grid_h, cfg.grid_w, cfg.tile_h, cfg.tile_w)
+                for b_ in range(cfg.batch):
+                    for p_ in range(cfg.n_tiles):
+                        xt = x_host[b_][ids[p_]].astype(np.float64)
+                        assert np.abs(dense[b_, p_] - O.merge_weights(xt, st.idx[b_, p_], cfg.tau)).max() <= 6e-4, (b_, p_)
         assert launches[1] == (3 if unfused else 1), f"reuse step launched {launches[1]} kernels"
     for step in (0, 1):
         assert np.abs(outs[(0, step)] - outs[(1, step)]).max() <= 2 ** -6, "the two forms of the step disagree"
+
+
+@pytest.mark.parametrize("over", [dict(merge_ratio=0.25), dict(merge_ratio=0.75), dict(merge_ratio=0.875, tile_h=4, tile_w=16),
+                                  dict(merge_ratio=0.5, batch=1, dim=320, n_heads=5, n_extra=77)],
+                         ids=["48-destinations", "16-destinations", "8-destinations-4x16", "text-tokens"])
+def test_block_small_tile_refresh_kernel_parity(toma, tuning, over):
+    """A refresh step on 64-token tiles takes Gram, greedy rounds and weights of a tile in one kernel (whatever the
+    rest of the step runs as).  Indices bit-exact, weights and output against the oracle, for destination counts
+    and shapes the one-kernel reuse step does not cover; the same step forced onto the separate kernels agrees."""
+    cfg = gen.config("cfg2", steps=1, reuse_interval=1, **over)
+    desc = toma.desc_from_config(cfg)
+    kw = dict(grid_h=cfg.grid_h, grid_w=cfg.grid_w, tile_h=cfg.tile_h, tile_w=cfg.tile_w, merge_ratio=cfg.merge_ratio,
+              tau=cfg.tau, n_heads=cfg.n_heads, reuse_interval=1, n_extra=cfg.n_extra)
+    x_host = next(iter(gen.feature_sequence(cfg)))
+    want, _, _ = O.block_step(x_host, 0, (st := O.BlockState()), **kw)
+    assert min(st.margins) > O.FRAGILE_MARGIN
+    ids = O.tile_token_ids(cfg.grid_h, cfg.grid_w, cfg.tile_h, cfg.tile_w)
+    dense = {}
+    for separate in (0, 1):
+        tuning(block_unfused=separate)
+        idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        x = to_dev(x_host, cfg.dtype)
+        out = torch.full_like(x, float("nan"))
+        n0 = toma.toma_launch_counter()
+        toma.toma_block(desc, 0, x, out, idx, w, ws, status)
+        torch.cuda.synchronize()
+        launches = toma.toma_launch_counter() - n0
+        assert int(status.item()) == 0
+        assert np.array_equal(idx.cpu().numpy().astype(np.int64), st.idx)
+        assert_close(to_host64(out), want, cfg.dtype, "block output")
+        d = torch.empty((cfg.batch, cfg.n_tiles, gd(toma, cfg), cfg.n_loc), dtype=torch.float32, device="cuda")
+        toma.toma_weights_export(desc, w, d)
+        torch.cuda.synchronize()
+        dense[separate] = d.cpu().numpy().astype(np.float64)
+        for b_ in range(cfg.batch):
+            for p_ in range(cfg.n_tiles):
+                xt = x_host[b_][ids[p_]].astype(np.float64)
+                assert np.abs(dense[separate][b_, p_] - O.merge_weights(xt, st.idx[b_, p_], cfg.tau)).max() <= 6e-4, (b_, p_)
+        dense[("launches", separate)] = launches
+    assert dense[("launches", 0)] == dense[("launches", 1)] - 3, "selection and weights should have taken two launches instead of five"
+    assert np.abs(dense[0] - dense[1]).max() <= 6e-4
 
 
 def test_block_separate_weight_schedule_parity(toma):
