@@ -81,14 +81,14 @@ struct Barriers {
 };
 static_assert(sizeof(Barriers) <= 512, "barrier block outgrew its reservation");
 
+constexpr int kSnapTiles = 2;
 constexpr int kMaxCtas = 160;  // scratch and the span table are sized for this many persistent CTAs
 
 // The iterations [0, T) are cut into G contiguous spans, CTA g running [bounds[g], bounds[g + 1]).
 // With whole units every bound is a multiple of nblk (no scratch traffic), which wins when the unit
-// count happens to fill the CTAs evenly; otherwise the spans are cut at single key tiles, equal to
-// within one tile, and then every bound that falls within kSnapTiles of a unit boundary is moved
-// onto it: a piece of one or two tiles costs its CTA a whole pipeline drain and epilogue, more than
-// the tiles it moves are worth.
+// count happens to fill the CTAs evenly; otherwise the spans are cut at single key tiles so that the
+// longest span is as short as possible when every piece is charged its pipeline drain and epilogue
+// (plan_spans): a piece of one or two tiles costs its CTA more than the tiles it moves are worth.
 struct Spans {
   int T, G, nblk, split;
   int bounds[kMaxCtas + 1];
@@ -104,7 +104,6 @@ struct Spans {
     return lo;
   }
 };
-constexpr int kSnapTiles = 2;
 
 // One piece = the part of a span inside one unit: key tiles [k0, k0 + cnt) of unit u.
 struct Piece {
@@ -686,8 +685,48 @@ int max_ctas() {
 // partial results at the end of its span.
 constexpr int kSplitCostTiles = 4;
 
+// What a piece costs its CTA beyond its key tiles, in half tiles: the pipeline drains, the accumulator is read
+// out and (partial pieces) goes through scratch, tickets and the addition of the unit's pieces.
+constexpr int kPieceCostWhole = 4, kPieceCostPartial = 7;
+
+// The farthest end of a span that starts at iteration `start` and costs at most C half tiles
+// (2 per key tile plus the piece costs above); `start` itself when not even one tile fits.
+int span_end(int start, int T, int nblk, long long C) {
+  long long cost = 0;
+  int it = start;
+  while (it < T) {
+    const int k0 = it % nblk, room = nblk - k0;
+    const long long rest_of_unit = 2LL * room + (k0 ? kPieceCostPartial : kPieceCostWhole);
+    if (cost + rest_of_unit <= C) {
+      cost += rest_of_unit;
+      it += room;
+      continue;
+    }
+    const long long cnt = (C - cost - kPieceCostPartial) / 2;  // a partial piece that ends inside the unit
+    if (cnt >= 1) it += (int)(cnt < room - 1 ? cnt : room - 1);
+    break;
+  }
+  return it;
+}
+
+// Spans of cost at most C, left to right; the number of spans, or 0 when C is too small for some span or more
+// than `gmax` spans would be needed.
+int cut_spans(int T, int nblk, long long C, int gmax, int* bounds) {
+  int g = 0, it = 0;
+  bounds[0] = 0;
+  while (it < T) {
+    if (g == gmax) return 0;
+    const int end = span_end(it, T, nblk, C);
+    if (end == it) return 0;
+    bounds[++g] = it = end;
+  }
+  return g;
+}
+
 // Whole units per CTA when that is at most kSplitCostTiles tiles slower than a perfectly even cut;
-// otherwise spans cut at single key tiles (see Spans).
+// otherwise spans cut at single key tiles: evenly where a span holds two units or more (the pieces' costs are
+// small beside it), else so that the longest span, pieces' costs included, is as short as possible (the
+// smallest budget C for which a left-to-right cut needs no more spans than there are CTAs).
 Spans plan_spans(int units, int nblk) {
   Spans sp;
   sp.nblk = nblk;
@@ -704,12 +743,22 @@ Spans plan_spans(int units, int nblk) {
   sp.G = quanta < gmax ? quanta : gmax;
   const int q = quanta / sp.G, r = quanta - q * sp.G;  // the first r spans hold q + 1 quanta, the others q
   for (int g = 0; g <= sp.G; ++g) sp.bounds[g] = (g * q + (g < r ? g : r)) * quantum;
-  if (mode == 1 && q >= 8 * kSnapTiles) {
+  if (mode == 1 && q >= 2 * nblk) {
+    // long spans: the even cut, with every bound that falls within kSnapTiles of a unit boundary moved onto it
     for (int g = 1; g < sp.G; ++g) {
       const int unit_edge = (sp.bounds[g] + nblk / 2) / nblk * nblk;
       const int off = sp.bounds[g] - unit_edge;
       if (off != 0 && off >= -kSnapTiles && off <= kSnapTiles) sp.bounds[g] = unit_edge;
     }
+  } else if (mode == 1) {
+    // spans of less than two units: the pieces' costs decide
+    long long lo = 2 + kPieceCostPartial, hi = 2LL * sp.T + (long long)kPieceCostPartial * (units + 2);
+    while (lo < hi) {  // cut_spans succeeds for every budget from some value on
+      const long long mid = (lo + hi) / 2;
+      if (cut_spans(sp.T, nblk, mid, gmax, sp.bounds)) hi = mid;
+      else lo = mid + 1;
+    }
+    sp.G = cut_spans(sp.T, nblk, lo, gmax, sp.bounds);
   }
   return sp;
 }

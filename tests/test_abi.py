@@ -137,12 +137,47 @@ def test_attention_work_plan_covers_every_key_tile_once(toma, shape, split):
     assert min(sizes) >= 1
     if split is not None:
         assert plan["split"] == (split == "1")
-    if plan["split"]:
-        # equal to within one tile, then bounds within two tiles of a unit boundary are moved onto it
+    if plan["split"] and (units * nblk) // plan["ctas"] >= 2 * nblk:
+        # long spans: equal to within one tile, then bounds within two tiles of a unit boundary are moved onto it
         assert max(sizes) - min(sizes) <= 1 + 2 * 2
         for x in b[1:-1]:
             off = min(x % nblk, nblk - x % nblk)
-            assert off == 0 or off > 2 or min(sizes) < 16, "a bound sits within two tiles of a unit boundary"
+            assert off == 0 or off > 2, "a bound sits within two tiles of a unit boundary"
+        assert plan["owner_first"] == list(range(plan["ctas"])) and plan["owner_last"] == list(range(plan["ctas"]))
+    elif plan["split"]:
+        # short spans: the longest span, charged 2 per key tile plus 4 per whole-unit piece and 7 per partial piece
+        # (half tiles), is as short as a left-to-right cut into at most 148 spans can make it
+        def cost(lo, hi):
+            c, it = 0, lo
+            while it < hi:
+                end = min(hi, (it // nblk + 1) * nblk)
+                c += 2 * (end - it) + (4 if (it % nblk == 0 and end % nblk == 0) else 7)
+                it = end
+            return c
+
+        def spans_needed(budget):
+            n, it, T = 0, 0, units * nblk
+            while it < T:
+                end = it
+                while end < T:
+                    # one more tile - or, where that is too dear, on to the end of the unit: completing a unit that
+                    # the span entered at its first tile makes the piece a whole one, which is cheaper
+                    edge = min(T, (end // nblk + 1) * nblk)
+                    if cost(it, end + 1) <= budget:
+                        end += 1
+                    elif cost(it, edge) <= budget:
+                        end = edge
+                    else:
+                        break
+                if end == it:
+                    return None
+                n, it = n + 1, end
+            return n
+
+        worst = max(cost(b[g], b[g + 1]) for g in range(plan["ctas"]))
+        assert plan["ctas"] <= 148
+        fewer = spans_needed(worst - 1)
+        assert fewer is None or fewer > 148, "a smaller budget would have done"
         assert plan["owner_first"] == list(range(plan["ctas"])) and plan["owner_last"] == list(range(plan["ctas"]))
     else:
         assert all(x % nblk == 0 for x in b) and max(sizes) - min(sizes) <= nblk
