@@ -375,6 +375,32 @@ def test_block_small_tile_refresh_kernel_parity(toma, tuning, over):
     assert np.abs(dense[0] - dense[1]).max() <= 6e-4
 
 
+@pytest.mark.parametrize("name", ["cfg2", "cfg3"])
+def test_block_steps_enqueued_back_to_back_equal_synchronised_steps(toma, name):
+    """Consecutive toma_block calls overlap on the device (programmatic dependent launch: a kernel's prologue runs
+    under the previous kernel's tail).  Thirty steps enqueued without a synchronisation in between must give,
+    bit for bit, what the same steps give with the device idle before each call."""
+    cfg = gen.config(name, batch=1, steps=6, reuse_interval=3)
+    desc = toma.desc_from_config(cfg)
+    xs = [to_dev(x, cfg.dtype) for x in gen.feature_sequence(cfg)]
+    runs = []
+    for synchronise in (True, False):
+        idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        out = torch.empty_like(xs[0])
+        outs = []
+        for t in range(30):
+            toma.toma_block(desc, t % 6, xs[t % 6], out, idx, w, ws, status)
+            outs.append(out.clone())   # on the same stream, behind the step
+            if synchronise:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        runs.append(outs)
+    for t, (a, b) in enumerate(zip(*runs)):
+        assert torch.equal(a, b), f"step {t} differs"
+
+
 def test_block_separate_weight_schedule_parity(toma):
     """Destinations every 4 steps, weights every 2 (the paper refreshes weights more often than
     destinations): indices stay put at step 2 while the weights follow the drifted features."""
