@@ -182,6 +182,168 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
 }
 
 // ------------------------------------------------------------------------------------------------
+// merge, persistent form: for launches of many more (tile, channel chunk) items than the SMs hold at once.
+// One CTA per SM takes items blockIdx.x, blockIdx.x + gridDim.x, ... (consecutive CTAs work on chunks of the same
+// tile, so the tile's weights are L2 hits for all but one of them).  The TMA ring runs on across items; two
+// accumulators in tensor memory alternate, so that an item's epilogue (tensor memory -> staging tile in shared
+// memory -> TMA store) runs under the next item's loads and MMAs, and the prologue, the cold first fetch and
+// the tail of a CTA are paid once per SM instead of once per item.
+// ------------------------------------------------------------------------------------------------
+struct PersistBars {
+  uint64_t full[4], empty[4];
+  uint64_t acc_full[2], acc_empty[2];  // accumulator complete / read out by the four epilogue warps
+  uint64_t staged, stored;             // the staging tile is written (4 warps) / the TMA store has read it
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__global__ void __launch_bounds__(192, 1)
+merge_persistent_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+                        const __grid_constant__ CUtensorMap tm_o, const LinParams p, int n_items, int n_chunks,
+                        uint32_t* dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_dest = p.Dloc;                          // <= kMaxCols: one CTA produces all of a tile's destinations
+  const int slabs = (n_dest + 63) / 64, n_mma = slabs * 64;
+  const int stage_bytes = (2 + 2 * slabs) * kSlab;
+  uint8_t* so = smem + p.stages * stage_bytes;        // staging tile: two 64-channel slabs of [out_rows][128 B]
+  PersistBars* bar = reinterpret_cast<PersistBars*>(so + 2 * p.out_rows * 128);
+  const int rows_per_chunk = kKC / p.tw;
+  const int nk = p.Nloc / kKC;
+  const uint32_t acc_cols = tmem_cols_for(n_mma);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&bar->full[s], 1);
+      mbar_init(&bar->empty[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&bar->acc_full[a], 1);
+      mbar_init(&bar->acc_empty[a], 4);
+    }
+    mbar_init(&bar->staged, 4);
+    mbar_init(&bar->stored, 1);
+    bar->abort_flag = 0;
+    mbar_fence_init();
+    prefetch_tmap(&tm_x);
+    prefetch_tmap(&tm_w);
+    prefetch_tmap(&tm_o);
+  }
+  dependency_wait();
+  if (threadIdx.x == 0) release_dependents();
+  if (warp == 1) tmem_alloc(&bar->tmem_base, 2 * acc_cols);
+  if (p.zero_words > 0) {
+    const int n_thr = gridDim.x * blockDim.x;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < p.zero_words; i += n_thr) p.zero[i] = 0u;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bar->tmem_base;
+  volatile int* abort_flag = &bar->abort_flag;
+
+  if (warp == 0) {
+    if (elect_one()) {
+      int kc = 0;  // k-steps issued so far, over all items: ring slot and phase follow it
+      bool ok = true;
+      for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+        const int batch = item / n_chunks, c0 = (item - batch * n_chunks) * 128;
+        const int b = batch / p.P, tile = batch - b * p.P;
+        const int ty = tile / p.tiles_x, tx = tile - ty * p.tiles_x;
+        for (int k = 0; k < nk; ++k, ++kc) {
+          const int s = kc % p.stages;
+          if (kc >= p.stages && !mbar_wait(&bar->empty[s], ((kc / p.stages) - 1) & 1, dev_status, abort_flag)) { ok = false; break; }
+          uint8_t* sx = smem + s * stage_bytes;
+          uint8_t* sw = sx + 2 * kSlab;
+          mbar_expect_tx(&bar->full[s], stage_bytes);
+          for (int c = 0; c < 2; ++c)
+            tma_load_4d(sx + c * kSlab, &tm_x, &bar->full[s], c0 + c * 64, tx * p.tw, ty * p.th + k * rows_per_chunk, b);
+          for (int pl = 0; pl < 2; ++pl)
+            for (int c = 0; c < slabs; ++c)
+              tma_load_3d(sw + (pl * slabs + c) * kSlab, &tm_w, &bar->full[s], c * 64, k * kKC, 2 * batch + pl);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (elect_one()) {
+      const uint32_t idesc = idesc_f16(kFmtBF16, kFmtBF16, true, true, 128, n_mma);
+      int kc = 0, n = 0;
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+        const int a = n & 1;
+        if (n >= 2 && !mbar_wait(&bar->acc_empty[a], ((n >> 1) - 1) & 1, dev_status, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t t_acc = tmem + a * acc_cols;
+        bool ok = true;
+        for (int k = 0; k < nk; ++k, ++kc) {
+          const int s = kc % p.stages;
+          if (!mbar_wait(&bar->full[s], (kc / p.stages) & 1, dev_status, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t xa = smem_u32(smem + s * stage_bytes), wa = xa + 2 * kSlab;
+#pragma unroll
+          for (int kk = 0; kk < kKC / 16; ++kk) {
+            const uint64_t xd = smem_desc_sw128(xa + kk * 2048, kSlab, 1024);
+            mma_ss(t_acc, xd, smem_desc_sw128(wa + kk * 2048, kSlab, 1024), idesc, k > 0 || kk > 0);
+            mma_ss(t_acc, xd, smem_desc_sw128(wa + slabs * kSlab + kk * 2048, kSlab, 1024), idesc, true);
+          }
+          mma_commit(&bar->empty[s]);
+        }
+        if (!ok) break;
+        mma_commit(&bar->acc_full[a]);
+      }
+    }
+  } else {
+    const int quarter = warp & 3, cl = quarter * 32 + lane;  // channel of the chunk = tensor-memory lane
+    uint8_t* mine = so + (cl >> 6) * p.out_rows * 128 + (cl & 7) * 2;
+    const int chunk = (cl & 63) >> 3;
+    int n = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+      const int a = n & 1;
+      const int batch = item / n_chunks, c0 = (item - batch * n_chunks) * 128;
+      const int b = batch / p.P, tile = batch - b * p.P;
+      // the accumulator is complete, and the previous item's store has read the staging tile that is written
+      // again below; one answer per warp (the tensor-memory loads are warp-wide operations)
+      const bool go = mbar_wait(&bar->acc_full[a], (n >> 1) & 1, dev_status, abort_flag) &&
+                      (n == 0 || mbar_wait(&bar->stored, (n - 1) & 1, dev_status, abort_flag));
+      if (!__all_sync(0xffffffffu, go)) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem + a * acc_cols + ((uint32_t)(quarter * 32) << 16);
+      for (int i0 = 0; i0 < n_dest; i0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + i0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const int row = i0 + e;
+          if (row < n_dest)
+            *reinterpret_cast<__nv_bfloat16*>(mine + row * 128 + ((chunk ^ (row & 7)) << 4)) = __float2bfloat16_rn(__uint_as_float(r[e]));
+        }
+      }
+      tc_fence_before();
+      fence_proxy_async();  // the staged tile is read by the TMA engine
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&bar->acc_empty[a]);  // the accumulator may be overwritten by the item after next
+        mbar_arrive(&bar->staged);
+      }
+      if (cl == 0 && mbar_wait(&bar->staged, n & 1, dev_status, abort_flag)) {  // a wait that ran out ends the loop at its top
+        for (int c = 0; c < 2; ++c)
+          if (c0 + c * 64 < p.d) tma_store_4d(&tm_o, so + c * p.out_rows * 128, c0 + c * 64, 0, tile, b);
+        tma_store_commit();
+        tma_store_wait_read();  // shared memory must outlive the engine's reads
+        mbar_arrive(&bar->stored);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 2 * acc_cols);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // unmerge: grid (tile, channel chunk, token block); K loop over the tile's destinations.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(192, 1)
@@ -395,6 +557,173 @@ unmerge_rows_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_const
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// unmerge with tokens on M, persistent form: for launches of many more (tile, 128-token block, channel block)
+// items than there are SMs.  One CTA per SM walks its items; the ring holds the next item's operands while the
+// current one is multiplied, the output tile has a staging area of its own, and an item's TMA store runs
+// under the next item's MMAs.  One accumulator set (up to 320 columns of tensor memory): the next item's MMAs
+// wait only until the epilogue warps have read the accumulators out.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(192, 1)
+unmerge_rows_persistent_kernel(const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_w,
+                               const __grid_constant__ CUtensorMap tm_o, const LinParams p, int n_items, int ch_blocks,
+                               uint32_t* dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int blocks_per_tile = p.Nloc / 128;
+  const int max_slabs = ((p.d < kRowsChBlock ? p.d : kRowsChBlock) + 63) / 64;
+  const int w_plane = 128 * 128;  // [128 tokens][64 destinations] of one plane
+  const int stage_bytes = 2 * w_plane + max_slabs * kSlab;
+  uint8_t* so = smem + p.stages * stage_bytes;  // staging: max_slabs slabs of [128 tokens][128 B]
+  PersistBars* bar = reinterpret_cast<PersistBars*>(so + max_slabs * (128 * 128));
+  const int nk = (p.Dloc + kKC - 1) / kKC;
+  constexpr uint32_t ncols = 512;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&bar->full[s], 1);
+      mbar_init(&bar->empty[s], 1);
+    }
+    mbar_init(&bar->acc_full[0], 1);
+    mbar_init(&bar->acc_empty[0], 4);
+    mbar_init(&bar->staged, 4);
+    mbar_init(&bar->stored, 1);
+    bar->abort_flag = 0;
+    mbar_fence_init();
+    prefetch_tmap(&tm_y);
+    prefetch_tmap(&tm_w);
+    prefetch_tmap(&tm_o);
+  }
+  dependency_wait();
+  if (threadIdx.x == 0) release_dependents();
+  if (warp == 1) tmem_alloc(&bar->tmem_base, ncols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bar->tmem_base;
+  volatile int* abort_flag = &bar->abort_flag;
+  // item -> (tile of the batch, 128-token block, channel block); channel blocks of one token block are neighbours,
+  // so that concurrently running CTAs share its weights in L2
+  auto decode = [&](int item, int& batch, int& t0, int& c0) {
+    const int cb = item % ch_blocks, tb = item / ch_blocks;
+    batch = tb / blocks_per_tile;
+    t0 = (tb - batch * blocks_per_tile) * 128;
+    c0 = cb * kRowsChBlock;
+  };
+
+  if (warp == 0) {
+    if (elect_one()) {
+      int kc = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+        int batch, t0, c0;
+        decode(item, batch, t0, c0);
+        const int b = batch / p.P, tile = batch - b * p.P;
+        const int slabs = (min(kRowsChBlock, p.d - c0) + 63) / 64;
+        for (int k = 0; k < nk; ++k, ++kc) {
+          const int s = kc % p.stages;
+          if (kc >= p.stages && !mbar_wait(&bar->empty[s], ((kc / p.stages) - 1) & 1, dev_status, abort_flag)) { ok = false; break; }
+          uint8_t* sw = smem + s * stage_bytes;
+          uint8_t* sy = sw + 2 * w_plane;
+          mbar_expect_tx(&bar->full[s], 2 * w_plane + slabs * kSlab);
+          for (int pl = 0; pl < 2; ++pl) tma_load_3d(sw + pl * w_plane, &tm_w, &bar->full[s], k * kKC, t0, 2 * batch + pl);
+          for (int c = 0; c < slabs; ++c)
+            tma_load_3d(sy + c * kSlab, &tm_y, &bar->full[s], c0 + c * 64, tile * p.Dloc + k * kKC, b);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (elect_one()) {
+      int kc = 0, n = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++n) {
+        int batch, t0, c0;
+        decode(item, batch, t0, c0);
+        const int slabs = (min(kRowsChBlock, p.d - c0) + 63) / 64;
+        const int n_a = min(slabs, 3) * 64, n_b = (slabs - min(slabs, 3)) * 64;
+        const uint32_t idesc_a = idesc_f16(kFmtBF16, kFmtBF16, false, true, 128, n_a);
+        const uint32_t idesc_b = idesc_f16(kFmtBF16, kFmtBF16, false, true, 128, n_b > 0 ? n_b : 64);
+        // the epilogue warps have read the previous item's accumulators
+        if (n >= 1 && !mbar_wait(&bar->acc_empty[0], (n - 1) & 1, dev_status, abort_flag)) break;
+        tc_fence_after();
+        for (int k = 0; k < nk; ++k, ++kc) {
+          const int s = kc % p.stages;
+          if (!mbar_wait(&bar->full[s], (kc / p.stages) & 1, dev_status, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t wa = smem_u32(smem + s * stage_bytes), ya = wa + 2 * w_plane;
+          const int ksteps = min(kKC, p.Dloc - k * kKC + 15) / 16;  // 16 destinations per MMA
+          for (int kk = 0; kk < ksteps; ++kk) {
+            const uint64_t yd_a = smem_desc_sw128(ya + kk * 2048, kSlab, 1024);
+            const uint64_t yd_b = smem_desc_sw128(ya + 3 * kSlab + kk * 2048, kSlab, 1024);
+            for (int pl = 0; pl < 2; ++pl) {
+              const uint64_t wd = smem_desc_sw128(wa + pl * w_plane + kk * 32, 16, 1024);
+              const bool acc = k > 0 || kk > 0 || pl > 0;
+              mma_ss(tmem, wd, yd_a, idesc_a, acc);
+              if (n_b > 0) mma_ss(tmem + 192, wd, yd_b, idesc_b, acc);
+            }
+          }
+          mma_commit(&bar->empty[s]);
+        }
+        if (ok) mma_commit(&bar->acc_full[0]);
+      }
+    }
+  } else {
+    const int quarter = warp & 3, row = quarter * 32 + lane;  // token slot t0 + row = tensor-memory lane
+    const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16);
+    int n = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+      int batch, t0, c0;
+      decode(item, batch, t0, c0);
+      const int b = batch / p.P, tile = batch - b * p.P;
+      const int n_ch = min(kRowsChBlock, p.d - c0), slabs = (n_ch + 63) / 64;
+      // the accumulators are complete, and the previous item's store has read the staging area; one answer per
+      // warp (the tensor-memory loads are warp-wide operations)
+      const bool go = mbar_wait(&bar->acc_full[0], n & 1, dev_status, abort_flag) &&
+                      (n == 0 || mbar_wait(&bar->stored, (n - 1) & 1, dev_status, abort_flag));
+      if (!__all_sync(0xffffffffu, go)) break;
+      tc_fence_after();
+      for (int c = 0; c < n_ch; c += 32) {  // accumulator column = channel (the second accumulator starts at 192)
+        uint32_t r[32];
+        tmem_ld32(taddr + c, r);
+        tmem_wait_ld();
+        uint8_t* slab = so + (c >> 6) * (128 * 128);
+#pragma unroll
+        for (int e = 0; e < 32; e += 8) {
+          if (c + e < n_ch) {
+            __align__(16) __nv_bfloat162 q[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              q[u] = __floats2bfloat162_rn(__uint_as_float(r[e + 2 * u]), __uint_as_float(r[e + 2 * u + 1]));
+            *reinterpret_cast<uint4*>(slab + sw128_offset(row, ((c & 63) + e) >> 3)) = *reinterpret_cast<const uint4*>(q);
+          }
+        }
+      }
+      tc_fence_before();
+      fence_proxy_async();  // the staged rows are read by the TMA engine
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&bar->acc_empty[0]);  // the next item's products may overwrite the accumulators
+        mbar_arrive(&bar->staged);
+      }
+      if (row == 0 && mbar_wait(&bar->staged, n & 1, dev_status, abort_flag)) {  // a wait that ran out ends the loop at its top
+        const int ty = tile / p.tiles_x, tx = tile - ty * p.tiles_x;
+        for (int c = 0; c < slabs; ++c)  // a slab cut short by the channel count is clipped by the store
+          tma_store_4d(&tm_o, so + c * (128 * 128), c0 + c * 64, tx * p.tw, ty * p.th + t0 / p.tw, b);
+        tma_store_commit();
+        tma_store_wait_read();  // shared memory must outlive the engine's reads
+        mbar_arrive(&bar->stored);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, ncols);
+  }
+}
+
 LinParams make_params(const Geom& g) {
   LinParams p;
   p.P = g.P; p.tiles_x = g.tiles_x; p.th = g.th; p.tw = g.tw; p.W = g.W; p.Nloc = g.Nloc; p.Dloc = g.Dloc;
@@ -465,6 +794,24 @@ cudaError_t launch_merge_tc(const Geom& g, const void* w, const void* x, void* x
   const int smem = 1024 + p.stages * stage_bytes + 256;
   dim3 grid(g.B * g.P, (g.d + 127) / 128, (g.Dloc + p.dest_block - 1) / p.dest_block);
   cudaError_t e;
+  const int n_chunks = (g.d + 127) / 128, n_items = g.B * g.P * n_chunks;
+  if (g.Dloc <= kMaxCols && n_items > 2 * sm_count()) {
+    // more items than the SMs hold at once: one CTA per SM walks them with the ring and two accumulators kept busy
+    const int staging = 2 * p.out_rows * 128;
+    p.stages = (227 * 1024 - 1024 - 512 - staging) / stage_bytes;
+    p.stages = p.stages > 4 ? 4 : p.stages;
+    if (p.stages >= 2) {
+      const int smem_p = 1024 + p.stages * stage_bytes + staging + 512;
+      static std::atomic<unsigned long long> raised_p{0};
+      e = raise_dynamic_smem(merge_persistent_kernel, 227 * 1024, raised_p);
+      if (e != cudaSuccess) return e;
+      const int ctas = n_items < sm_count() ? n_items : sm_count();
+      e = launch_dependent(merge_persistent_kernel, dim3(ctas), dim3(192), (size_t)smem_p, s, tx, tw, to, p, n_items, n_chunks, dev_status);
+      count_launch();
+      return e != cudaSuccess ? e : cudaGetLastError();
+    }
+    p.stages = 2;
+  }
   if (g.Dloc > kMaxCols) {
     static std::atomic<unsigned long long> raised_b{0};
     e = raise_dynamic_smem(merge_tc_kernel<true>, 200 * 1024, raised_b);
@@ -496,6 +843,29 @@ cudaError_t launch_unmerge_tc(const Geom& g, const void* w, const void* y, void*
   const int rows_ctas = g.B * g.P * (g.Nloc / 128) * ((g.d + kRowsChBlock - 1) / kRowsChBlock);
   const int classic_ctas = g.B * g.P * ((g.d + 127) / 128) * (g.Nloc / n_tok);
   const bool one_wave = rows_ctas <= sms && classic_ctas > 2 * sms;
+  if (g.Dloc <= kMaxCols && g.Nloc % 128 == 0 && rows_ctas > sms) {
+    // many more items than SMs: tokens on M, one CTA per SM walking its items
+    CUtensorMap tw128, to;
+    if (!encode_w(g, w, &tw128, 128)) return cudaErrorInvalidValue;
+    const uint64_t odims[4] = {(uint64_t)g.d, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.B};
+    const uint64_t ostrides[3] = {(uint64_t)g.d * 2, (uint64_t)g.W * g.d * 2, (uint64_t)g.tokens_all() * g.d * 2};
+    const uint32_t obox[4] = {64, (uint32_t)g.tw, (uint32_t)(128 / g.tw), 1};
+    if (!encode_tmap_16bit(&to, out, 4, odims, ostrides, obox)) return cudaErrorInvalidValue;
+    const int max_slabs = ((g.d < kRowsChBlock ? g.d : kRowsChBlock) + 63) / 64;
+    const int stage_bytes = 2 * 128 * 128 + max_slabs * kSlab, staging = max_slabs * 128 * 128;
+    p.stages = (227 * 1024 - 1024 - 512 - staging) / stage_bytes;
+    p.stages = p.stages > 4 ? 4 : p.stages;
+    if (p.stages >= 2) {
+      const int smem = 1024 + p.stages * stage_bytes + staging + 512;
+      static std::atomic<unsigned long long> raised_rp{0};
+      if (cudaError_t e = raise_dynamic_smem(unmerge_rows_persistent_kernel, 227 * 1024, raised_rp); e != cudaSuccess) return e;
+      const int ch_blocks = (g.d + kRowsChBlock - 1) / kRowsChBlock;
+      cudaError_t e = launch_dependent(unmerge_rows_persistent_kernel, dim3(sms), dim3(192), (size_t)smem, s, ty, tw128, to, p, rows_ctas,
+                                       ch_blocks, dev_status);
+      count_launch();
+      return e != cudaSuccess ? e : cudaGetLastError();
+    }
+  }
   if ((g.Dloc > kMaxCols || one_wave) && g.Nloc % 128 == 0) {
     CUtensorMap tw128;
     if (!encode_w(g, w, &tw128, 128)) return cudaErrorInvalidValue;
