@@ -989,6 +989,24 @@ def test_degenerate_inputs_identical_and_zero_tokens(toma):
     for p in range(2):
         want, _ = O.select_tile(tile_tokens(cfg, x_host, 0, p), od(cfg))
         assert np.array_equal(idx[0, p], want)
+    # the same through a refresh step of toma_block, which runs selection and weights of 64-token tiles as one
+    # kernel with a one-warp greedy: the same picks, weights against Sec. 4.2.1, finite output
+    desc = toma.desc_from_config(cfg)
+    idx_b, w_b, ws_b = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    x = to_dev(x_host, cfg.dtype)
+    out = torch.full_like(x, float("nan"))
+    toma.toma_block(desc, 0, x, out, idx_b, w_b, ws_b, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert np.array_equal(idx_b.cpu().numpy().astype(np.int64), idx)
+    dense = torch.empty((1, 2, 32, 64), dtype=torch.float32, device="cuda")
+    toma.toma_weights_export(desc, w_b, dense)
+    torch.cuda.synchronize()
+    for p in range(2):
+        want_w = O.merge_weights(tile_tokens(cfg, x_host, 0, p), idx[0, p], cfg.tau)
+        assert np.abs(dense[0, p].cpu().numpy().astype(np.float64) - want_w).max() <= 6e-4
+    assert torch.isfinite(out.float()).all()
 
 
 def test_results_are_deterministic(toma):
