@@ -401,6 +401,30 @@ def test_block_steps_enqueued_back_to_back_equal_synchronised_steps(toma, name):
         assert torch.equal(a, b), f"step {t} differs"
 
 
+def test_small_tile_refresh_kernel_agrees_with_the_separate_kernels_on_many_inputs(toma, tuning):
+    """Both forms of a refresh step on 64-token tiles work on the same integers (the fixed-point Gram) with the same
+    rule (largest gain, lowest index), so their picks must be identical on any input, fragile or not; twenty seeds,
+    two noise levels (smooth tiles give many near-ties)."""
+    for seed in range(20):
+        cfg = gen.config("cfg2", batch=1, steps=1, reuse_interval=1, seed=1000 + seed, noise_sigma=0.05 if seed % 2 else 0.5)
+        desc = toma.desc_from_config(cfg)
+        x = to_dev(next(iter(gen.feature_sequence(cfg))), cfg.dtype)
+        got = {}
+        for separate in (0, 1):
+            tuning(block_unfused=separate)
+            idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+            status = torch.zeros(1, dtype=torch.int32, device="cuda")
+            out = torch.empty_like(x)
+            toma.toma_block(desc, 0, x, out, idx, w, ws, status)
+            dense = torch.empty((cfg.batch, cfg.n_tiles, gd(toma, cfg), cfg.n_loc), dtype=torch.float32, device="cuda")
+            toma.toma_weights_export(desc, w, dense)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            got[separate] = (idx.cpu().numpy().copy(), dense.cpu().numpy().copy())
+        assert np.array_equal(got[0][0], got[1][0]), f"picks differ for seed {seed}"
+        assert np.abs(got[0][1] - got[1][1]).max() <= 6e-4, f"weights differ for seed {seed}"
+
+
 def test_block_separate_weight_schedule_parity(toma):
     """Destinations every 4 steps, weights every 2 (the paper refreshes weights more often than
     destinations): indices stay put at step 2 while the weights follow the drifted features."""
