@@ -6,9 +6,11 @@
 // (two MMAs along N, at most 192 + 128).  A is the K-major operand exactly as stored ([m][k] row-major),
 // W the MN-major one exactly as stored ([k][n] row-major), so neither is transposed or copied.
 // blockIdx.z selects one of up to three weight / output pairs that share A (Q, K and V in one
-// launch).  Warp 0 feeds a TMA ring, warp 1 issues the MMAs, warps 2..5 write each token row's
-// columns as one contiguous run, after the activation when one is asked for (the first layer of the
-// MLP, the other module ToMA wraps).
+// launch).  Warp 0 feeds a TMA ring, warp 1 issues the MMAs, warps 2..5 take the accumulators out of tensor
+// memory (through the activation when one is asked for: the first layer of the MLP, the other module ToMA
+// wraps), stage each warp's 32 rows in shared memory as 64-column slabs in the layout of the output tensor
+// map's box (the ring is free by then) and store them with one TMA store per warp and slab: whole lines,
+// asynchronous, instead of 16-byte stores to 32 different rows per warp instruction.
 #include <cstdlib>
 
 #include "common.cuh"
@@ -30,9 +32,6 @@ struct GemmBars {
   int abort_flag;
 };
 
-struct GemmOut {
-  __nv_bfloat16* c[3];
-};
 
 // kCols = 320: two accumulators (192 + 128 columns), 512 tensor-memory columns, one CTA per SM, deep ring.
 // kCols = 256: one accumulator, 256 tensor-memory columns, two CTAs per SM, for grids that would otherwise
@@ -43,20 +42,22 @@ struct GemmOut {
 template <int kCols, int kRowBlocks = 1>
 __global__ void __launch_bounds__(192, 1)
 linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w0,
-                   const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2, GemmOut out, int M,
-                   int N, int K, int stages, int act, uint32_t* dev_status) {
+                   const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2,
+                   const __grid_constant__ CUtensorMap tm_c0, const __grid_constant__ CUtensorMap tm_c1,
+                   const __grid_constant__ CUtensorMap tm_c2, int M, int N, int K, int stages, int ring_bytes, int act,
+                   uint32_t* dev_status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int kFirst = kCols == 320 ? 3 : 4;  // 64-column slabs of the first accumulator
   const int m0 = blockIdx.x * 128 * kRowBlocks, n0 = blockIdx.y * kCols;
   const CUtensorMap* tm_w = blockIdx.z == 0 ? &tm_w0 : blockIdx.z == 1 ? &tm_w1 : &tm_w2;
-  __nv_bfloat16* c = out.c[blockIdx.z];
+  const CUtensorMap* tm_c = blockIdx.z == 0 ? &tm_c0 : blockIdx.z == 1 ? &tm_c1 : &tm_c2;
   const int n_cols = min(kCols, N - n0);         // columns of this CTA (multiple of 8)
   const int slabs = (n_cols + 63) / 64;
   const int n_a = min(slabs, kFirst) * 64, n_b = (slabs - min(slabs, kFirst)) * 64;
   const int stage_bytes = kRowBlocks * kABytes + slabs * kSlab;
-  GemmBars* bar = reinterpret_cast<GemmBars*>(smem + stages * stage_bytes);
+  GemmBars* bar = reinterpret_cast<GemmBars*>(smem + ring_bytes);  // behind the ring and the output's staging area, whichever is larger
   const int nk = (K + kKC - 1) / kKC;
   constexpr uint32_t ncols = (kCols == 320 || kRowBlocks == 2) ? 512 : 256;
   static_assert(kRowBlocks == 1 || kCols == 256, "two row blocks need the one-accumulator column form");
@@ -71,6 +72,7 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
     mbar_fence_init();
     prefetch_tmap(&tm_a);
     prefetch_tmap(tm_w);
+    prefetch_tmap(tm_c);
   }
   dependency_wait();
   if (threadIdx.x == 0) release_dependents();
@@ -119,14 +121,15 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
       if (ok) mma_commit(&bar->done);
     }
   } else {
-    const int quarter = warp & 3;
-    if (mbar_wait(&bar->done, 0, dev_status, abort_flag)) {
+    const int quarter = warp & 3, r_in = quarter * 32 + lane;  // row inside a 128-row block = tensor-memory lane
+    // one answer per warp: the tensor-memory loads below are warp-wide operations
+    if (__all_sync(0xffffffffu, mbar_wait(&bar->done, 0, dev_status, abort_flag))) {
       tc_fence_after();
+      // every load has been consumed: slab j of row block rb goes to smem + (rb * slabs + j) * 16 KB as
+      // [128 rows][128 B], 128-byte swizzled; a warp's 32 rows are 4 KB of it
 #pragma unroll 1
       for (int rb = 0; rb < kRowBlocks; ++rb) {
-        const int row = m0 + rb * 128 + quarter * 32 + lane;
         const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + rb * 256;
-        __nv_bfloat16* dst = c + (size_t)(row < M ? row : 0) * N + n0;
         for (int j = 0; j < n_cols; j += 32) {
           uint32_t r[32];
           tmem_ld32(taddr + j, r);
@@ -135,19 +138,28 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
 #pragma unroll
             for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(gelu(__uint_as_float(r[e])));
           }
-          if (row < M) {
+          uint8_t* slab = smem + (rb * slabs + (j >> 6)) * (128 * 128);
 #pragma unroll
-            for (int e = 0; e < 32; e += 8) {
-              if (j + e < n_cols) {
-                __align__(16) __nv_bfloat162 q[4];
+          for (int e = 0; e < 32; e += 8) {
+            __align__(16) __nv_bfloat162 q[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
-                  q[u] = __floats2bfloat162_rn(__uint_as_float(r[e + 2 * u]), __uint_as_float(r[e + 2 * u + 1]));
-                *reinterpret_cast<uint4*>(dst + j + e) = *reinterpret_cast<const uint4*>(q);
-              }
-            }
+            for (int u = 0; u < 4; ++u)
+              q[u] = __floats2bfloat162_rn(__uint_as_float(r[e + 2 * u]), __uint_as_float(r[e + 2 * u + 1]));
+            *reinterpret_cast<uint4*>(slab + sw128_offset(r_in, ((j & 63) + e) >> 3)) = *reinterpret_cast<const uint4*>(q);
           }
         }
+      }
+      fence_proxy_async();  // the staged rows are read by the TMA engine
+      __syncwarp();
+      if (lane == 0) {
+        for (int rb = 0; rb < kRowBlocks; ++rb) {
+          const int row0 = m0 + rb * 128 + quarter * 32;
+          if (row0 >= M) continue;  // rows past M and columns past N inside a box are clipped by the store
+          for (int j = 0; j < slabs; ++j)
+            tma_store_2d(tm_c, smem + (rb * slabs + j) * (128 * 128) + quarter * 4096, n0 + j * 64, row0);
+        }
+        tma_store_commit();
+        tma_store_wait_read();  // shared memory must outlive the engine's reads
       }
     }
   }
@@ -166,7 +178,7 @@ bool linear_tc_shape_ok(int M, int N, int K) { return M >= 1 && N >= 8 && K >= 8
 // c[i] = a * w[i] for i < n_mats (1..3); a [M][K], w[i] [K][N], c[i] [M][N], all bf16 row-major.
 cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* const* w, void* const* c, int n_mats, int act,
                              uint32_t* dev_status, cudaStream_t s) {
-  CUtensorMap ta, tw[3];
+  CUtensorMap ta, tw[3], tc_[3];
   const uint64_t adims[2] = {(uint64_t)K, (uint64_t)M};
   const uint64_t astr[1] = {(uint64_t)K * 2};
   const uint32_t abox[2] = {64, 128};
@@ -174,11 +186,12 @@ cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* con
   const uint64_t wdims[2] = {(uint64_t)N, (uint64_t)K};
   const uint64_t wstr[1] = {(uint64_t)N * 2};
   const uint32_t wbox[2] = {64, 64};
-  GemmOut out;
+  const uint64_t cdims[2] = {(uint64_t)N, (uint64_t)M};
+  const uint32_t cbox[2] = {64, 32};  // a warp's 32 rows of one 64-column slab
   for (int i = 0; i < 3; ++i) {
     const int j = i < n_mats ? i : 0;
-    if (!encode_tmap_16bit(&tw[i], w[j], 2, wdims, wstr, wbox)) return cudaErrorInvalidValue;
-    out.c[i] = (__nv_bfloat16*)c[j];
+    if (!encode_tmap_16bit(&tw[i], w[j], 2, wdims, wstr, wbox) || !encode_tmap_16bit(&tc_[i], c[j], 2, cdims, wstr, cbox))
+      return cudaErrorInvalidValue;
   }
   // Tile form: the one with the least serial work per SM, counted as CTAs per SM (rounded up) times the
   // multiply-adds of a tile, the 256 x 256 form credited with the 1.3x it gains from moving fewer operand
@@ -205,7 +218,9 @@ cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* con
   stages = stages > 4 ? 4 : stages < 1 ? 1 : stages;
   const int nk = (K + kKC - 1) / kKC;
   if (stages > nk) stages = nk;
-  const int smem = 1024 + stages * stage_bytes + 256;
+  const int staging = (pair ? 2 : 1) * slabs * 128 * 128;  // the output tile, staged where the ring was
+  const int ring_bytes = stages * stage_bytes > staging ? stages * stage_bytes : staging;
+  const int smem = 1024 + ring_bytes + 256;
   {
     static std::atomic<unsigned long long> r320{0}, r256{0}, rpair{0};
     cudaError_t e = raise_dynamic_smem(linear_rows_kernel<320>, 227 * 1024, r320);
@@ -214,12 +229,12 @@ cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* con
     if (e != cudaSuccess) return e;
   }
   dim3 grid(pair ? (M + 255) / 256 : mb, (N + cols - 1) / cols, n_mats);
-  cudaError_t e = pair ? launch_dependent(linear_rows_kernel<256, 2>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out,
-                                          M, N, K, stages, act, dev_status)
-                  : narrow ? launch_dependent(linear_rows_kernel<256>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out,
-                                            M, N, K, stages, act, dev_status)
-                         : launch_dependent(linear_rows_kernel<320>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], out,
-                                            M, N, K, stages, act, dev_status);
+  cudaError_t e = pair ? launch_dependent(linear_rows_kernel<256, 2>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], tc_[0], tc_[1],
+                                          tc_[2], M, N, K, stages, ring_bytes, act, dev_status)
+                  : narrow ? launch_dependent(linear_rows_kernel<256>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], tc_[0], tc_[1],
+                                            tc_[2], M, N, K, stages, ring_bytes, act, dev_status)
+                         : launch_dependent(linear_rows_kernel<320>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], tc_[0], tc_[1],
+                                            tc_[2], M, N, K, stages, ring_bytes, act, dev_status);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }
