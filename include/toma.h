@@ -110,7 +110,7 @@ TOMA_API uint64_t toma_launch_counter(void);
  * on these settings, only the launch configuration does.  Process-wide; not for concurrent use.
  *   attention_split: 0 = whole work units per CTA, 1 = spans cut at single key tiles, other = heuristic
  *   attention_ctas : > 0 = number of persistent CTAs (clamped to the scratch capacity), else heuristic
- *   linear_tile    : 1 = 128 x 256, 2 = 128 x 320, 3 = 256 x 256 tiles, else heuristic
+ *   linear_tile    : 1 = 128 x 256, 2 = 128 x 320, 3 = 256 x 256, 4 = 128 x 128 tiles, else heuristic
  *   block_unfused  : 1 = toma_block runs merge, attention and unmerge as three kernels even for the shapes its
  *                    one-kernel reuse step covers, and selection and weights of 64-token tiles as their separate
  *                    kernels instead of one (so that both paths can be compared), else the library chooses */

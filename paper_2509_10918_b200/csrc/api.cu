@@ -541,5 +541,5 @@ extern "C" void toma_test_set_tuning(int32_t attention_split, int32_t attention_
   toma::g_tune_block_unfused.store(block_unfused == 1 ? 1 : 0);
   toma::g_tune_attention_split.store(attention_split == 0 || attention_split == 1 ? attention_split : -1);
   toma::g_tune_attention_ctas.store(attention_ctas > 0 ? attention_ctas : 0);
-  toma::g_tune_linear_tile.store(linear_tile >= 1 && linear_tile <= 3 ? linear_tile : 0);
+  toma::g_tune_linear_tile.store(linear_tile >= 1 && linear_tile <= 4 ? linear_tile : 0);
 }

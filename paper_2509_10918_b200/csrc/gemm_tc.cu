@@ -36,6 +36,8 @@ struct GemmBars {
 // kCols = 320: two accumulators (192 + 128 columns), 512 tensor-memory columns, one CTA per SM, deep ring.
 // kCols = 256: one accumulator, 256 tensor-memory columns, two CTAs per SM, for grids that would otherwise
 // spill into a second wave or leave most SMs idle.
+// kCols = 128: 128 tensor-memory columns and 32 KB stages, two CTAs per SM, for narrow outputs with a long
+// contraction (the second layer of the MLP: 4096 x 640 x 2560 is 64 tiles of 128 x 320 but 160 of 128 x 128).
 // kRowBlocks = 2 (with kCols = 256): two 128-row blocks per CTA share every W slab, so a CTA moves 64 KB
 // per 256 x 256 x 64 multiply-adds instead of 48 KB per 128 x 256 x 64 (these shapes re-read their operands
 // from L2 many times and are bound by that traffic); one CTA per SM.
@@ -59,7 +61,7 @@ linear_rows_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_consta
   const int stage_bytes = kRowBlocks * kABytes + slabs * kSlab;
   GemmBars* bar = reinterpret_cast<GemmBars*>(smem + ring_bytes);  // behind the ring and the output's staging area, whichever is larger
   const int nk = (K + kKC - 1) / kKC;
-  constexpr uint32_t ncols = (kCols == 320 || kRowBlocks == 2) ? 512 : 256;
+  constexpr uint32_t ncols = (kCols == 320 || kRowBlocks == 2) ? 512 : kCols == 128 ? 128 : 256;
   static_assert(kRowBlocks == 1 || kCols == 256, "two row blocks need the one-accumulator column form");
 
   if (threadIdx.x == 0) {
@@ -205,16 +207,22 @@ cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* con
   const long long cost320 = ((ctas320 + sms - 1) / sms) * (128 * 320) * 13;
   const long long cost256 = ctas256 <= 2 * sms ? ((ctas256 + sms - 1) / sms) * (128 * 256) * 13 : cost320 + 1;
   const long long cost_pair = M > 128 ? ((ctas_pair + sms - 1) / sms) * (256 * 256) * 10 : cost320 + 1;
-  int pair = cost_pair < cost320 && cost_pair < cost256;
-  bool narrow = !pair && cost256 < cost320;
-  if (const int v = g_tune_linear_tile.load(std::memory_order_relaxed)) {  // test-only override: 128 x 256 (1), 128 x 320 (2) or 256 x 256 (3) tiles
+  // 128 x 128 tiles, two CTAs per SM sharing its tensor pipe: serial work = CTAs per SM (rounded up) tiles
+  const long long ctas128 = (long long)mb * ((N + 127) / 128) * n_mats;
+  const long long cost128 = ctas128 <= 2 * sms ? ((ctas128 + sms - 1) / sms) * (128 * 128) * 13 : cost320 + 1;
+  // ties go to the form with more, smaller CTAs (more SMs take in operands at once)
+  bool small = cost128 <= cost256 && cost128 <= cost_pair && cost128 < cost320;
+  bool narrow = !small && cost256 <= cost_pair && cost256 < cost320;
+  int pair = !small && !narrow && cost_pair < cost320;
+  if (const int v = g_tune_linear_tile.load(std::memory_order_relaxed)) {  // test-only override: 128 x 256 (1), 128 x 320 (2), 256 x 256 (3) or 128 x 128 (4) tiles
     pair = v == 3 && M > 128;
     narrow = v == 1;
+    small = v == 4;
   }
-  const int cols = (narrow || pair) ? 256 : 320;
+  const int cols = small ? 128 : (narrow || pair) ? 256 : 320;
   const int slabs = ((N < cols ? N : cols) + 63) / 64;
   const int stage_bytes = (pair ? 2 : 1) * kABytes + slabs * kSlab;
-  int stages = ((narrow && !pair ? 110 : 222) * 1024) / stage_bytes;
+  int stages = (((narrow && !pair) || small ? 110 : 222) * 1024) / stage_bytes;
   stages = stages > 4 ? 4 : stages < 1 ? 1 : stages;
   const int nk = (K + kKC - 1) / kKC;
   if (stages > nk) stages = nk;
@@ -222,8 +230,9 @@ cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* con
   const int ring_bytes = stages * stage_bytes > staging ? stages * stage_bytes : staging;
   const int smem = 1024 + ring_bytes + 256;
   {
-    static std::atomic<unsigned long long> r320{0}, r256{0}, rpair{0};
+    static std::atomic<unsigned long long> r320{0}, r256{0}, rpair{0}, r128{0};
     cudaError_t e = raise_dynamic_smem(linear_rows_kernel<320>, 227 * 1024, r320);
+    if (e == cudaSuccess) e = raise_dynamic_smem(linear_rows_kernel<128>, 227 * 1024, r128);
     if (e == cudaSuccess) e = raise_dynamic_smem(linear_rows_kernel<256>, 227 * 1024, r256);
     if (e == cudaSuccess) e = raise_dynamic_smem(linear_rows_kernel<256, 2>, 227 * 1024, rpair);
     if (e != cudaSuccess) return e;
@@ -231,6 +240,8 @@ cudaError_t launch_linear_tc(int M, int N, int K, const void* a, const void* con
   dim3 grid(pair ? (M + 255) / 256 : mb, (N + cols - 1) / cols, n_mats);
   cudaError_t e = pair ? launch_dependent(linear_rows_kernel<256, 2>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], tc_[0], tc_[1],
                                           tc_[2], M, N, K, stages, ring_bytes, act, dev_status)
+                  : small ? launch_dependent(linear_rows_kernel<128>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], tc_[0], tc_[1],
+                                            tc_[2], M, N, K, stages, ring_bytes, act, dev_status)
                   : narrow ? launch_dependent(linear_rows_kernel<256>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], tc_[0], tc_[1],
                                             tc_[2], M, N, K, stages, ring_bytes, act, dev_status)
                          : launch_dependent(linear_rows_kernel<320>, grid, dim3(192), (size_t)smem, s, ta, tw[0], tw[1], tw[2], tc_[0], tc_[1],

@@ -649,10 +649,10 @@ def test_linear_parity(toma, dtype, m, n, k):
     assert_close(to_host64(c)[rows], O.linear(a_host[rows], w_host), dtype, "linear")
 
 
-@pytest.mark.parametrize("tile", [0, 1, 2], ids=["128x256", "128x320", "256x256"])
+@pytest.mark.parametrize("tile", [0, 1, 2, 3], ids=["128x256", "128x320", "256x256", "128x128"])
 @pytest.mark.parametrize("m,n,k", [(300, 328, 200), (129, 1920, 640), (1024, 72, 136), (640, 512, 64)])
 def test_linear_every_tile_form(toma, tuning, tile, m, n, k):
-    """Each of the projection kernel's three tile forms, forced, on shapes with a ragged last row block (the
+    """Each of the projection kernel's four tile forms, forced, on shapes with a ragged last row block (the
     second row block of a 256-row tile partly or wholly past the end), partial column blocks and a partial
     last k-step."""
     tuning(linear_tile=tile + 1)
