@@ -99,51 +99,6 @@ __device__ __forceinline__ void store_slab_row(uint8_t* slab, const SlabRow& w, 
   }
 }
 
-// ---- the two CTAs of a head as a cluster
-__device__ __forceinline__ uint32_t cluster_rank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-// Every thread of both CTAs arrives; nobody passes before all have (shared memory and barriers of the peer exist).
-__device__ __forceinline__ void cluster_sync() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// The address of the peer CTA's copy of a shared-memory location of this CTA.
-__device__ __forceinline__ uint32_t peer_addr(uint32_t local, uint32_t peer) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(peer));
-  return r;
-}
-// Bulk copy of `bytes` of this CTA's shared memory to the peer's (same layout); the bytes count on the peer's barrier.
-__device__ __forceinline__ void copy_to_peer(uint32_t peer_dst, const void* src, uint32_t bytes, uint32_t peer_bar) {
-  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(peer_dst),
-               "r"(smem_u32(src)), "r"(bytes), "r"(peer_bar)
-               : "memory");
-}
-// One arrival on a barrier of the peer.
-__device__ __forceinline__ void mbar_arrive_peer(uint32_t addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(addr) : "memory");
-}
-// mbar_wait() whose acquire spans the cluster: the barrier also counts bytes the peer CTA sends.
-__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, uint32_t* dev_status, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    if (done) return true;
-    if ((it & 1023u) == 1023u && *abort_flag) return false;
-  }
-  *abort_flag = 1;
-  if (dev_status) atomicOr(dev_status, kStatusTimeout);
-  return false;
-}
-
 // 64 fp32 of a tensor-memory row -> one 128-byte bf16 row of a swizzled shared-memory tile, scaled.
 __device__ __forceinline__ void row_to_smem(uint32_t taddr, uint8_t* tile, int row, float scale) {
 #pragma unroll

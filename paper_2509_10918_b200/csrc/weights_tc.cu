@@ -24,6 +24,7 @@ constexpr int kKC = 64;
 
 struct WBars {
   uint64_t full[4], empty[4], done;
+  uint64_t z_in;  // paired form: the peer CTA's row sums have arrived
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -238,8 +239,12 @@ weights_logits_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
 // fp32 shares never exist in memory.
 //   kMB: 128-source blocks per tile (1 or 2).  Warp 0 TMA, warp 1 MMA, then four epilogue warps
 //   per source block (thread = source token = tensor-memory lane).
+//   kPair (with kMB = 1): a tile of two source blocks is shared by the two CTAs of a cluster, one block each,
+//   which send each other their halves of the row sums (a store into the peer's shared memory per
+//   destination, counted on a barrier of the peer's) - for launches of few tiles, where one CTA per tile would
+//   leave most SMs idle and each CTA bound by what one SM takes in.
 // ------------------------------------------------------------------------------------------------
-template <int kMB>
+template <int kMB, bool kPair = false>
 __global__ void __launch_bounds__(64 + 128 * kMB, 1)
 weights_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_d,
                      __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wu, const WParams p, uint32_t* dev_status) {
@@ -253,8 +258,11 @@ weights_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   WBars* bar = reinterpret_cast<WBars*>(smem + p.stages * stage_bytes);
   float* zw = reinterpret_cast<float*>(bar + 1);  // [4 kMB warps][D_loc] partial row sums
   float* zinv = zw + 4 * kMB * Dl;                // [D_loc] reciprocal row sums of the tile
+  float* zpeer = zinv + Dl;                       // [D_loc] paired form: the peer block's row sums
+  static_assert(!kPair || kMB == 1, "the paired form has one source block per CTA");
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int batch = blockIdx.x;
+  const int batch = kPair ? blockIdx.x >> 1 : blockIdx.x;
+  const int half = kPair ? (int)(blockIdx.x & 1) : 0;  // = rank in the cluster: the tile's source block of this CTA
   const int b = batch / p.P, tile = batch - b * p.P;
   const int ty = tile / p.tiles_x, tx = tile - ty * p.tiles_x;
   const int rows_per_box = p.m_tok / p.tw;
@@ -268,6 +276,7 @@ weights_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       mbar_init(&bar->empty[s], 1);
     }
     mbar_init(&bar->done, 1);
+    mbar_init(&bar->z_in, 128);  // every epilogue thread of the peer arrives once
     bar->abort_flag = 0;
     mbar_fence_init();
     prefetch_tmap(&tm_x);
@@ -279,6 +288,7 @@ weights_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (kPair) cluster_sync();  // the peer's barrier is initialised before anything is sent to it
   const uint32_t tmem = bar->tmem_base;
   volatile int* abort_flag = &bar->abort_flag;
 
@@ -290,7 +300,7 @@ weights_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         uint8_t* sa = smem + s * stage_bytes;
         mbar_expect_tx(&bar->full[s], kMB * p.m_tok * 128 + Dl * 128);
         for (int mb = 0; mb < kMB; ++mb)
-          tma_load_4d(sa + mb * a_bytes, &tm_x, &bar->full[s], k * kKC, tx * p.tw, ty * p.th + mb * rows_per_box, b);
+          tma_load_4d(sa + mb * a_bytes, &tm_x, &bar->full[s], k * kKC, tx * p.tw, ty * p.th + (mb + half) * rows_per_box, b);
         tma_load_3d(sa + kMB * a_bytes, &tm_d, &bar->full[s], k * kKC, 0, batch);
       }
     }
@@ -373,20 +383,38 @@ weights_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     // the tile's row sums: warps of a block pairwise, then the blocks in order (a fixed order: the
     // result does not depend on scheduling); a row sum that underflowed to 0 gives a zero row
     asm volatile("bar.sync 1, %0;" ::"n"(128 * kMB) : "memory");
-    for (int i = threadIdx.x - 64; i < Dl; i += 128 * kMB) {
-      float z = 0.f;
-#pragma unroll
-      for (int m = 0; m < kMB; ++m) {
-        const float* q = zw + m * 4 * Dl + i;
-        z += (q[0] + q[Dl]) + (q[2 * Dl] + q[3 * Dl]);
+    if (kPair) {
+      // this block's sums go to the peer, the peer's arrive here; both add block 0 + block 1 in that order
+      const uint32_t peer = (uint32_t)(half ^ 1);
+      const uint32_t peer_z = peer_addr(smem_u32(zpeer), peer);
+      for (int i = threadIdx.x - 64; i < Dl; i += 128) {
+        const float* q = zw + i;
+        const float z = (q[0] + q[Dl]) + (q[2 * Dl] + q[3 * Dl]);
+        zinv[i] = z;  // own half, for now
+        st_peer_f32(peer_z + 4u * (uint32_t)i, z);
       }
-      zinv[i] = z > 0.f ? 1.f / z : 0.f;
+      mbar_arrive_peer(peer_addr(smem_u32(&bar->z_in), peer));
+      const bool got = mbar_wait_cluster(&bar->z_in, 0, dev_status, abort_flag);
+      for (int i = threadIdx.x - 64; i < Dl; i += 128) {
+        const float z = !got ? 0.f : half == 0 ? zinv[i] + zpeer[i] : zpeer[i] + zinv[i];
+        zinv[i] = z > 0.f ? 1.f / z : 0.f;
+      }
+    } else {
+      for (int i = threadIdx.x - 64; i < Dl; i += 128 * kMB) {
+        float z = 0.f;
+#pragma unroll
+        for (int m = 0; m < kMB; ++m) {
+          const float* q = zw + m * 4 * Dl + i;
+          z += (q[0] + q[Dl]) + (q[2 * Dl] + q[3 * Dl]);
+        }
+        zinv[i] = z > 0.f ? 1.f / z : 0.f;
+      }
     }
     asm volatile("bar.sync 1, %0;" ::"n"(128 * kMB) : "memory");
     if (ok && valid) {
       // pass 4: A~_ik = A_ik / Z_i, written as row k of A~^T [N_loc][D_loc], hi plane then lo plane
       const size_t plane = (size_t)p.Nloc * Dl;
-      const size_t row = (size_t)(mb * p.m_tok + k_loc) * Dl;
+      const size_t row = (size_t)((mb + half) * p.m_tok + k_loc) * Dl;
       __nv_bfloat16* t_hi = w + (size_t)batch * 2 * plane + row;
       __nv_bfloat16* u_hi = wu ? wu + (size_t)batch * 2 * plane + row : nullptr;
       for (int i0 = 0; i0 < Dl; i0 += 32) {
@@ -422,6 +450,7 @@ weights_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     tc_fence_after();
     tmem_dealloc(tmem, ncols);
   }
+  if (kPair) cluster_sync();  // neither CTA's shared memory goes away while the other could still write to it
 }
 
 __global__ void __launch_bounds__(256)
@@ -600,6 +629,8 @@ cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, 
   // wins once there are enough tiles to occupy the SMs anyway (measured: 77 against 91 us on 256 tiles, 30
   // against 26 us on 32 tiles); with one source block per tile it only saves the second kernel.
   const bool fused = g.Dloc <= 256 && g.Dloc % 8 == 0 && (mblocks == 1 || (mblocks == 2 && (int)tiles >= sm_count() / 2));
+  // few tiles of two source blocks: the fused form with the tile shared by a cluster of two CTAs (one block each)
+  const bool paired = !fused && g.Dloc <= 256 && g.Dloc % 8 == 0 && mblocks == 2;
   const uint64_t xdims[4] = {(uint64_t)g.d, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.B};
   const uint64_t xstr[3] = {(uint64_t)g.d * 2, (uint64_t)g.W * g.d * 2, (uint64_t)g.tokens_all() * g.d * 2};
   const uint32_t xbox[4] = {64, (uint32_t)g.tw, (uint32_t)(p.m_tok / g.tw), 1};
@@ -610,12 +641,25 @@ cudaError_t launch_weights_tc(const Geom& g, const void* x, const int32_t* idx, 
     return cudaErrorInvalidValue;
   const int b_rows = g.Dloc > 256 ? 512 : ((g.Dloc + 7) & ~7);
   const int nk = (g.d + kKC - 1) / kKC;
+  if (paired) {
+    const int stage_bytes = 128 * 128 + ((b_rows * 128 + 1023) / 1024) * 1024;
+    p.stages = (200 * 1024) / stage_bytes;
+    p.stages = p.stages > 4 ? 4 : p.stages;
+    if (p.stages > nk) p.stages = nk;
+    const int smem = 1024 + p.stages * stage_bytes + (int)sizeof(WBars) + (4 + 2) * g.Dloc * 4 + 64;
+    static std::atomic<unsigned long long> raised_p{0};
+    if (cudaError_t e = raise_dynamic_smem(weights_fused_kernel<1, true>, 227 * 1024, raised_p); e != cudaSuccess) return e;
+    le = launch_dependent_cluster(weights_fused_kernel<1, true>, dim3((unsigned)(2 * tiles)), dim3(192), (size_t)smem, 2, s, tx, td,
+                                  (__nv_bfloat16*)w, (__nv_bfloat16*)wu, p, dev_status);
+    count_launch();
+    return le != cudaSuccess ? le : cudaGetLastError();
+  }
   if (fused) {
     const int stage_bytes = mblocks * 128 * 128 + ((b_rows * 128 + 1023) / 1024) * 1024;
     p.stages = (200 * 1024) / stage_bytes;
     p.stages = p.stages > 4 ? 4 : p.stages;
     if (p.stages > nk) p.stages = nk;
-    const int smem = 1024 + p.stages * stage_bytes + (int)sizeof(WBars) + (4 * mblocks + 1) * g.Dloc * 4 + 64;
+    const int smem = 1024 + p.stages * stage_bytes + (int)sizeof(WBars) + (4 * mblocks + 2) * g.Dloc * 4 + 64;
     if (mblocks == 2) {
       static std::atomic<unsigned long long> raised2{0};
       if (cudaError_t e = raise_dynamic_smem(weights_fused_kernel<2>, 227 * 1024, raised2); e != cudaSuccess) return e;
