@@ -348,6 +348,13 @@ static toma_status block_impl(const toma_desc* desc, int32_t step, const void* x
     __nv_bfloat16* y = (__nv_bfloat16*)(wsb + l.y_off);
     e = launch_quantise(g, x, y, s);
     if (e == cudaSuccess) e = launch_refresh_fused(g, y, x, idx_state, w_state, dev_status, s);
+  } else if (refresh_sel && refresh_w && weights_gram_supported(g) && !unfused) {
+    // few large tiles: the raw Gram matrix of every tile is computed on the SMs that idle during the greedy rounds
+    // (it takes the place of the quantised tokens, dead by then), and the weights are read out of it
+    float* G = (float*)(wsb + l.y_off);
+    e = do_select(g, x, idx_state, wsb, dev_status, s);
+    if (e == cudaSuccess) e = launch_gram_raw(g, x, G, dev_status, s);
+    if (e == cudaSuccess) e = launch_weights_gram(g, G, idx_state, w_state, dev_status, s);
   } else {
     if (refresh_sel) e = do_select(g, x, idx_state, wsb, dev_status, s);
     if (e == cudaSuccess && refresh_w) e = do_weights(g, x, idx_state, w_state, wsb, dev_status, s);

@@ -106,6 +106,11 @@ cudaError_t launch_attention_tc(int B, int L, int heads, int dh, const void* q, 
 // The reuse step (merge, attention over the merged tokens, unmerge) as one kernel, for the shapes it is written for.
 bool block_fused_supported(const Geom& g);
 bool block_fused_launchable(const Geom& g);
+// Merge weights out of the raw Gram matrix G = X X^T of every tile (computed on the SMs that idle during the greedy
+// rounds): launch_gram_raw goes directly behind launch_greedy, launch_weights_gram behind that.
+bool weights_gram_supported(const Geom& g);
+cudaError_t launch_gram_raw(const Geom& g, const void* x, float* G, uint32_t* dev_status, cudaStream_t s);
+cudaError_t launch_weights_gram(const Geom& g, const float* G, const int32_t* idx, void* w, uint32_t* dev_status, cudaStream_t s);
 // Selection and merge weights of 64-token tiles in one kernel (after launch_quantise), for the shapes it is written for.
 bool refresh_fused_supported(const Geom& g);
 cudaError_t launch_refresh_fused(const Geom& g, const __nv_bfloat16* y, const void* x, int32_t* idx, void* w, uint32_t* dev_status,

@@ -401,6 +401,46 @@ def test_block_steps_enqueued_back_to_back_equal_synchronised_steps(toma, name):
         assert torch.equal(a, b), f"step {t} differs"
 
 
+@pytest.mark.parametrize("over", [dict(batch=1), dict(batch=2, merge_ratio=0.25), dict(batch=1, tile_h=8, tile_w=16, merge_ratio=0.75)],
+                         ids=["128-of-256", "192-of-256", "32-of-128"])
+def test_block_weights_out_of_the_raw_gram_matrix_parity(toma, tuning, over):
+    """A refresh step on few large tiles computes X X^T of every tile on the SMs that idle during the greedy rounds
+    and reads the merge weights out of it.  Indices bit-exact, weights within 6e-4 of Sec. 4.2.1 on every tile,
+    output against the oracle; the same step forced onto the separate kernels (gather and the tensor-core logits with
+    their softmax) agrees."""
+    cfg = gen.config("cfg3", steps=1, reuse_interval=1, **over)
+    desc = toma.desc_from_config(cfg)
+    kw = dict(grid_h=cfg.grid_h, grid_w=cfg.grid_w, tile_h=cfg.tile_h, tile_w=cfg.tile_w, merge_ratio=cfg.merge_ratio,
+              tau=cfg.tau, n_heads=cfg.n_heads, reuse_interval=1)
+    x_host = next(iter(gen.feature_sequence(cfg)))
+    want, _, _ = O.block_step(x_host, 0, (st := O.BlockState()), **kw)
+    assert min(st.margins) > O.FRAGILE_MARGIN
+    ids = O.tile_token_ids(cfg.grid_h, cfg.grid_w, cfg.tile_h, cfg.tile_w)
+    dense, launches = {}, {}
+    for separate in (0, 1):
+        tuning(block_unfused=separate)
+        idx, w, ws = toma.alloc_idx(desc), toma.alloc_weights(desc), toma.alloc_workspace(desc)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        x = to_dev(x_host, cfg.dtype)
+        out = torch.full_like(x, float("nan"))
+        n0 = toma.toma_launch_counter()
+        toma.toma_block(desc, 0, x, out, idx, w, ws, status)
+        torch.cuda.synchronize()
+        launches[separate] = toma.toma_launch_counter() - n0
+        assert int(status.item()) == 0
+        assert np.array_equal(idx.cpu().numpy().astype(np.int64), st.idx)
+        assert_close(to_host64(out), want, cfg.dtype, "block output")
+        d = torch.empty((cfg.batch, cfg.n_tiles, gd(toma, cfg), cfg.n_loc), dtype=torch.float32, device="cuda")
+        toma.toma_weights_export(desc, w, d)
+        torch.cuda.synchronize()
+        dense[separate] = d.cpu().numpy().astype(np.float64)
+        for b_ in range(cfg.batch):
+            for p_ in range(cfg.n_tiles):
+                xt = x_host[b_][ids[p_]].astype(np.float64)
+                assert np.abs(dense[separate][b_, p_] - O.merge_weights(xt, st.idx[b_, p_], cfg.tau)).max() <= 6e-4, (b_, p_)
+    assert np.abs(dense[0] - dense[1]).max() <= 6e-4
+
+
 def test_small_tile_refresh_kernel_agrees_with_the_separate_kernels_on_many_inputs(toma, tuning):
     """Both forms of a refresh step on 64-token tiles work on the same integers (the fixed-point Gram) with the same
     rule (largest gain, lowest index), so their picks must be identical on any input, fragile or not; twenty seeds,
