@@ -112,8 +112,10 @@ TOMA_API uint64_t toma_launch_counter(void);
  *   attention_ctas : > 0 = number of persistent CTAs (clamped to the scratch capacity), else heuristic
  *   linear_tile    : 1 = 128 x 256, 2 = 128 x 320, 3 = 256 x 256, 4 = 128 x 128 tiles, else heuristic
  *   block_unfused  : 1 = toma_block runs merge, attention and unmerge as three kernels even for the shapes its
- *                    one-kernel reuse step covers, and selection and weights of 64-token tiles as their separate
- *                    kernels instead of one (so that both paths can be compared), else the library chooses */
+ *                    one-kernel reuse step covers, selection and weights of 64-token tiles as their separate
+ *                    kernels instead of one, and the weights of large tiles through the gather and the logits
+ *                    contraction instead of out of the raw Gram matrix (so that both paths can be compared), else
+ *                    the library chooses */
 TOMA_API void toma_test_set_tuning(int32_t attention_split, int32_t attention_ctas, int32_t linear_tile,
                                    int32_t block_unfused);
 /* TEST-ONLY (no counterpart in the paper): launches one CTA that waits, with the library's bounded wait and
