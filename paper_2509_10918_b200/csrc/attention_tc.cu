@@ -58,10 +58,11 @@ struct AttCfg {
   static constexpr int kQBytes = 2 * kQTile;               // both query tiles of a unit
   static constexpr int kKvSlab = kBN * 128;                // 64 key rows x 128 B
   static constexpr int kKvBytes = kChunks * kKvSlab;       // one K or V tile
-  static constexpr int kOnesBytes = kBN * 128;             // [64 keys][64] bf16 ones: the N chunk after V in the PV operand
-  static constexpr int kBarBytes = 512;
-  static constexpr int kSmemBytes = 1024 + kQBufs * kQBytes + 2 * kStages * kKvBytes + kOnesBytes + kBarBytes;
   static constexpr bool kSumMma = DH == 64;                // row sums on the tensor pipe, truncated P
+  static constexpr int kOnesBytes = kSumMma ? kBN * 128 : 0;  // [64 keys][64] bf16 ones: the N chunk after V in the PV operand
+  static constexpr int kOutBytes = 8 * 32 * 128;           // per softmax warp: 32 output rows of one 64-channel slab, staged for a TMA store
+  static constexpr int kBarBytes = 512;
+  static constexpr int kSmemBytes = 1024 + kQBufs * kQBytes + 2 * kStages * kKvBytes + kOnesBytes + kOutBytes + kBarBytes;
   static constexpr int kTmemCols = 512;
   // S buffer (q, b) at column (2 q + b) * 64; O_q (and, behind it, the row sums) from column 256
   static constexpr int kColS = 0, kColO = 256, kOStride = DH == 64 ? 96 : 128;
@@ -254,12 +255,58 @@ struct Row {
   int row;      // query row inside the unit, 0..255
   uint32_t ob;  // tensor-memory address of this row's accumulator
 };
+// Where a softmax warp stages its output rows, and the map they are stored through: kept out of Row (the softmax
+// loop holds a Row in registers) and derived where a piece ends.
+struct OutStage {
+  uint8_t* stage;           // this warp's 4 KB of the output staging area (it lies right below the barriers)
+  const CUtensorMap* tm_o;  // output as (channel, token, batch), box = 64 channels x 32 tokens
+};
+template <int DH>
+__device__ __forceinline__ OutStage out_stage(const void* bar, int warp, const CUtensorMap* tm_o) {
+  return OutStage{const_cast<uint8_t*>(reinterpret_cast<const uint8_t*>(bar)) - AttCfg<DH>::kOutBytes + warp * 4096, tm_o};
+}
+
+// Output rows leave through shared memory: a thread puts 32 channels of its row (scaled, bf16) into its warp's
+// staged slab (64 channels x 32 rows, 128-byte swizzled = the output map's box), and when a slab is complete the
+// warp stores it with one TMA store - whole lines instead of 16-byte stores to 32 different rows per warp
+// instruction.  Rows past the end of the sequence are clipped by the store.
+__device__ __forceinline__ void stage_half(const OutStage& os, int lane, int half, const uint32_t (&r)[32], float inv) {
+#pragma unroll
+  for (int e = 0; e < 32; e += 8) {
+    uint4 v;
+    v.x = pack_bf16_rn(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
+    v.y = pack_bf16_rn(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+    v.z = pack_bf16_rn(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+    v.w = pack_bf16_rn(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+    *reinterpret_cast<uint4*>(os.stage + sw128_offset(lane, half * 4 + (e >> 3))) = v;
+  }
+}
+// Whole warp.  (ch0, row0, b): first channel of the slab, first token of the warp's 32 rows, batch item.
+__device__ __forceinline__ void flush_slab(const OutStage& os, int lane, int ch0, int row0, int b, int L) {
+  fence_proxy_async();  // the staged rows are read by the TMA engine
+  __syncwarp();
+  if (lane == 0 && row0 < L) {
+    tma_store_3d(os.tm_o, os.stage, ch0, row0, b);
+    tma_store_commit();
+    tma_store_wait_read();  // the slab is staged again right away
+  }
+  __syncwarp();
+}
+// Batch item, first channel and first token of the 32 rows that warp t.warp holds of unit u.
+template <int DH>
+__device__ __forceinline__ void warp_rows_of(int u, const Row& t, int L, int heads, int& b, int& ch0, int& row0) {
+  const int nq = (L + kUM - 1) / kUM;
+  const int bh = u / nq;
+  b = bh / heads;
+  ch0 = (bh - b * heads) * DH;
+  row0 = (u - bh * nq) * kUM + (t.row & ~31);
+}
 
 // End of a piece that covers all keys of its unit (the only kind when units are kept whole), run by
 // the softmax warps: wait for the accumulator, normalise, write the rows out.  Returns false when
 // the wait ran out.
 template <int DH>
-__device__ __forceinline__ bool finish_whole(const Row& t, Barriers* bar, int unit, int pc, float l, __nv_bfloat16* o, int L,
+__device__ __forceinline__ bool finish_whole(const Row& t, Barriers* bar, int unit, int pc, float l, const CUtensorMap* tm_o, int L,
                                              int heads, uint32_t* dev_status) {
   using C = AttCfg<DH>;
   if (!mbar_wait(&bar->o_done[t.q], pc & 1, dev_status, &bar->abort_flag)) return false;
@@ -270,14 +317,17 @@ __device__ __forceinline__ bool finish_whole(const Row& t, Barriers* bar, int un
     tmem_wait_ld();
     l = __uint_as_float(rs[0]);
   }
-  __nv_bfloat16* dst = out_row<DH>(o, unit, t.row, L, heads);
+  int b, ch0, row0;
+  warp_rows_of<DH>(unit, t, L, heads, b, ch0, row0);
+  const OutStage os = out_stage<DH>(bar, t.warp, tm_o);
   const float inv = 1.f / l;
 #pragma unroll
   for (int c = 0; c < DH / 32; ++c) {
     uint32_t r[32];
     tmem_ld32(t.ob + c * 32, r);
     tmem_wait_ld();
-    if (dst) store_row32(dst + c * 32, r, inv);
+    stage_half(os, t.lane, c & 1, r, inv);
+    if (c & 1) flush_slab(os, t.lane, ch0 + (c >> 1) * 64, row0, b, L);
   }
   tc_fence_before();
   __syncwarp();
@@ -300,8 +350,8 @@ __device__ __forceinline__ bool finish_whole(const Row& t, Barriers* bar, int un
 // ran out.
 template <int DH>
 __device__ __noinline__ bool finish_partial(Row t, Barriers* bar, Piece p, int pc, bool last_of_span, float m_used, float l,
-                                            __nv_bfloat16* o, int L, int heads, const Spans& sp, uint32_t* tickets, float* pieces,
-                                            uint32_t* dev_status) {
+                                            __nv_bfloat16* o, const CUtensorMap* tm_o, int L, int heads, const Spans& sp,
+                                            uint32_t* tickets, float* pieces, uint32_t* dev_status) {
   using C = AttCfg<DH>;
   constexpr size_t kM = (size_t)kUM * DH, kL = (size_t)kUM * DH + kUM;
   const int row = t.row, lane = t.lane;
@@ -338,6 +388,9 @@ __device__ __noinline__ bool finish_partial(Row t, Barriers* bar, Piece p, int p
     l = __uint_as_float(rs[0]);
   }
   __nv_bfloat16* dst = out_row<DH>(o, p.u, row, L, heads);
+  int b_item, ch0, row0;
+  warp_rows_of<DH>(p.u, t, L, heads, b_item, ch0, row0);
+  const OutStage os = out_stage<DH>(bar, t.warp, tm_o);
   float* slot = pieces + (size_t)(2 * blockIdx.x + (pc > 0 ? 1 : 0)) * piece_floats<DH>();
   float w_own = 1.f, w_o = 0.f, inv = 1.f;
   if (direct) {
@@ -366,7 +419,8 @@ __device__ __noinline__ bool finish_partial(Row t, Barriers* bar, Piece p, int p
           r[4 * q + e] = __float_as_uint(own_first ? fmaf(w_o, vv[e], w_own * own) : fmaf(w_own, own, w_o * vv[e]));
         }
       }
-      if (dst) store_row32(dst + c * 32, r, inv);
+      stage_half(os, t.lane, c & 1, r, inv);
+      if (c & 1) flush_slab(os, t.lane, ch0 + (c >> 1) * 64, row0, b_item, L);
     } else {
 #pragma unroll
       for (int e = 0; e < 32; e += 4)
@@ -418,7 +472,8 @@ __device__ __noinline__ bool softmax_tile_ragged(uint32_t sb, uint32_t ob, float
 template <int DH>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                    const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, int L, int heads,
+                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                    __nv_bfloat16* __restrict__ o, int L, int heads,
                     float scale_log2, const __grid_constant__ Spans sp, uint32_t* __restrict__ tickets, float* __restrict__ pieces,
                     uint32_t* dev_status) {
   using C = AttCfg<DH>;
@@ -428,7 +483,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   uint8_t* sK = sQ + C::kQBufs * C::kQBytes;
   uint8_t* sV = sK + C::kStages * C::kKvBytes;
   uint8_t* sOnes = sV + C::kStages * C::kKvBytes;
-  Barriers* bar = reinterpret_cast<Barriers*>(sOnes + C::kOnesBytes);
+  uint8_t* sOut = sOnes + C::kOnesBytes;
+  Barriers* bar = reinterpret_cast<Barriers*>(sOut + C::kOutBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nblk = sp.nblk;
@@ -465,6 +521,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     prefetch_tmap(&tm_q);
     prefetch_tmap(&tm_k);
     prefetch_tmap(&tm_v);
+    prefetch_tmap(&tm_o);
   }
   dependency_wait();
   if (threadIdx.x == 0) release_dependents();
@@ -655,8 +712,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (lane == 0) mbar_arrive(&bar->p_full[t.q][b]);
       }
       if (!ok) break;
-      if (p.cnt == nblk) ok = finish_whole<DH>(t, bar, p.u, pc, l, o, L, heads, dev_status);
-      else ok = finish_partial<DH>(t, bar, p, pc, it >= it_end, m_used, l, o, L, heads, sp, tickets, pieces, dev_status);
+      if (p.cnt == nblk) ok = finish_whole<DH>(t, bar, p.u, pc, l, &tm_o, L, heads, dev_status);
+      else ok = finish_partial<DH>(t, bar, p, pc, it >= it_end, m_used, l, o, &tm_o, L, heads, sp, tickets, pieces, dev_status);
     }
     if (ok) settle_first_piece<DH>(bar, it_begin, it_end, t, o, L, heads, sp, pieces, dev_status);
   }
@@ -767,13 +824,14 @@ template <int DH>
 cudaError_t launch(int B, int L, int heads, const void* q, const void* k, const void* v, void* o, void* ws,
                    bool tickets_clean, uint32_t* dev_status, cudaStream_t s) {
   using C = AttCfg<DH>;
-  CUtensorMap tq, tk, tv;
+  CUtensorMap tq, tk, tv, to;
   const uint64_t dims[3] = {(uint64_t)heads * DH, (uint64_t)L, (uint64_t)B};
   const uint64_t strides[2] = {(uint64_t)heads * DH * 2, (uint64_t)L * heads * DH * 2};
   const uint32_t box_q[3] = {64, kBM, 1};
   const uint32_t box_kv[3] = {64, kBN, 1};
+  const uint32_t box_o[3] = {64, 32, 1};  // a softmax warp's 32 rows of one 64-channel slab
   if (!encode_tmap_16bit(&tq, q, 3, dims, strides, box_q) || !encode_tmap_16bit(&tk, k, 3, dims, strides, box_kv) ||
-      !encode_tmap_16bit(&tv, v, 3, dims, strides, box_kv))
+      !encode_tmap_16bit(&tv, v, 3, dims, strides, box_kv) || !encode_tmap_16bit(&to, o, 3, dims, strides, box_o))
     return cudaErrorInvalidValue;
   static std::atomic<unsigned long long> smem_raised{0};
   cudaError_t e = raise_dynamic_smem(attention_tc_kernel<DH>, C::kSmemBytes, smem_raised);
@@ -788,7 +846,7 @@ cudaError_t launch(int B, int L, int heads, const void* q, const void* k, const 
     if (e != cudaSuccess) return e;
   }
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  e = launch_dependent(attention_tc_kernel<DH>, dim3(sp.G), dim3(kThreads), (size_t)C::kSmemBytes, s, tq, tk, tv,
+  e = launch_dependent(attention_tc_kernel<DH>, dim3(sp.G), dim3(kThreads), (size_t)C::kSmemBytes, s, tq, tk, tv, to,
                        (__nv_bfloat16*)o, L, heads, scale_log2, sp, (uint32_t*)ws, (float*)((char*)ws + tb), dev_status);
   if (e != cudaSuccess) return e;
   count_launch();
