@@ -744,7 +744,7 @@ constexpr int kSplitCostTiles = 4;
 
 // What a piece costs its CTA beyond its key tiles, in half tiles: the pipeline drains, the accumulator is read
 // out and (partial pieces) goes through scratch, tickets and the addition of the unit's pieces.
-constexpr int kPieceCostWhole = 4, kPieceCostPartial = 7;
+constexpr int kPieceCostWhole = 4, kPieceCostPartial = 9;
 
 // The farthest end of a span that starts at iteration `start` and costs at most C half tiles
 // (2 per key tile plus the piece costs above); `start` itself when not even one tile fits.
