@@ -105,6 +105,7 @@ cudaError_t launch_attention_tc(int B, int L, int heads, int dh, const void* q, 
                                 void* ws, bool tickets_clean, uint32_t* dev_status, cudaStream_t s);
 // The reuse step (merge, attention over the merged tokens, unmerge) as one kernel, for the shapes it is written for.
 bool block_fused_supported(const Geom& g);
+// ... and this device holds its launch (host-side occupancy query, cached per device).
 bool block_fused_launchable(const Geom& g);
 // Merge weights out of the raw Gram matrix G = X X^T of every tile (computed on the SMs that idle during the greedy
 // rounds): launch_gram_raw goes directly behind launch_greedy, launch_weights_gram behind that.
@@ -115,7 +116,6 @@ cudaError_t launch_weights_gram(const Geom& g, const float* G, const int32_t* id
 bool refresh_fused_supported(const Geom& g);
 cudaError_t launch_refresh_fused(const Geom& g, const __nv_bfloat16* y, const void* x, int32_t* idx, void* w, uint32_t* dev_status,
                                  cudaStream_t s);
-//  // this device holds its launch (host-side query, cached per device)
 cudaError_t launch_block_fused(const Geom& g, const void* w, const void* x, void* out, uint32_t* dev_status, cudaStream_t s);
 // Image-level destination ids [batch][D] (tile-major, pick order) from the tile-local picks.
 cudaError_t launch_global_idx(const Geom& g, const int32_t* idx, int32_t* gidx, cudaStream_t s);
