@@ -83,7 +83,7 @@ struct Barriers {
 static_assert(sizeof(Barriers) <= 512, "barrier block outgrew its reservation");
 
 constexpr int kSnapTiles = 2;
-constexpr int kMaxCtas = 160;  // scratch and the span table are sized for this many persistent CTAs
+constexpr int kMaxCtas = 160;  // scratch and the span table are sized for this many persistent CTAs (ids fit a byte)
 
 // The iterations [0, T) are cut into G contiguous spans, CTA g running [bounds[g], bounds[g + 1]).
 // With whole units every bound is a multiple of nblk (no scratch traffic), which wins when the unit
@@ -93,6 +93,10 @@ constexpr int kMaxCtas = 160;  // scratch and the span table are sized for this 
 struct Spans {
   int T, G, nblk, split;
   int bounds[kMaxCtas + 1];
+  // Lowest and highest CTA among those whose spans hold key tiles of the unit CTA g's span starts in ([0][g])
+  // and of the unit it ends in ([1][g]): the only units a CTA can share.  Filled in by the host, so that the
+  // kernel does not search the bounds at the end of a piece.
+  uint8_t unit_lo[2][kMaxCtas], unit_hi[2][kMaxCtas];
   __host__ __device__ int bound(int g) const { return bounds[g]; }
   // the CTA whose span holds iteration `it`
   __host__ __device__ int owner(int it) const {
@@ -281,6 +285,18 @@ __device__ __forceinline__ void stage_half(const OutStage& os, int lane, int hal
     *reinterpret_cast<uint4*>(os.stage + sw128_offset(lane, half * 4 + (e >> 3))) = v;
   }
 }
+// The same for 16 channels (quarter 0..3 of the slab's 64).
+__device__ __forceinline__ void stage_quarter(const OutStage& os, int lane, int quarter, const uint32_t (&r)[16], float inv) {
+#pragma unroll
+  for (int e = 0; e < 16; e += 8) {
+    uint4 v;
+    v.x = pack_bf16_rn(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
+    v.y = pack_bf16_rn(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+    v.z = pack_bf16_rn(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+    v.w = pack_bf16_rn(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+    *reinterpret_cast<uint4*>(os.stage + sw128_offset(lane, quarter * 2 + (e >> 3))) = v;
+  }
+}
 // Whole warp.  (ch0, row0, b): first channel of the slab, first token of the warp's 32 rows, batch item.
 __device__ __forceinline__ void flush_slab(const OutStage& os, int lane, int ch0, int row0, int b, int L) {
   fence_proxy_async();  // the staged rows are read by the TMA engine
@@ -356,11 +372,18 @@ __device__ __noinline__ bool finish_partial(Row t, Barriers* bar, Piece p, int p
   constexpr size_t kM = (size_t)kUM * DH, kL = (size_t)kUM * DH + kUM;
   const int row = t.row, lane = t.lane;
   uint32_t* ticket = tickets + (size_t)p.u * 8 + t.warp;
-  const int g_first = sp.owner(p.u * sp.nblk), g_last = sp.owner((p.u + 1) * sp.nblk - 1);
+  // a partial piece lies in the unit the span starts in or in the one it ends in
+  const int which = p.u == sp.bound(blockIdx.x) / sp.nblk ? 0 : 1;
+  const int g_first = sp.unit_lo[which][blockIdx.x], g_last = sp.unit_hi[which][blockIdx.x];
   bool own_first = false;  // this CTA is the lower of the two contributors
+  // The direct path comes in two forms.  The wide one holds 64 columns of the other piece in registers (the
+  // function then spills); the lean one takes 16 columns at a time with the next 16 on their way.  Timed as a
+  // whole, the kernel is 3-4 % faster with the lean form at head_dim 128 and 5-7 % slower at head_dim 64, where
+  // the register allocation of the tile loop changes with this function's needs: each keeps the form that wins.
+  constexpr bool kLean = DH == 128;
   const float* other = nullptr;
   float m_o = 0.f, l_o = 0.f;
-  float4 vo[16];
+  float4 vo[kLean ? 4 : 16];
   // the publisher warp watches the tickets of the span's last unit; its answer carries the
   // acquire that orders the loads below after the other contributor's writes
   uint32_t others = 0;
@@ -377,7 +400,7 @@ __device__ __noinline__ bool finish_partial(Row t, Barriers* bar, Piece p, int p
     m_o = __ldcg(other + kM + row);
     l_o = __ldcg(other + kL + row);
 #pragma unroll
-    for (int q = 0; q < 16; ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)q * kUM + row);
+    for (int q = 0; q < (kLean ? 4 : 16); ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)q * kUM + row);
   }
   if (!mbar_wait(&bar->o_done[t.q], pc & 1, dev_status, &bar->abort_flag)) return false;
   tc_fence_after();
@@ -399,33 +422,74 @@ __device__ __noinline__ bool finish_partial(Row t, Barriers* bar, Piece p, int p
     w_o = ex2_mufu(m_o - M);
     inv = 1.f / (own_first ? fmaf(w_o, l_o, w_own * l) : fmaf(w_own, l, w_o * l_o));
   }
+  // rows of the piece into its scratch slot (32 columns at a time)
+  auto to_scratch = [&](int c, const uint32_t (&r)[32]) {
 #pragma unroll
-  for (int c = 0; c < DH / 32; ++c) {
-    uint32_t r[32];
-    tmem_ld32(t.ob + c * 32, r);
-    tmem_wait_ld();
+    for (int e = 0; e < 32; e += 4)
+      reinterpret_cast<float4*>(slot)[(size_t)(c * 8 + (e >> 2)) * kUM + row] =
+          make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+  };
+  if constexpr (kLean) {
     if (direct) {
-      if (c > 0 && (c & 1) == 0) {  // next 64 columns of the other piece
 #pragma unroll
-        for (int q = 0; q < 16; ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)(c * 8 + q) * kUM + row);
-      }
+      for (int c = 0; c < DH / 16; ++c) {
+        float4 vc[4];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) {
-        const float4 v = vo[(c & 1) * 8 + q];
-        const float vv[4] = {v.x, v.y, v.z, v.w};
+        for (int q = 0; q < 4; ++q) vc[q] = vo[q];
+        if (c + 1 < DH / 16) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float own = __uint_as_float(r[4 * q + e]);
-          r[4 * q + e] = __float_as_uint(own_first ? fmaf(w_o, vv[e], w_own * own) : fmaf(w_own, own, w_o * vv[e]));
+          for (int q = 0; q < 4; ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)((c + 1) * 4 + q) * kUM + row);
         }
+        uint32_t r[16];
+        tmem_ld16(t.ob + c * 16, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float vv[4] = {vc[q].x, vc[q].y, vc[q].z, vc[q].w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float own = __uint_as_float(r[4 * q + e]);
+            r[4 * q + e] = __float_as_uint(own_first ? fmaf(w_o, vv[e], w_own * own) : fmaf(w_own, own, w_o * vv[e]));
+          }
+        }
+        stage_quarter(os, t.lane, c & 3, r, inv);
+        if ((c & 3) == 3) flush_slab(os, t.lane, ch0 + (c >> 2) * 64, row0, b_item, L);
       }
-      stage_half(os, t.lane, c & 1, r, inv);
-      if (c & 1) flush_slab(os, t.lane, ch0 + (c >> 1) * 64, row0, b_item, L);
     } else {
 #pragma unroll
-      for (int e = 0; e < 32; e += 4)
-        reinterpret_cast<float4*>(slot)[(size_t)(c * 8 + (e >> 2)) * kUM + row] =
-            make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+      for (int c = 0; c < DH / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32(t.ob + c * 32, r);
+        tmem_wait_ld();
+        to_scratch(c, r);
+      }
+    }
+  } else {
+#pragma unroll
+    for (int c = 0; c < DH / 32; ++c) {
+      uint32_t r[32];
+      tmem_ld32(t.ob + c * 32, r);
+      tmem_wait_ld();
+      if (direct) {
+        if (c > 0 && (c & 1) == 0) {  // next 64 columns of the other piece
+#pragma unroll
+          for (int q = 0; q < 16; ++q) vo[q] = __ldcg(reinterpret_cast<const float4*>(other) + (size_t)(c * 8 + q) * kUM + row);
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const float4 v = vo[(c & 1) * 8 + q];
+          const float vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float own = __uint_as_float(r[4 * q + e]);
+            r[4 * q + e] = __float_as_uint(own_first ? fmaf(w_o, vv[e], w_own * own) : fmaf(w_own, own, w_o * vv[e]));
+          }
+        }
+        stage_half(os, t.lane, c & 1, r, inv);
+        if (c & 1) flush_slab(os, t.lane, ch0 + (c >> 1) * 64, row0, b_item, L);
+      } else {
+        to_scratch(c, r);
+      }
     }
   }
   tc_fence_before();
@@ -453,7 +517,7 @@ __device__ __noinline__ void settle_first_piece(Barriers* bar, int it_begin, int
   const int nblk = sp.nblk, u = it_begin / nblk;
   const bool first_partial = it_begin > u * nblk || it_end < (u + 1) * nblk;
   if (!first_partial || it_end <= (u + 1) * nblk) return;  // whole, or also the span's last piece: settled already
-  const int g_first = sp.owner(u * nblk), g_last = sp.owner((u + 1) * nblk - 1);
+  const int g_first = sp.unit_lo[0][blockIdx.x], g_last = sp.unit_hi[0][blockIdx.x];
   if (!mbar_wait(&bar->pub_done, 0, dev_status, &bar->abort_flag)) return;
   if (bar->first_ticket[t.warp] != (uint32_t)(g_last - g_first)) return;
   __threadfence();
@@ -668,7 +732,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       // straight from tensor memory if the answer is there when their last piece ends, and go
       // through scratch and tickets otherwise.  Polling keeps the ticket out of their registers.
       const int ul = (it_end - 1) / nblk;
-      if (it_end < (ul + 1) * nblk && sp.owner((ul + 1) * nblk - 1) == sp.owner(ul * nblk) + 1) {
+      if (it_end < (ul + 1) * nblk && sp.unit_hi[1][blockIdx.x] == sp.unit_lo[1][blockIdx.x] + 1) {
         const uint32_t* tk = tickets + (size_t)ul * 8;
         for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
           if ((*(volatile uint32_t*)&bar->poll_stop[0] && *(volatile uint32_t*)&bar->poll_stop[1]) || *abort_flag) break;
@@ -744,7 +808,7 @@ constexpr int kSplitCostTiles = 4;
 
 // What a piece costs its CTA beyond its key tiles, in half tiles: the pipeline drains, the accumulator is read
 // out and (partial pieces) goes through scratch, tickets and the addition of the unit's pieces.
-constexpr int kPieceCostWhole = 4, kPieceCostPartial = 9;
+constexpr int kPieceCostWhole = 4, kPieceCostPartial = 8;
 
 // The farthest end of a span that starts at iteration `start` and costs at most C half tiles
 // (2 per key tile plus the piece costs above); `start` itself when not even one tile fits.
@@ -785,7 +849,7 @@ int cut_spans(int T, int nblk, long long C, int gmax, int* bounds) {
 // small beside it), else so that the longest span, pieces' costs included, is as short as possible (the
 // smallest budget C for which a left-to-right cut needs no more spans than there are CTAs).
 Spans plan_spans(int units, int nblk) {
-  Spans sp;
+  Spans sp = {};
   sp.nblk = nblk;
   sp.T = units * nblk;
   const int gmax = max_ctas();
@@ -816,6 +880,13 @@ Spans plan_spans(int units, int nblk) {
       else lo = mid + 1;
     }
     sp.G = cut_spans(sp.T, nblk, lo, gmax, sp.bounds);
+  }
+  for (int g = 0; g < sp.G; ++g) {
+    const int unit[2] = {sp.bounds[g] / nblk, (sp.bounds[g + 1] - 1) / nblk};
+    for (int e = 0; e < 2; ++e) {
+      sp.unit_lo[e][g] = (uint8_t)sp.owner(unit[e] * nblk);
+      sp.unit_hi[e][g] = (uint8_t)sp.owner((unit[e] + 1) * nblk - 1);
+    }
   }
   return sp;
 }

@@ -145,13 +145,13 @@ def test_attention_work_plan_covers_every_key_tile_once(toma, shape, split):
             assert off == 0 or off > 2, "a bound sits within two tiles of a unit boundary"
         assert plan["owner_first"] == list(range(plan["ctas"])) and plan["owner_last"] == list(range(plan["ctas"]))
     elif plan["split"]:
-        # short spans: the longest span, charged 2 per key tile plus 4 per whole-unit piece and 9 per partial piece
+        # short spans: the longest span, charged 2 per key tile plus 4 per whole-unit piece and 8 per partial piece
         # (half tiles), is as short as a left-to-right cut into at most 148 spans can make it
         def cost(lo, hi):
             c, it = 0, lo
             while it < hi:
                 end = min(hi, (it // nblk + 1) * nblk)
-                c += 2 * (end - it) + (4 if (it % nblk == 0 and end % nblk == 0) else 9)
+                c += 2 * (end - it) + (4 if (it % nblk == 0 and end % nblk == 0) else 8)
                 it = end
             return c
 
