@@ -20,16 +20,48 @@ __device__ __forceinline__ float ex2_mufu(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// 2^x for x <= ~9 on the FMA pipe: round to nearest integer with the 1.5*2^23 trick, degree-3
+// Two floats in one 64-bit register and the packed fp32 arithmetic of sm_100 on them (one issue slot for two
+// results on the FMA pipe).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t v;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+  return v;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// 2^x for x <= ~9 on the FMA pipe, two at a time: round to nearest integer with the 1.5*2^23 trick, degree-3
 // near-minimax polynomial for 2^f on [-0.5, 0.5], exponent patched in with an integer add.
-__device__ __forceinline__ float ex2_poly(float x) {
-  x = fmaxf(x, -126.f);
-  const float t = x + 12582912.f;
-  const float f = x - (t - 12582912.f);
-  float p = fmaf(0.0551716648f, f, 0.2426111251f);
-  p = fmaf(p, f, 0.6932609677f);
-  p = fmaf(p, f, 0.9999280572f);
-  return __int_as_float(__float_as_int(p) + (int)((unsigned)__float_as_int(t) << 23));
+__device__ __forceinline__ void ex2_poly2(uint64_t x2, float& p0, float& p1) {
+  float x0, x1;
+  unpack2(x2, x0, x1);
+  x2 = pack2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+  const uint64_t k2 = pack2(12582912.f, 12582912.f);
+  const uint64_t t2 = add2(x2, k2);
+  const uint64_t f2 = sub2(x2, sub2(t2, k2));
+  uint64_t q2 = fma2(pack2(0.0551716648f, 0.0551716648f), f2, pack2(0.2426111251f, 0.2426111251f));
+  q2 = fma2(q2, f2, pack2(0.6932609677f, 0.6932609677f));
+  q2 = fma2(q2, f2, pack2(0.9999280572f, 0.9999280572f));
+  float q0, q1, t0, t1;
+  unpack2(q2, q0, q1);
+  unpack2(t2, t0, t1);
+  p0 = __int_as_float(__float_as_int(q0) + (int)((unsigned)__float_as_int(t0) << 23));
+  p1 = __int_as_float(__float_as_int(q1) + (int)((unsigned)__float_as_int(t1) << 23));
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
@@ -70,10 +102,17 @@ __device__ __forceinline__ float chunk_exp(const uint32_t (&r)[32], uint32_t (&p
   float l = 0.f;
 #pragma unroll
   for (int e = 0; e < 32; e += 2) {
-    const float x0 = fmaf(__uint_as_float(r[e]), scale, neg_m);
-    const float x1 = fmaf(__uint_as_float(r[e + 1]), scale, neg_m);
-    float p0 = ex2_mufu(x0);
-    float p1 = (e & 2) ? ex2_poly(x1) : ex2_mufu(x1);  // every fourth exponential on the FMA pipe
+    // S * c - m for a pair of columns in one packed multiply-add
+    const uint64_t x2 = fma2(pack2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), pack2(scale, scale), pack2(neg_m, neg_m));
+    float p0, p1;
+    if ((e & 6) == 6) {  // every fourth pair of exponentials on the FMA pipe
+      ex2_poly2(x2, p0, p1);
+    } else {
+      float x0, x1;
+      unpack2(x2, x0, x1);
+      p0 = ex2_mufu(x0);
+      p1 = ex2_mufu(x1);
+    }
     if (kMask) {
       if (first + e >= valid) p0 = 0.f;
       if (first + e + 1 >= valid) p1 = 0.f;
