@@ -28,10 +28,10 @@
 //                             the normalised result
 //   running maximum        -> O (and the row sums) are rescaled only when the maximum grew by more
 //                             than 2^8; the final division by the row sum makes a stale maximum exact
-//   exponentials           -> one pair of columns in four goes through a degree-3 polynomial on the FMA
-//                             pipe (relative error 7.5e-5, far below bf16 resolution of P), the rest
-//                             through MUFU ex2; the scaling S*c - m and the polynomial run in packed
-//                             f32x2 arithmetic (one issue slot for two columns)
+//   exponentials           -> one pair of columns in four (three in eight at head_dim 128) goes through
+//                             a degree-3 polynomial on the FMA pipe (relative error 7.5e-5, far below
+//                             bf16 resolution of P), the rest through MUFU ex2; the scaling S*c - m and
+//                             the polynomial run in packed f32x2 arithmetic (one issue slot for two columns)
 // The whole S row of a tile (64 fp32) is fetched with one tensor-memory round trip and kept in
 // registers for both the maximum and the exponentials.
 // Keys past the sequence end are zero-filled by TMA and masked out; query rows past the end are
